@@ -1,0 +1,19 @@
+"""CPU oracle of the HGF linear-layer forward pass: test infrastructure, never the product path.
+
+Only the tests, the smoke check and the benchmark's cpu-baseline leg import this package.
+"""
+from .hgf_oracle import (  # noqa: F401
+    FLAG_NO_SILU,
+    act_quant,
+    build,
+    effective_bits,
+    forward,
+    gamma_w,
+    int_gemm,
+    pack,
+    packed_bytes,
+    ternarise,
+    threads,
+    tmax,
+    unpack,
+)

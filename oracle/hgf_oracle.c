@@ -1,0 +1,234 @@
+/*
+ * CPU oracle for the forward pass of the Hybrid Gated Flow (HGF) dual-stream linear layer.
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, scalar restatement of the
+ * paper's definitions (Section 2.2 "Ternary Weight Quantization", Section 2.2.1 "Activation
+ * Quantization", Section 2.3 "Gated Low-Rank Correction", Algorithm 1 "HGF 1.0 Forward Pass").
+ * Only the tests, the smoke check and the benchmark's cpu-baseline leg may call it.  It shares no
+ * code, header, table or helper with the CUDA library; the packed-weight layout is re-implemented
+ * here from its written description (two bits per weight, see oracle_pack below).
+ *
+ * Precision: every real-valued quantity is a C double; integer quantities are int32/int64.
+ * Loops are written in the order of the definitions; the only concession to run time is one
+ * OpenMP "parallel for" over independent output rows, which changes no arithmetic.
+ *
+ * Pins (tests/test_oracle_pins.py): numpy float64 mean(|W|); threshold invariants and crafted
+ * +-gamma/2 ties; pack/unpack round trips; int8 invariants, crafted rounding ties; brute-force
+ * integer matmul on tiny shapes and numpy int64 matmul; gate = 0 reduces to the pure ternary
+ * layer; hand-worked 2x2 correction; SiLU-off equals (x A) B; the fake-quant float restatement;
+ * the paper's T_max worked example (7B, FP16, 500 GB/s -> 35.7 tokens/s).
+ * No function here is "parity unpinned".
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_FLAG_NO_SILU 1u /* correction is (x A) B instead of SiLU(x A) B */
+
+/* ---- exact decoding of the 16-bit input encodings ------------------------------------------ */
+
+/* bfloat16: the upper 16 bits of an IEEE-754 binary32. */
+static double bf16_to_double(uint16_t h) {
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* IEEE-754 binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static double fp16_to_double(uint16_t h) {
+    int sign = (h >> 15) & 1;
+    int e = (h >> 10) & 0x1f;
+    int f = h & 0x3ff;
+    double v;
+    if (e == 0)
+        v = ldexp((double)f, -24); /* zero and subnormals: f * 2^-10 * 2^-14 */
+    else if (e == 31)
+        v = f ? NAN : INFINITY;
+    else
+        v = ldexp(1.0 + (double)f / 1024.0, e - 15);
+    return sign ? -v : v;
+}
+
+int oracle_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ---- Section 2.2, weight scale: gamma_W = (1/(m n)) sum_ij |W_ij| ---------------------------- */
+/* Summed in double in index order, rounded once to binary32 (the stored scale is one fp32). */
+float oracle_gamma_w(const float *W, int64_t d_out, int64_t d_in) {
+    double acc = 0.0;
+    for (int64_t i = 0; i < d_out * d_in; ++i) acc += fabs((double)W[i]);
+    return (float)(acc / (double)(d_out * d_in));
+}
+
+/* ---- Section 2.2, ternary codes: Clip(Round(W / gamma_W), -1, 1) ------------------------------ */
+/* Round-to-nearest of W/gamma followed by the clip has decision boundaries at +-gamma/2 (the
+ * paper states these boundaries); a value exactly on a boundary is a tie between 0 and +-1 and
+ * round-half-to-even sends it to 0.  gamma/2 is exact in binary32, so the comparison is exact. */
+void oracle_ternarise(const float *W, int64_t d_out, int64_t d_in, float gamma, int8_t *T) {
+    double half = (double)gamma / 2.0;
+    for (int64_t i = 0; i < d_out * d_in; ++i) {
+        double w = (double)W[i];
+        T[i] = (w > half) ? 1 : (w < -half) ? -1 : 0;
+    }
+}
+
+/* ---- packed layout (the paper only says "1.58-bit"; two bits per weight are used) ------------ */
+/* Row n of the matrix occupies d_in/4 bytes starting at byte n*d_in/4.  A row is a sequence of
+ * little-endian 32-bit words; word i holds the 16 weights k = 16 i .. 16 i + 15.  Writing
+ * k = 16 i + 4 j + b with j, b in 0..3, the weight's code c = t + 1 (0, 1 or 2; 3 is never
+ * written) sits in bits 8 b + 2 j and 8 b + 2 j + 1 of word i. */
+int64_t oracle_packed_bytes(int64_t d_out, int64_t d_in) { return d_out * d_in / 4; }
+
+void oracle_pack(const int8_t *T, int64_t d_out, int64_t d_in, uint8_t *packed) {
+    int64_t words_per_row = d_in / 16;
+    for (int64_t n = 0; n < d_out; ++n)
+        for (int64_t i = 0; i < words_per_row; ++i) {
+            uint32_t word = 0;
+            for (int j = 0; j < 4; ++j)
+                for (int b = 0; b < 4; ++b) {
+                    int t = T[n * d_in + 16 * i + 4 * j + b];
+                    uint32_t c = (uint32_t)(t + 1);
+                    word |= c << (8 * b + 2 * j);
+                }
+            uint8_t *dst = packed + (n * words_per_row + i) * 4;
+            dst[0] = (uint8_t)(word & 0xff);
+            dst[1] = (uint8_t)((word >> 8) & 0xff);
+            dst[2] = (uint8_t)((word >> 16) & 0xff);
+            dst[3] = (uint8_t)((word >> 24) & 0xff);
+        }
+}
+
+/* Returns the number of invalid codes (value 3) met; those decode to 0. */
+int64_t oracle_unpack(const uint8_t *packed, int64_t d_out, int64_t d_in, int8_t *T) {
+    int64_t words_per_row = d_in / 16, bad = 0;
+    for (int64_t n = 0; n < d_out; ++n)
+        for (int64_t i = 0; i < words_per_row; ++i) {
+            const uint8_t *src = packed + (n * words_per_row + i) * 4;
+            uint32_t word = (uint32_t)src[0] | ((uint32_t)src[1] << 8) | ((uint32_t)src[2] << 16) |
+                            ((uint32_t)src[3] << 24);
+            for (int j = 0; j < 4; ++j)
+                for (int b = 0; b < 4; ++b) {
+                    uint32_t c = (word >> (8 * b + 2 * j)) & 3u;
+                    if (c == 3u) { ++bad; c = 1u; }
+                    T[n * d_in + 16 * i + 4 * j + b] = (int8_t)((int)c - 1);
+                }
+        }
+    return bad;
+}
+
+/* ---- Section 2.2.1 / Algorithm 1 steps 1-2: per-token absmax int8 quantisation --------------- */
+/* gamma_x = max_k |x_k| (floored at 1e-5 so that an all-zero token does not divide by zero; the
+ * floored value is used for both quantisation and dequantisation);
+ * x~_k = Clip(Round(x_k / gamma_x * 127), -127, 127), Round = nearest, ties to even, of the
+ * exact quotient.  127*x is exact in double for a bf16 x, so one correctly rounded division
+ * followed by rint() yields the exact result. */
+void oracle_act_quant(const uint16_t *x_bf16, int64_t M, int64_t d_in, int8_t *xq, float *gamma_x) {
+    for (int64_t m = 0; m < M; ++m) {
+        double amax = 0.0;
+        for (int64_t k = 0; k < d_in; ++k) {
+            double a = fabs(bf16_to_double(x_bf16[m * d_in + k]));
+            if (a > amax) amax = a;
+        }
+        float g = (float)amax; /* exact: a bf16 value is a binary32 value */
+        if (g < 1e-5f) g = 1e-5f;
+        gamma_x[m] = g;
+        for (int64_t k = 0; k < d_in; ++k) {
+            double q = rint(127.0 * bf16_to_double(x_bf16[m * d_in + k]) / (double)g);
+            if (q > 127.0) q = 127.0;
+            if (q < -127.0) q = -127.0;
+            xq[m * d_in + k] = (int8_t)q;
+        }
+    }
+}
+
+/* ---- Algorithm 1 step 3: Y_int = X~ (int8)  x  W~^T (ternary), integer arithmetic ------------- */
+/* Returns 0, or 1 if any sum left the int32 range (it cannot for d_in < 2^24). */
+int oracle_int_gemm(const int8_t *xq, const int8_t *T, int64_t M, int64_t d_out, int64_t d_in,
+                    int32_t *y_int) {
+    int overflow = 0;
+#pragma omp parallel for schedule(static) reduction(| : overflow)
+    for (int64_t n = 0; n < d_out; ++n)
+        for (int64_t m = 0; m < M; ++m) {
+            int64_t acc = 0;
+            for (int64_t k = 0; k < d_in; ++k)
+                acc += (int64_t)xq[m * d_in + k] * (int64_t)T[n * d_in + k];
+            if (acc > INT32_MAX || acc < INT32_MIN) overflow |= 1;
+            y_int[m * d_out + n] = (int32_t)acc;
+        }
+    return overflow;
+}
+
+static double silu(double z) { return z / (1.0 + exp(-z)); } /* z * sigmoid(z) */
+
+/* ---- Algorithm 1, whole layer ----------------------------------------------------------------- */
+/* y[m][n] = Y_int[m][n] * gamma_x[m] * gamma_W / 127  +  g[n] * sum_j SiLU(sum_k x[m][k] A[k][j]) B[j][n]
+ *
+ * Storage: x [M][d_in] bf16 bits; T [d_out][d_in] int8 ternary codes; At [r][d_in] fp16 bits
+ * (the transpose of the paper's A); Bt [d_out][r] fp16 bits (the transpose of the paper's B);
+ * gate [d_out] fp32 (the evaluated g = tanh(alpha), one value per output channel; the paper's
+ * scalar gate is the constant vector); y [M][d_out] double.  r = 0 or a null gate gives the pure
+ * ternary layer.  Optional outputs (nullable): xq_out [M][d_in], gamma_x_out [M],
+ * y_int_out [M][d_out], h_out [M][r] double (after the activation). */
+int oracle_forward(const uint16_t *x_bf16, int64_t M, const int8_t *T, float gamma_w, int64_t d_in,
+                   int64_t d_out, const uint16_t *At_fp16, const uint16_t *Bt_fp16, int32_t r,
+                   const float *gate, uint32_t flags, double *y, int8_t *xq_out, float *gamma_x_out,
+                   int32_t *y_int_out, double *h_out, int8_t *xq_scratch, float *gx_scratch,
+                   int32_t *yint_scratch, double *h_scratch) {
+    int8_t *xq = xq_out ? xq_out : xq_scratch;
+    float *gx = gamma_x_out ? gamma_x_out : gx_scratch;
+    int32_t *yi = y_int_out ? y_int_out : yint_scratch;
+    double *H = h_out ? h_out : h_scratch;
+    int have_corr = (r > 0 && At_fp16 && Bt_fp16 && gate);
+
+    /* Path 1: structural backbone. */
+    oracle_act_quant(x_bf16, M, d_in, xq, gx);
+    int overflow = oracle_int_gemm(xq, T, M, d_out, d_in, yi);
+
+    /* Path 2: H = SiLU(X A). */
+    if (have_corr) {
+#pragma omp parallel for schedule(static)
+        for (int64_t m = 0; m < M; ++m)
+            for (int32_t j = 0; j < r; ++j) {
+                double z = 0.0;
+                for (int64_t k = 0; k < d_in; ++k)
+                    z += bf16_to_double(x_bf16[m * d_in + k]) * fp16_to_double(At_fp16[(int64_t)j * d_in + k]);
+                H[m * r + j] = (flags & ORACLE_FLAG_NO_SILU) ? z : silu(z);
+            }
+    }
+
+    /* Dequantise, Y_corr = H B, gated fusion. */
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < d_out; ++n)
+        for (int64_t m = 0; m < M; ++m) {
+            double y_tern = (double)yi[m * d_out + n] * ((double)gx[m] * (double)gamma_w / 127.0);
+            double y_corr = 0.0;
+            if (have_corr) {
+                for (int32_t j = 0; j < r; ++j)
+                    y_corr += H[m * r + j] * fp16_to_double(Bt_fp16[n * r + j]);
+                y_corr *= (double)gate[n];
+            }
+            y[m * d_out + n] = y_tern + y_corr;
+        }
+    return overflow;
+}
+
+/* ---- Introduction, memory-wall bound: T_max = B_mem / (P * b / 8) tokens per second ----------- */
+double oracle_tmax(double bmem_bytes_per_s, double params, double bits_per_param) {
+    return bmem_bytes_per_s / (params * bits_per_param / 8.0);
+}
+
+/* ---- Section 4.2, effective bit-width: b_eff = log2(3) + g * b_corr * r / d -------------------- */
+double oracle_effective_bits(double g, double b_corr, double r, double d) {
+    return log2(3.0) + g * b_corr * r / d;
+}
