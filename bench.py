@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the HGF linear-layer forward pass on B200.
+
+A step is one pass of the whole hot path (activation quantisation, LoRA down-projection, packed
+ternary GEMV/GEMM, fused dequantisation + gated correction) over every layer of the workload.
+
+Headline workload (N = 1): decode, M = 1, over the seven projections of a 1.2B-class block
+(d = 2048, FFN 5632, r = 32) replicated over enough distinct weight copies that the working set
+is > 4x the 126 MB L2, so the weight stream really comes from HBM.  The metric is algorithmic
+bytes per second (packed W + A + B + gate + x + y).  Further lines of evidence (other token counts,
+the 7B-class stack, prefill TOPS) are reported under "extra".
+
+`--impl reference` times the CPU oracle (test infrastructure, as it stands) on the same metric.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "HGF layer HBM GB/s (M=1 decode)"
+UNIT = "GB/s"
+L2_BYTES = 126e6
+
+
+def layer_bytes(K, N, r, M, out_bytes=4):
+    """Algorithmic bytes one layer call must move: packed W, A, B, gate, x, y."""
+    return K * N // 4 + 2 * r * (K + N) + 4 * N + 2 * M * K + out_bytes * M * N
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d.get("hbm_gbs", 6650.0), "bf16_tflops": d.get("bf16_tflops", 1590.0),
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", 1400.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------ GPU arm
+class Workload:
+    """A list of independent layer problems with everything resident on the device."""
+
+    def __init__(self, hgf, torch, shapes, M, copies, flags=0, seed=0, host_io=False):
+        self.hgf, self.torch, self.M, self.flags = hgf, torch, M, flags
+        dev = torch.device("cuda")
+        g = torch.Generator(device=dev)
+        g.manual_seed(seed)
+        out_dt = torch.bfloat16 if flags & hgf.FLAG_OUT_BF16 else torch.float32
+        self.layers = []
+        x_elems = sum(M * s.d_in for s in shapes) * copies
+        y_elems = sum(M * s.d_out for s in shapes) * copies
+        self.x_all = torch.empty(x_elems, dtype=torch.bfloat16, device=dev)
+        self.y_all = torch.empty(y_elems, dtype=out_dt, device=dev)
+        xo = yo = 0
+        self.bytes = 0
+        self.ops = 0
+        ws_bytes = max(hgf.workspace_bytes(M, s.d_in, s.d_out, s.r, flags) for s in shapes)
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        for c in range(copies):
+            for s in shapes:
+                W = torch.randn((s.d_out, s.d_in), generator=g, device=dev, dtype=torch.float32) * 0.02
+                packed, gamma = hgf.pack_ternary(W)
+                del W
+                At = (torch.randn((s.r, s.d_in), generator=g, device=dev) / s.d_in ** 0.5).to(torch.float16)
+                Bt = (torch.randn((s.d_out, s.r), generator=g, device=dev) / s.r ** 0.5).to(torch.float16)
+                gate = torch.rand(s.d_out, generator=g, device=dev)
+                x = self.x_all[xo:xo + M * s.d_in].view(M, s.d_in)
+                xf = torch.randn((M, s.d_in), generator=g, device=dev)
+                ch = torch.randperm(s.d_in, generator=g, device=dev)[: int(0.02 * s.d_in)]
+                xf[:, ch] *= 20.0
+                x.copy_(xf.to(torch.bfloat16))
+                y = self.y_all[yo:yo + M * s.d_out].view(M, s.d_out)
+                xo += M * s.d_in
+                yo += M * s.d_out
+                self.layers.append((s, x, packed, gamma, At, Bt, gate, y))
+                self.bytes += layer_bytes(s.d_in, s.d_out, s.r, M, 2 if flags & hgf.FLAG_OUT_BF16 else 4)
+                self.ops += 2 * M * s.d_in * s.d_out
+        self.weight_bytes = sum(l[2].numel() + l[4].numel() * 2 + l[5].numel() * 2 for l in self.layers)
+        self.graph = None
+        self.launches_per_step = 0
+        if host_io:
+            self.x_host = torch.empty(x_elems, dtype=torch.bfloat16).pin_memory()
+            self.x_host.copy_(self.x_all)
+            self.y_host = torch.empty(y_elems, dtype=out_dt).pin_memory()
+
+    def enqueue(self, stream):
+        for (s, x, packed, gamma, At, Bt, gate, y) in self.layers:
+            self.hgf.linear_forward(x, packed, gamma, s.d_in, s.d_out, At, Bt, gate, y=y, workspace=self.ws,
+                                    flags=self.flags, stream=stream)
+
+    def capture(self, stream):
+        torch = self.torch
+        with torch.cuda.stream(stream):
+            self.enqueue(stream)           # first call outside capture: one-time set-up happens here
+            stream.synchronize()
+            before = self.hgf.launch_count()
+            self.graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(self.graph, stream=stream):
+                self.enqueue(stream)
+            self.launches_per_step = self.hgf.launch_count() - before
+        stream.synchronize()
+
+    def time_steps(self, stream, steps, warmup, e2e=False):
+        """Milliseconds per step, CUDA events on the launching stream."""
+        torch = self.torch
+        with torch.cuda.stream(stream):
+            def one():
+                if e2e:
+                    self.x_all.copy_(self.x_host, non_blocking=True)
+                self.graph.replay()
+                if e2e:
+                    self.y_host.copy_(self.y_all, non_blocking=True)
+            for _ in range(warmup):
+                one()
+            stream.synchronize()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record(stream)
+            for _ in range(steps):
+                one()
+            t1.record(stream)
+            stream.synchronize()
+        return t0.elapsed_time(t1) / steps
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2602_05269_b200 import hgf, inputs as syn
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    hgf.lib()
+    stream = torch.cuda.Stream()
+    peaks = measured_peaks()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- headline: config 1 decode, M = 1 -------------------------------------------------------
+    shapes1 = syn.CONFIGS[1]["layers"]
+    block_bytes = sum(layer_bytes(s.d_in, s.d_out, s.r, 1) for s in shapes1)
+    copies = int(np.ceil(4.4 * L2_BYTES / block_bytes))
+    main = Workload(hgf, torch, shapes1, 1, copies, host_io=True)
+    main.capture(stream)
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    ms = main.time_steps(stream, args.steps, args.warmup)
+    barrier()
+    clocks = sampler.stop()
+    ms = max_over_ranks(ms)
+    ms_e2e = max_over_ranks(main.time_steps(stream, max(args.steps // 4, 1), args.warmup, e2e=True))
+    value = world * main.bytes / (ms * 1e-3) / 1e9
+    value_e2e = world * main.bytes / (ms_e2e * 1e-3) / 1e9
+
+    n_layers = len(main.layers)
+    per_launch_bytes = main.bytes / n_layers
+    per_launch_us = ms * 1e3 / n_layers
+    roofline = {"bound": "hbm", "kernel": "decode_gemv_kernel (+ its prologue launch)",
+                "achieved": per_launch_bytes / (per_launch_us * 1e-6) / 1e9, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": None, "traffic": None, "peak_source": peaks["source"],
+                "bytes_per_launch": per_launch_bytes, "us_per_launch": per_launch_us,
+                "frac_of_nominal_8000": None}
+    roofline["frac"] = roofline["achieved"] / roofline["peak"]
+    roofline["frac_of_nominal_8000"] = roofline["achieved"] / 8000.0
+    traffic_file = os.path.join(ROOT, "profiles", "decode_gemv_traffic.json")
+    if os.path.exists(traffic_file):
+        roofline["traffic"] = json.load(open(traffic_file)).get("dram_bytes_per_launch_scaled")
+
+    extra = {}
+    if rank == 0 and not args.quick:
+        extra = run_extra(hgf, torch, syn, stream, args, peaks)
+
+    cpu = cpu_baseline(10.0) if (rank == 0 and world == 1 and not args.no_cpu) else None
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8 x ternary (int32 accumulate) + fp16 correction",
+            "data": "synthetic",
+            "config": {"workload": "config1: 1.2B-class block (d=2048, FFN 5632, r=32), 7 projections x "
+                                   f"{copies} distinct weight copies, decode M=1, one hgf_linear_forward per layer, "
+                                   "CUDA-graph chained",
+                       "layers_per_step": n_layers, "weight_bytes": main.weight_bytes,
+                       "l2_policy": "inputs larger than L2 (weight working set %.0f MB > 4 x 126 MB)"
+                                    % (main.weight_bytes / 1e6),
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "e2e": {"value": value_e2e, "unit": UNIT, "h2d_bytes_per_step": main.x_host.numel() * 2,
+                    "d2h_bytes_per_step": main.y_host.numel() * main.y_host.element_size()},
+            "gpu_launches": main.launches_per_step * args.steps,
+            "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu, "extra": extra,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_extra(hgf, torch, syn, stream, args, peaks):
+    """Secondary measurements, same timing rules, each with its own workload."""
+    extra = {"decode": [], "prefill": []}
+    steps = max(args.steps // 4, 10)
+
+    def decode_case(cfg, shapes, M, label, min_copies=1):
+        block = sum(layer_bytes(s.d_in, s.d_out, s.r, M) for s in shapes)
+        copies = max(min_copies, int(np.ceil(4.4 * L2_BYTES / block)))
+        w = Workload(hgf, torch, shapes, M, copies)
+        w.capture(stream)
+        ms = w.time_steps(stream, steps, args.warmup)
+        gbs = w.bytes / (ms * 1e-3) / 1e9
+        row = {"workload": label, "M": M, "layers": len(w.layers), "ms_per_step": ms, "GB/s": gbs,
+               "frac_measured_peak": gbs / peaks["hbm_gbs"], "frac_nominal_8000": gbs / 8000.0}
+        del w
+        torch.cuda.empty_cache()
+        return row
+
+    for M in (4, 16):
+        extra["decode"].append(decode_case(1, syn.CONFIGS[1]["layers"], M, "config1 1.2B-class block"))
+    for M in (1, 8):
+        extra["decode"].append(decode_case(2, syn.CONFIGS[2]["layers"], M, "config2 3B-class block"))
+    # config 4: the 7B-class stack, 32 blocks x 7 projections, decode M = 1 -> tokens/s
+    row = decode_case(4, syn.CONFIGS[4]["layers"], 1, "config4 7B-class stack (32 blocks)", min_copies=32)
+    params = 32 * sum(s.d_in * s.d_out for s in syn.CONFIGS[4]["layers"])
+    tok_s = 1e3 / row["ms_per_step"] * (32 * 7 / row["layers"])
+    row.update({"tokens_per_s": tok_s, "params": params,
+                "tmax_2bit_measured_bw": hgf.tmax_tokens_per_s(peaks["hbm_gbs"] * 1e9, params, 2.0),
+                "tmax_1p58bit_measured_bw": hgf.tmax_tokens_per_s(peaks["hbm_gbs"] * 1e9, params, 1.58),
+                "tmax_2bit_8TBs": hgf.tmax_tokens_per_s(8e12, params, 2.0),
+                "tmax_1p58bit_8TBs": hgf.tmax_tokens_per_s(8e12, params, 1.58)})
+    extra["decode"].append(row)
+
+    # prefill: config 3 shapes, bf16 output
+    int8_peak_nominal = 4500.0
+    int8_peak_2x_bf16 = 2.0 * peaks["bf16_tflops"]
+    for M in (512, 2048, 8192):
+        for s in syn.distinct_shapes(3):
+            w = Workload(hgf, torch, [s], M, 1, flags=hgf.FLAG_OUT_BF16)
+            w.capture(stream)
+            psteps = max(10, min(200, int(2e11 / w.ops) * 10))
+            ms = w.time_steps(stream, psteps, args.warmup)
+            tops = w.ops / (ms * 1e-3) / 1e12
+            extra["prefill"].append({"shape": f"{s.d_in}->{s.d_out}", "r": s.r, "M": M, "ms": ms, "TOPS": tops,
+                                     "frac_nominal_4500": tops / int8_peak_nominal,
+                                     "frac_2x_measured_bf16": tops / int8_peak_2x_bf16})
+            del w
+            torch.cuda.empty_cache()
+    return extra
+
+
+# ----------------------------------------------------------------------------------- CPU arms
+def cpu_baseline(budget_s: float):
+    """The oracle, as it stands, on this host's cores, on a bounded sample of the headline workload."""
+    import oracle
+    from paper_2602_05269_b200 import inputs as syn
+
+    shapes = syn.distinct_shapes(1)
+    probs = []
+    for i, s in enumerate(shapes):
+        L = syn.make_layer(s, 1, config=1, layer=i)
+        g = oracle.gamma_w(L["W"])
+        probs.append((s, L, oracle.ternarise(L["W"], g), g))
+    nbytes = 0
+    reps = 0
+    t0 = time.perf_counter()
+    while True:
+        for s, L, T, g in probs:
+            oracle.forward(L["x"], T, g, L["At"], L["Bt"], L["gate"])
+            nbytes += layer_bytes(s.d_in, s.d_out, s.r, 1)
+        reps += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "host_cores": os.cpu_count(),
+            "sample": f"{reps} passes over one layer of each distinct config-1 shape "
+                      "(2048->2048, 2048->5632, 5632->2048, r=32) at M=1; bytes are the same algorithmic "
+                      "bytes as the GPU metric (the oracle itself reads unpacked int8 codes)"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps, warm = max(args.steps, 1), max(args.warmup, 0)
+    per_step = max(0.05, min(2.0, 90.0 / (steps + warm)))
+    for _ in range(warm):
+        cpu_baseline(per_step)
+    vals = []
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        vals.append(cpu_baseline(per_step))
+    dt = time.perf_counter() - t0
+    v = float(np.mean([c["value"] for c in vals]))
+    cb = dict(vals[-1])
+    cb["value"] = v
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": steps, "warmup": warm, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64 / int64 (CPU oracle)", "data": "synthetic",
+        "config": {"workload": "config1 decode M=1, bounded sample: one layer of each distinct shape per pass"},
+        "cpu_baseline": cb,
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--quick", action="store_true", help="headline measurement only")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,143 @@
+/*
+ * hgf.h - C ABI of the B200 (sm_100a) forward pass of the Hybrid Gated Flow dual-stream linear layer.
+ *
+ * The layer (paper, Algorithm 1 "HGF 1.0 Forward Pass (Inference Mode)"):
+ *
+ *     gamma_x[m] = max_k |x[m][k]|                                   (per-token scale)
+ *     xq[m][k]   = Clip(Round(x[m][k] / gamma_x[m] * 127), -127, 127)   (int8)
+ *     Y_int      = xq  x  T^T            T in {-1,0,1}^(d_out x d_in)   (integer GEMM)
+ *     Y_tern     = Y_int * gamma_x[m] * gamma_W / 127
+ *     H          = SiLU(x A)             A in R^(d_in x r)
+ *     Y_corr     = H B                   B in R^(r x d_out)
+ *     y          = Y_tern + g * Y_corr
+ *
+ * Conventions for every call
+ *   - Plain C ABI, no exceptions; every call that can fail returns an hgf_status.
+ *   - Unless a parameter says "host", tensor pointers are DEVICE pointers owned by the caller.
+ *     The library never frees, keeps or reallocates them.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Forward calls only
+ *     enqueue work and return without synchronising; they allocate nothing.
+ *   - All tensors are dense and row-major; all device pointers must be 16-byte aligned.
+ *   - The library is CUDA-only: there is no CPU fallback.  Without a usable device a call
+ *     returns HGF_ERR_CUDA.
+ */
+#ifndef HGF_H
+#define HGF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HGF_OK = 0,
+    HGF_ERR_INVALID_ARG = 1,       /* null pointer, non-positive size, unknown flag */
+    HGF_ERR_UNSUPPORTED_SHAPE = 2, /* d_in % 64 != 0, r not in {0,16,32,48,64}, M too large, ... */
+    HGF_ERR_MISALIGNED = 3,        /* a device pointer is not 16-byte aligned */
+    HGF_ERR_WORKSPACE = 4,         /* workspace missing or smaller than hgf_workspace_bytes() */
+    HGF_ERR_CUDA = 5,              /* a CUDA runtime/driver call failed (launch error, no device) */
+    HGF_ERR_TIMEOUT = 6            /* a bounded device-side wait gave up (reported by hgf_check_status) */
+} hgf_status;
+
+/* flags of hgf_linear_forward / hgf_workspace_bytes */
+#define HGF_FLAG_OUT_BF16 0x1u /* y is bfloat16 instead of fp32 */
+#define HGF_FLAG_NO_SILU 0x2u  /* correction is (x A) B, without the SiLU the paper defines */
+#define HGF_FLAG_FORCE_GEMM 0x4u /* route to the tensor-core GEMM path even when M <= 16 (testing) */
+
+/* Largest token count the register-resident decode path handles; above it the GEMM path runs. */
+#define HGF_DECODE_MAX_M 16
+
+/* Optional copies of intermediate results, for parity checks.  Device pointers, each nullable. */
+typedef struct {
+    int8_t *xq;      /* [M][d_in]   quantised activations (Algorithm 1, step 2) */
+    float *gamma_x;  /* [M]         per-token scales, after the 1e-5 floor (step 1) */
+    int32_t *y_int;  /* [M][d_out]  integer accumulators sum_k xq[m][k] T[n][k] (step 3) */
+    float *h;        /* [M][r]      SiLU(x A) (steps 5-6) */
+} hgf_debug_out;
+
+/*
+ * Size in bytes of the packed form of a d_out x d_in ternary matrix: d_out * d_in / 4.
+ * Packed layout (the paper fixes none; it only states 1.58 bits of information per weight):
+ * two bits per weight, code c = t + 1 in {0,1,2}.  Row n occupies d_in/4 bytes from byte
+ * n * d_in / 4.  A row is a sequence of little-endian 32-bit words; word i holds weights
+ * k = 16 i .. 16 i + 15, and with k = 16 i + 4 j + b (j, b in 0..3) the code of weight k is in
+ * bits 8 b + 2 j and 8 b + 2 j + 1.  So (word >> 2 j) & 0x03030303 is four consecutive-k codes,
+ * one per byte.  Returns 0 for invalid sizes (d_in % 64 != 0 or non-positive).
+ */
+size_t hgf_packed_bytes(int64_t d_out, int64_t d_in);
+
+/*
+ * Offline weight preparation (paper, Definition "Absmax Quantization", Section 2.2):
+ *     gamma_W = mean |W|,  t = Clip(Round(W / gamma_W), -1, 1)   (boundaries at +-gamma_W/2,
+ *     a weight exactly on a boundary becomes 0), then 2-bit packing as above.
+ * W: device, fp32 [d_out][d_in].  packed: device, hgf_packed_bytes(d_out, d_in) bytes.
+ * gamma_out: HOST pointer, receives gamma_W (sum in double, rounded once to fp32).
+ * This call allocates a small temporary, synchronises `stream` and is not meant for the hot path.
+ * Requires d_in % 64 == 0.
+ */
+hgf_status hgf_pack_ternary(const float *W, int64_t d_out, int64_t d_in, void *packed,
+                            float *gamma_out, void *stream);
+
+/* Inverse of the packing: T[n][k] in {-1,0,1} as int8, device [d_out][d_in].  Enqueue only. */
+hgf_status hgf_unpack_ternary(const void *packed, int64_t d_out, int64_t d_in, int8_t *T,
+                              void *stream);
+
+/* Bytes of caller-provided scratch hgf_linear_forward needs for this problem (never 0). */
+size_t hgf_workspace_bytes(int64_t M, int64_t d_in, int64_t d_out, int32_t r, uint32_t flags);
+
+/*
+ * The layer forward pass (paper, Algorithm 1; Definitions "Dynamic Activation Quantization",
+ * "Low-Rank Correction", "Gated Fusion").
+ *
+ *   x       [M][d_in]      bfloat16
+ *   packed  from hgf_pack_ternary, gamma = its gamma_W
+ *   At      [r][d_in]      fp16: the transpose of the paper's A (d_in contiguous)
+ *   Bt      [d_out][r]     fp16: the transpose of the paper's B (r contiguous)
+ *   gate    [d_out]        fp32: the evaluated gate g = tanh(alpha), one value per output
+ *                          channel (the paper's scalar gate is the constant vector)
+ *   y       [M][d_out]     fp32, or bfloat16 with HGF_FLAG_OUT_BF16
+ *   workspace              device scratch of at least hgf_workspace_bytes(...) bytes, 256-byte
+ *                          aligned; holds xq, gamma_x, row sums and H between the kernels
+ *   dbg                    nullable; see hgf_debug_out
+ *
+ * r = 0, or any of At/Bt/gate null, computes the pure ternary layer (Y_tern only).
+ * The per-token scale is floored at 1e-5 (an all-zero token yields zeros).
+ * Requirements: M >= 1; d_in % 64 == 0; d_out >= 1; r in {0,16,32,48,64}; 16-byte aligned
+ * pointers.  M <= HGF_DECODE_MAX_M runs the bandwidth-bound GEMV path, larger M the tcgen05
+ * int8 GEMM path (which additionally needs d_in % 128 == 0 and d_out % 8 == 0).
+ * Calls on the same workspace must not overlap on the device.
+ */
+hgf_status hgf_linear_forward(const void *x, int64_t M, const void *packed, float gamma,
+                              int64_t d_in, int64_t d_out, const void *At, const void *Bt,
+                              int32_t r, const float *gate, void *y, void *workspace,
+                              size_t workspace_bytes, const hgf_debug_out *dbg, uint32_t flags,
+                              void *stream);
+
+/*
+ * Step a1 alone (paper, Definition "Dynamic Activation Quantization"): xq, gamma_x and the row
+ * sums sum_k xq[m][k] (row_sum nullable).  Enqueue only.
+ */
+hgf_status hgf_act_quant(const void *x, int64_t M, int64_t d_in, int8_t *xq, float *gamma_x,
+                         int32_t *row_sum, void *stream);
+
+/*
+ * Device-side waits in the GEMM path are bounded; when one gives up the kernel records it and
+ * returns.  This call synchronises `stream`, reads and clears that record, and returns
+ * HGF_ERR_TIMEOUT if a wait gave up since the last check (HGF_OK otherwise).
+ */
+hgf_status hgf_check_status(void *stream);
+
+/* Memory-wall bound of the paper's introduction: T_max = B_mem / (P * b / 8) tokens/s. */
+double hgf_tmax_tokens_per_s(double bmem_bytes_per_s, double params, double bits_per_param);
+
+/* Kernels launched by this library in this process so far (for launch accounting). */
+uint64_t hgf_launch_count(void);
+
+const char *hgf_status_string(hgf_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HGF_H */

@@ -1,0 +1,498 @@
+// GEMM path (M > 16 tokens): Y_int = X~ x T^T on the 5th-generation tensor cores
+// (tcgen05.mma kind::i8, int32 accumulators in tensor memory), with the dequantisation, the
+// LoRA up-projection (a second, small tcgen05.mma kind::f16 into an fp32 accumulator) and the
+// gated fusion in the epilogue.  Algorithm 1, steps 3, 4, 7, 8.
+//
+// One persistent CTA per SM, 10 warps with fixed roles:
+//   warp 0      TMA producer: per 128-wide k block, the int8 activation tile (128 tokens x 128 B,
+//               128-byte swizzle) and the packed weight tile (256 rows x 32 B)
+//   warp 1      allocates tensor memory; one lane issues the MMAs and commits to mbarriers
+//   warps 2-5   epilogue: stage the LoRA operands of the tile, then read both accumulators with
+//               tcgen05.ld, combine, and write through shared memory with TMA stores
+//   warps 6-9   expand the 2-bit codes of a packed tile into the int8, K-major, 128-byte-swizzled
+//               operand layout the tensor core reads from shared memory
+// The tile is 128 tokens (MMA M) x 256 output channels (MMA N).  Codes are c = t + 1 (unsigned
+// operand); sum_k t x~ = sum_k c x~ - sum_k x~ is restored in the epilogue from the row sums.
+//
+// Every wait is bounded: when one gives up, the CTA records it in the device status word, all
+// roles leave their loops, in-flight bulk copies are drained, tensor memory is freed and the
+// kernel returns.
+#include <cuda.h>
+
+#include "hgf_common.cuh"
+
+namespace hgf {
+
+constexpr int TILE_M = 128, TILE_N = 256, KBLK = 128;
+constexpr int XSTAGES = 3, BSTAGES = 2;
+constexpr int X_TILE_BYTES = TILE_M * KBLK;      // 16 KiB
+constexpr int P_TILE_BYTES = TILE_N * KBLK / 4;  // 8 KiB
+constexpr int B_TILE_BYTES = TILE_N * KBLK;      // 32 KiB
+constexpr int LORA_A_BYTES = TILE_M * 128;       // 128 tokens x 64 fp16
+constexpr int LORA_B_BYTES = TILE_N * 128;       // 256 channels x 64 fp16
+constexpr int STORE_BUF_BYTES = 32 * 128;        // 32 rows x 128 B per epilogue warp and buffer
+constexpr int GEMM_THREADS = 320;
+constexpr int TMEM_COLS = 512, TMEM_COL_INT = 0, TMEM_COL_FP = 256;
+
+constexpr int OFF_X = 0;
+constexpr int OFF_B = OFF_X + XSTAGES * X_TILE_BYTES;
+constexpr int OFF_LA = OFF_B + BSTAGES * B_TILE_BYTES;
+constexpr int OFF_LB = OFF_LA + LORA_A_BYTES;
+constexpr int OFF_ST = OFF_LB + LORA_B_BYTES;
+constexpr int OFF_P = OFF_ST + 4 * 2 * STORE_BUF_BYTES;
+constexpr int OFF_GATE = OFF_P + XSTAGES * P_TILE_BYTES;
+constexpr int OFF_BAR = OFF_GATE + 4 * TILE_N * 4;  // one gate copy per epilogue warp
+constexpr int SMEM_USED = OFF_BAR + 256;
+constexpr int SMEM_BYTES = SMEM_USED + 1024;  // slack for the 1024-byte alignment of the base
+
+// barrier slots (8 bytes each) inside the OFF_BAR block
+enum { BAR_FULL = 0, BAR_EMPTY = BAR_FULL + XSTAGES, BAR_BFULL = BAR_EMPTY + XSTAGES,
+       BAR_BEMPTY = BAR_BFULL + BSTAGES, BAR_ACCFULL = BAR_BEMPTY + BSTAGES, BAR_ACCEMPTY,
+       BAR_LORAFULL, BAR_COUNT };
+static_assert(BAR_COUNT * 8 + 16 <= 256, "barrier block too small");
+
+constexpr uint32_t kSpinLimit = 1u << 22;  // bounded waits: about a second at worst
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if it gave up or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned int *status, unsigned int code) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicExch(status, code);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int x, int y, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];\n"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;\n" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mma_i8(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_f16(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: register i of lane l = TMEM[lane base + l][col + i]
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, groups of 8 rows
+// 1024 bytes apart.  Fields: start address >> 4 (bits 0-13), leading byte offset >> 4 (16-29,
+// unused for this layout, set to 1), stride byte offset >> 4 (32-45), version 1 (46-47),
+// layout type 2 = 128-byte swizzle (61-63).
+__device__ __forceinline__ uint64_t make_sw128_desc(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+// Instruction descriptor: D format (bits 4-5), A format (7-9), B format (10-12), K-major A and B,
+// N >> 3 (17-22), M >> 4 (24-28).
+constexpr uint32_t IDESC_I8 = (2u << 4) /*s32*/ | (1u << 7) /*A signed*/ | (0u << 10) /*B unsigned*/ |
+                              ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+constexpr uint32_t IDESC_F16 = (1u << 4) /*f32*/ | (0u << 7) /*A f16*/ | (0u << 10) /*B f16*/ |
+                               ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+
+template <bool OUT_BF16>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                    const __grid_constant__ CUtensorMap tmap_y, const GemmParams p, unsigned int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + OFF_BAR;
+    auto bar = [&](int i) { return bar0 + 8u * i; };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + OFF_BAR + BAR_COUNT * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_BAR + BAR_COUNT * 8 + 4);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tiles_m = (p.M + TILE_M - 1) / TILE_M, tiles_n = (p.N + TILE_N - 1) / TILE_N;
+    const int num_tiles = tiles_m * tiles_n;
+    const int kblocks = (p.K + KBLK - 1) / KBLK;
+    const bool has_lora = p.r > 0;
+
+    if (tid == 0) {
+        for (int s = 0; s < XSTAGES; ++s) {
+            mbar_init(bar(BAR_FULL + s), 1);
+            mbar_init(bar(BAR_EMPTY + s), 1 + 4);  // MMA commit + four unpack warps
+        }
+        for (int u = 0; u < BSTAGES; ++u) {
+            mbar_init(bar(BAR_BFULL + u), 4);
+            mbar_init(bar(BAR_BEMPTY + u), 1);
+        }
+        mbar_init(bar(BAR_ACCFULL), 1);
+        mbar_init(bar(BAR_ACCEMPTY), 4);
+        mbar_init(bar(BAR_LORAFULL), 4);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        fence_proxy_async();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            uint32_t issued[XSTAGES] = {0, 0, 0};
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int m0 = (tile % tiles_m) * TILE_M, n0 = (tile / tiles_m) * TILE_N;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!(ok = mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x100u + s))) break;
+                    mbar_arrive_expect_tx(bar(BAR_FULL + s), X_TILE_BYTES + P_TILE_BYTES);
+                    tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, m0, bar(BAR_FULL + s));
+                    tma_load_2d(sbase + OFF_P + s * P_TILE_BYTES, &tmap_w, kb * (KBLK / 4), n0, bar(BAR_FULL + s));
+                    ++issued[s];
+                    if (++s == XSTAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+            // drain: wait (bounded) until every copy this thread issued has landed, so that the CTA
+            // never exits with a bulk copy in flight (immediate when the consumers ran to the end)
+            for (int q = 0; q < XSTAGES; ++q)
+                if (issued[q]) {
+                    const uint32_t par = (issued[q] - 1u) & 1u;
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_FULL + q), par); ++i) {}
+                }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int s = 0, u = 0;
+            uint32_t ph = 0, bph = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+                if (it > 0 && !(ok = mbar_wait(bar(BAR_ACCEMPTY), (uint32_t)(it - 1) & 1u, abort_flag, status, 0x200u)))
+                    break;
+                tc_fence_after();
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!(ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag, status, 0x210u + s))) break;
+                    if (!(ok = mbar_wait(bar(BAR_BFULL + u), bph, abort_flag, status, 0x220u + u))) break;
+                    tc_fence_after();
+                    const uint64_t adesc = make_sw128_desc(sbase + OFF_X + s * X_TILE_BYTES);
+                    const uint64_t bdesc = make_sw128_desc(sbase + OFF_B + u * B_TILE_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < KBLK / 32; ++kk)
+                        mma_i8(tmem_base + TMEM_COL_INT, adesc + 2u * kk, bdesc + 2u * kk, IDESC_I8,
+                               (kb | kk) ? 1u : 0u);
+                    tc_commit(bar(BAR_EMPTY + s));
+                    tc_commit(bar(BAR_BEMPTY + u));
+                    if (++s == XSTAGES) { s = 0; ph ^= 1u; }
+                    if (++u == BSTAGES) { u = 0; bph ^= 1u; }
+                }
+                if (!ok) break;
+                if (has_lora) {
+                    if (!(ok = mbar_wait(bar(BAR_LORAFULL), (uint32_t)it & 1u, abort_flag, status, 0x230u))) break;
+                    tc_fence_after();
+                    const uint64_t adesc = make_sw128_desc(sbase + OFF_LA);
+                    const uint64_t bdesc = make_sw128_desc(sbase + OFF_LB);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)  // 64 fp16 = 4 x (K = 16)
+                        mma_f16(tmem_base + TMEM_COL_FP, adesc + 2u * kk, bdesc + 2u * kk, IDESC_F16, kk ? 1u : 0u);
+                }
+                tc_commit(bar(BAR_ACCFULL));
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------------ epilogue warps
+        const int e = warp - 2;          // staging role index
+        const int q = warp & 3;          // TMEM lane quarter this warp may read
+        uint8_t *stbuf = smem + OFF_ST + e * 2 * STORE_BUF_BYTES;
+        float *gate_s = reinterpret_cast<float *>(smem + OFF_GATE) + e * TILE_N;
+        const float gw = p.gw_over_127;
+        constexpr int ES = OUT_BF16 ? 2 : 4;
+        constexpr int COLS_PER_STORE = 128 / ES;  // 32 fp32 or 64 bf16 columns per 128-byte row
+        bool ok = true;
+        int it = 0, sbuf = 0;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+            const int m0 = (tile % tiles_m) * TILE_M, n0 = (tile / tiles_m) * TILE_N;
+            if (has_lora) {
+                // H tile: rows 32 e .. 32 e + 31, 8 chunks of 16 bytes each
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int idx = i * 32 + lane, row = 32 * e + idx / 8, c = idx % 8, m = m0 + row;
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (m < p.M) v = *reinterpret_cast<const uint4 *>(p.h16 + (size_t)m * 64 + c * 8);
+                    *reinterpret_cast<uint4 *>(smem + OFF_LA + row * 128 + ((c ^ (row & 7)) << 4)) = v;
+                }
+                // B^T tile: rows 64 e .. 64 e + 63
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int idx = i * 32 + lane, row = 64 * e + idx / 8, c = idx % 8, n = n0 + row;
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (n < p.N && c * 8 < p.r) v = *reinterpret_cast<const uint4 *>(p.Bt + (size_t)n * p.r + c * 8);
+                    *reinterpret_cast<uint4 *>(smem + OFF_LB + row * 128 + ((c ^ (row & 7)) << 4)) = v;
+                }
+#pragma unroll
+                for (int i = 0; i < TILE_N / 32; ++i) {  // this warp's own copy of the tile's gate values
+                    const int col = 32 * i + lane, n = n0 + col;
+                    gate_s[col] = n < p.N ? p.gate[n] : 0.0f;
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_LORAFULL));
+            }
+
+            const int m = m0 + 32 * q + lane;  // this thread's token = its TMEM lane
+            const float scale = m < p.M ? p.gamma_x[m] * gw : 0.0f;
+            const int rs = m < p.M ? p.row_sum[m] : 0;
+
+            ok = mbar_wait(bar(BAR_ACCFULL), (uint32_t)it & 1u, abort_flag, status, 0x300u);
+            if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
+            tc_fence_after();
+            const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16);
+
+            for (int c0 = 0; c0 < TILE_N; c0 += COLS_PER_STORE) {
+                uint8_t *buf = stbuf + sbuf * STORE_BUF_BYTES;
+                // the buffer was handed to a TMA store two stores ago: wait until it was read
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
+#pragma unroll
+                for (int sub = 0; sub < COLS_PER_STORE / 32; ++sub) {
+                    const int cc = c0 + 32 * sub;
+                    uint32_t ai[32], af[32];
+                    tmem_ld32(lane_base + TMEM_COL_INT + cc, ai);
+                    if (has_lora) tmem_ld32(lane_base + TMEM_COL_FP + cc, af);
+                    tmem_ld_wait();
+                    float yv[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int yi = (int)ai[j] - rs;
+                        float y = (float)yi * scale;
+                        if (has_lora) y = fmaf(gate_s[cc + j], __uint_as_float(af[j]), y);
+                        yv[j] = y;
+                        ai[j] = (uint32_t)yi;
+                    }
+                    if (p.dbg_y_int && m < p.M) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + cc + j < p.N) p.dbg_y_int[(size_t)m * p.N + n0 + cc + j] = (int)ai[j];
+                    }
+                    if (OUT_BF16) {
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {  // 8 bf16 per 16-byte chunk
+                            uint32_t w[4];
+#pragma unroll
+                            for (int h = 0; h < 4; ++h) {
+                                __nv_bfloat162 b2 = __floats2bfloat162_rn(yv[8 * ch + 2 * h], yv[8 * ch + 2 * h + 1]);
+                                w[h] = *reinterpret_cast<uint32_t *>(&b2);
+                            }
+                            const int chunk = 4 * sub + ch;
+                            *reinterpret_cast<uint4 *>(buf + lane * 128 + ((chunk ^ (lane & 7)) << 4)) =
+                                make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int ch = 0; ch < 8; ++ch)  // 4 fp32 per 16-byte chunk
+                            *reinterpret_cast<uint4 *>(buf + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
+                                make_uint4(__float_as_uint(yv[4 * ch]), __float_as_uint(yv[4 * ch + 1]),
+                                           __float_as_uint(yv[4 * ch + 2]), __float_as_uint(yv[4 * ch + 3]));
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&tmap_y, n0 + c0, m0 + 32 * q, smem_u32(buf));
+                    bulk_commit();
+                }
+                sbuf ^= 1;
+            }
+            // all TMEM reads of this tile are done: hand the accumulators back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_ACCEMPTY));
+        }
+        if (lane == 0) bulk_wait_read<0>();
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ unpack warps
+        const int ut = tid - 6 * 32;  // 0..127
+        int s = 0, u = 0;
+        uint32_t ph = 0, bph = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            for (int kb = 0; kb < kblocks; ++kb) {
+                ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag, status, 0x400u + s) &&
+                     mbar_wait(bar(BAR_BEMPTY + u), bph ^ 1u, abort_flag, status, 0x410u + u);
+                if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
+                const uint8_t *psrc = smem + OFF_P + s * P_TILE_BYTES;
+                uint8_t *bdst = smem + OFF_B + u * B_TILE_BYTES;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int idx = i * 128 + ut;          // 16-byte piece of the packed tile
+                    const int row = idx >> 1, half = idx & 1;  // 32 packed bytes per row
+                    const uint4 pk = *reinterpret_cast<const uint4 *>(psrc + idx * 16);
+                    const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
+#pragma unroll
+                    for (int qd = 0; qd < 4; ++qd) {
+                        // word qd holds 16 consecutive k; (w >> 2 j) & 0x03030303 = k 4 j .. 4 j + 3
+                        const uint4 o = make_uint4(w[qd] & 0x03030303u, (w[qd] >> 2) & 0x03030303u,
+                                                   (w[qd] >> 4) & 0x03030303u, (w[qd] >> 6) & 0x03030303u);
+                        const int chunk = 4 * half + qd;
+                        *reinterpret_cast<uint4 *>(bdst + row * 128 + ((chunk ^ (row & 7)) << 4)) = o;
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar(BAR_BFULL + u));
+                    mbar_arrive(bar(BAR_EMPTY + s));
+                }
+                if (++s == XSTAGES) { s = 0; ph ^= 1u; }
+                if (++u == BSTAGES) { u = 0; bph ^= 1u; }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side: tensor maps and launch -----------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
+}
+
+static bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, const void *base, uint64_t inner, uint64_t outer,
+                        uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle sw) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {row_stride_bytes};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
+    static int sm_count = 0;
+    static bool attr_set = false;
+    if (!sm_count) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+    }
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(prefill_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(prefill_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const bool bf16 = (p.flags & HGF_FLAG_OUT_BF16) != 0;
+    CUtensorMap mx, mw, my;
+    if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.xq, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.K, KBLK, TILE_M,
+                     CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorInvalidValue;
+    if (!make_map_2d(&mw, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.packed, (uint64_t)p.K / 4, (uint64_t)p.N, (uint64_t)p.K / 4,
+                     KBLK / 4, TILE_N, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return cudaErrorInvalidValue;
+    if (!make_map_2d(&my, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, p.y, (uint64_t)p.N,
+                     (uint64_t)p.M, (uint64_t)p.N * (bf16 ? 2 : 4), bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorInvalidValue;
+    const int tiles = ((p.M + TILE_M - 1) / TILE_M) * ((p.N + TILE_N - 1) / TILE_N);
+    const int grid = tiles < sm_count ? tiles : sm_count;
+    unsigned int *status = device_status_word();
+    if (!status) return cudaErrorMemoryAllocation;
+    if (bf16)
+        prefill_gemm_kernel<true><<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(mx, mw, my, p, status);
+    else
+        prefill_gemm_kernel<false><<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(mx, mw, my, p, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace hgf

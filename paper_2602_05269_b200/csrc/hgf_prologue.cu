@@ -1,0 +1,284 @@
+// Prologue kernels: per-token absmax int8 quantisation (Algorithm 1, steps 1-2) and the LoRA
+// down-projection H = SiLU(x A) (Algorithm 1, steps 5-6).
+#include "hgf_common.cuh"
+
+namespace hgf {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ int warp_sum_i(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Round-to-nearest-even of the exact quotient 127 x / gamma: 127 x is exact in fp32 for a bf16 x,
+// the IEEE division is correctly rounded and k + 1/2 is representable, so rintf of the rounded
+// quotient equals the rounding of the exact one.
+__device__ __forceinline__ int quant1(float x, float gamma) {
+    float q = rintf(__fdiv_rn(127.0f * x, gamma));
+    q = fminf(fmaxf(q, -127.0f), 127.0f);
+    return __float2int_rn(q);
+}
+
+// One block quantises one token row.
+__device__ void quant_row(const PrologueParams &p, int m) {
+    __shared__ float s_red_f[kWarps];
+    __shared__ int s_red_i[kWarps];
+    const int K = p.K, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint4 *xv = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K);
+    const int nv = K / 8;
+
+    float amax = 0.0f;
+    for (int i = tid; i < nv; i += kThreads) {
+        uint4 v = xv[i];
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            amax = fmaxf(amax, fabsf(bf16lo_to_float(w[j])));
+            amax = fmaxf(amax, fabsf(bf16hi_to_float(w[j])));
+        }
+    }
+    amax = warp_max(amax);
+    if (lane == 0) s_red_f[warp] = amax;
+    __syncthreads();
+    float g = s_red_f[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) g = fmaxf(g, s_red_f[w]);
+    g = fmaxf(g, 1e-5f);
+
+    int sum = 0;
+    uint2 *qv = reinterpret_cast<uint2 *>(p.xq + (size_t)m * K);
+    uint2 *dq = p.dbg_xq ? reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * K) : nullptr;
+    for (int i = tid; i < nv; i += kThreads) {
+        uint4 v = xv[i];
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[2] = {0u, 0u};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int q0 = quant1(bf16lo_to_float(w[j]), g);
+            int q1 = quant1(bf16hi_to_float(w[j]), g);
+            sum += q0 + q1;
+            o[j >> 1] |= (uint32_t)(q0 & 0xff) << (16 * (j & 1));
+            o[j >> 1] |= (uint32_t)(q1 & 0xff) << (16 * (j & 1) + 8);
+        }
+        qv[i] = make_uint2(o[0], o[1]);
+        if (dq) dq[i] = make_uint2(o[0], o[1]);
+    }
+    sum = warp_sum_i(sum);
+    if (lane == 0) s_red_i[warp] = sum;
+    __syncthreads();
+    if (tid == 0) {
+        int tot = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) tot += s_red_i[w];
+        if (p.row_sum) p.row_sum[m] = tot;
+        p.gamma_x[m] = g;
+        if (p.dbg_gamma_x) p.dbg_gamma_x[m] = g;
+    }
+}
+
+// One block computes column j of H for up to 16 tokens: H[m][j] = act(sum_k x[m][k] A[k][j]).
+// fp32 accumulation of exact bf16 x fp16 products.
+__device__ void lora_down_column(const PrologueParams &p, int j) {
+    __shared__ float s_part[kWarps][HGF_DECODE_MAX_M];
+    const int K = p.K, M = p.M, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint4 *av = reinterpret_cast<const uint4 *>(p.At + (size_t)j * K);
+    const int nv = K / 8;
+    float acc[HGF_DECODE_MAX_M];
+#pragma unroll
+    for (int m = 0; m < HGF_DECODE_MAX_M; ++m) acc[m] = 0.0f;
+
+    for (int i = tid; i < nv; i += kThreads) {
+        uint4 a4 = av[i];
+        float a[8];
+        {
+            const __half2 *h2 = reinterpret_cast<const __half2 *>(&a4);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float2 f = __half22float2(h2[q]);
+                a[2 * q] = f.x;
+                a[2 * q + 1] = f.y;
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < HGF_DECODE_MAX_M; ++m) {
+            if (m < M) {
+                uint4 x4 = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K)[i];
+                uint32_t w[4] = {x4.x, x4.y, x4.z, x4.w};
+                float s = acc[m];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    s = fmaf(bf16lo_to_float(w[q]), a[2 * q], s);
+                    s = fmaf(bf16hi_to_float(w[q]), a[2 * q + 1], s);
+                }
+                acc[m] = s;
+            }
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < HGF_DECODE_MAX_M; ++m) {
+        float v = warp_sum_f(acc[m]);
+        if (lane == 0) s_part[warp][m] = v;
+    }
+    __syncthreads();
+    if (tid < M) {
+        float z = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) z += s_part[w][tid];
+        float h = (p.flags & HGF_FLAG_NO_SILU) ? z : silu_f(z);
+        p.h[(size_t)tid * p.r + j] = h;
+        if (p.dbg_h) p.dbg_h[(size_t)tid * p.r + j] = h;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p) {
+    quant_row(p, blockIdx.x);
+}
+
+// Decode prologue: blocks [0, M) quantise one token each, blocks [M, M + r) compute one column of H.
+__global__ void __launch_bounds__(kThreads) decode_prologue_kernel(const PrologueParams p) {
+    if ((int)blockIdx.x < p.M)
+        quant_row(p, blockIdx.x);
+    else
+        lora_down_column(p, blockIdx.x - p.M);
+}
+
+// ---- GEMM-path LoRA down-projection on tensor cores (legacy warp MMA, tf32 inputs) -----------
+// bf16 and fp16 values are both exactly representable in tf32 (8 exponent, 10 mantissa bits), so
+// the products are formed from exact inputs and accumulated in fp32.
+// Block = 4 warps, tile = 32 tokens x r columns; the warps split K in 32-element chunks and the
+// partial sums are reduced through shared memory.
+constexpr int kLdThreads = 128;
+constexpr int kLdTokens = 32;
+
+__device__ __forceinline__ void mma_tf32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                         uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int JT>  // r = 8 * JT column tiles
+__global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const PrologueParams p) {
+    extern __shared__ float s_acc[];  // [4 warps][32 tokens][8*JT]
+    const int K = p.K, M = p.M, r = 8 * JT;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    const int m0 = blockIdx.x * kLdTokens;
+
+    float acc[2][JT][4];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < JT; ++b)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.0f;
+
+    // rows this thread feeds: tokens m0 + 16 mt + g and + 8 (clamped; clamped rows are not stored)
+    const __nv_bfloat16 *xrow[2][2];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            int m = m0 + 16 * mt + 8 * hh + g;
+            m = m < M ? m : M - 1;
+            xrow[mt][hh] = p.x + (size_t)m * K;
+        }
+
+    const int nchunks = K / 32;
+    for (int c = warp; c < nchunks; c += 4) {
+        const int k = c * 32 + 8 * t;  // this thread's 8 consecutive k
+        uint4 xa[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) xa[mt][hh] = *reinterpret_cast<const uint4 *>(xrow[mt][hh] + k);
+#pragma unroll
+        for (int jt = 0; jt < JT; ++jt) {
+            uint4 a4 = *reinterpret_cast<const uint4 *>(p.At + (size_t)(8 * jt + g) * K + k);
+            const uint32_t aw[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                __half2 hv = *reinterpret_cast<const __half2 *>(&aw[i]);
+                float2 bf = __half22float2(hv);
+                uint32_t b0 = __float_as_uint(bf.x), b1 = __float_as_uint(bf.y);
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    const uint32_t x0 = (&xa[mt][0].x)[i], x1 = (&xa[mt][1].x)[i];
+                    mma_tf32(acc[mt][jt], x0 << 16, x1 << 16, x0 & 0xffff0000u, x1 & 0xffff0000u, b0, b1);
+                }
+            }
+        }
+    }
+
+    // cross-warp reduction
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int jt = 0; jt < JT; ++jt) {
+            float *base = s_acc + ((size_t)warp * kLdTokens + 16 * mt) * r + 8 * jt;
+            base[(g)*r + 2 * t] = acc[mt][jt][0];
+            base[(g)*r + 2 * t + 1] = acc[mt][jt][1];
+            base[(g + 8) * r + 2 * t] = acc[mt][jt][2];
+            base[(g + 8) * r + 2 * t + 1] = acc[mt][jt][3];
+        }
+    __syncthreads();
+    for (int e = tid; e < kLdTokens * r; e += kLdThreads) {
+        int ml = e / r, j = e % r, m = m0 + ml;
+        float z = s_acc[e] + s_acc[kLdTokens * r + e] + s_acc[2 * kLdTokens * r + e] + s_acc[3 * kLdTokens * r + e];
+        float h = (p.flags & HGF_FLAG_NO_SILU) ? z : silu_f(z);
+        if (m < M) {
+            p.h[(size_t)m * r + j] = h;
+            if (p.dbg_h) p.dbg_h[(size_t)m * r + j] = h;
+            if (p.h16) p.h16[(size_t)m * 64 + j] = __float2half_rn(h);
+        }
+    }
+    if constexpr (JT < 8) {  // zero padding of the fp16 copy up to 64 columns
+        if (p.h16)
+        for (int e = tid; e < kLdTokens * (64 - r); e += kLdThreads) {
+            int ml = e / (64 - r), j = r + e % (64 - r), m = m0 + ml;
+            if (m < M) p.h16[(size_t)m * 64 + j] = __float2half_rn(0.0f);
+        }
+    }
+}
+
+cudaError_t launch_quant(const PrologueParams &p, cudaStream_t stream) {
+    quant_kernel<<<p.M, kThreads, 0, stream>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_prologue(const PrologueParams &p, cudaStream_t stream) {
+    decode_prologue_kernel<<<p.M + p.r, kThreads, 0, stream>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream) {
+    const int blocks = (p.M + kLdTokens - 1) / kLdTokens;
+    const size_t smem = (size_t)4 * kLdTokens * p.r * sizeof(float);
+    switch (p.r) {
+        case 16: lora_down_gemm_kernel<2><<<blocks, kLdThreads, smem, stream>>>(p); break;
+        case 32: lora_down_gemm_kernel<4><<<blocks, kLdThreads, smem, stream>>>(p); break;
+        case 48: lora_down_gemm_kernel<6><<<blocks, kLdThreads, smem, stream>>>(p); break;
+        case 64: lora_down_gemm_kernel<8><<<blocks, kLdThreads, smem, stream>>>(p); break;
+        default: return cudaErrorInvalidValue;
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace hgf

@@ -1,0 +1,178 @@
+"""Thin ctypes binding of libhgf_b200.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch CUDA tensors used purely as device memory; every step of the layer runs in the
+library's kernels.  If the library is missing, or a call fails, this raises: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhgf_b200.so")
+
+HGF_OK = 0
+FLAG_OUT_BF16 = 0x1
+FLAG_NO_SILU = 0x2
+FLAG_FORCE_GEMM = 0x4
+DECODE_MAX_M = 16
+
+# every symbol include/hgf.h declares
+EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_workspace_bytes",
+           "hgf_linear_forward", "hgf_act_quant", "hgf_check_status", "hgf_tmax_tokens_per_s",
+           "hgf_launch_count", "hgf_status_string"]
+
+
+class HgfError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        self.status = status
+        super().__init__(f"{call} failed: status {status} ({status_string(status)})")
+
+
+class DebugOut(ctypes.Structure):
+    _fields_ = [("xq", ctypes.c_void_p), ("gamma_x", ctypes.c_void_p), ("y_int", ctypes.c_void_p),
+                ("h", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (built in-tree by paper_2602_05269_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2602_05269_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        c = ctypes
+        i64, i32, u32, vp, sz = c.c_int64, c.c_int32, c.c_uint32, c.c_void_p, c.c_size_t
+        L.hgf_packed_bytes.restype = sz
+        L.hgf_packed_bytes.argtypes = [i64, i64]
+        L.hgf_pack_ternary.restype = c.c_int
+        L.hgf_pack_ternary.argtypes = [vp, i64, i64, vp, c.POINTER(c.c_float), vp]
+        L.hgf_unpack_ternary.restype = c.c_int
+        L.hgf_unpack_ternary.argtypes = [vp, i64, i64, vp, vp]
+        L.hgf_workspace_bytes.restype = sz
+        L.hgf_workspace_bytes.argtypes = [i64, i64, i64, i32, u32]
+        L.hgf_linear_forward.restype = c.c_int
+        L.hgf_linear_forward.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, vp, sz,
+                                         c.POINTER(DebugOut), u32, vp]
+        L.hgf_act_quant.restype = c.c_int
+        L.hgf_act_quant.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+        L.hgf_check_status.restype = c.c_int
+        L.hgf_check_status.argtypes = [vp]
+        L.hgf_tmax_tokens_per_s.restype = c.c_double
+        L.hgf_tmax_tokens_per_s.argtypes = [c.c_double] * 3
+        L.hgf_launch_count.restype = c.c_uint64
+        L.hgf_launch_count.argtypes = []
+        L.hgf_status_string.restype = c.c_char_p
+        L.hgf_status_string.argtypes = [c.c_int]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(call, status):
+    if status != HGF_OK:
+        raise HgfError(call, status)
+
+
+def status_string(status: int) -> str:
+    return lib().hgf_status_string(int(status)).decode()
+
+
+def packed_bytes(d_out: int, d_in: int) -> int:
+    return int(lib().hgf_packed_bytes(d_out, d_in))
+
+
+def pack_ternary(W: torch.Tensor, stream=None):
+    """W: CUDA fp32 [d_out][d_in] -> (packed uint8 [d_out*d_in/4] on the device, gamma_W as float)."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
+    d_out, d_in = W.shape
+    nbytes = packed_bytes(d_out, d_in)
+    if nbytes == 0:
+        raise HgfError("hgf_packed_bytes", 2)
+    packed = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
+    gamma = ctypes.c_float(0.0)
+    _check("hgf_pack_ternary",
+           lib().hgf_pack_ternary(_ptr(W), d_out, d_in, _ptr(packed), ctypes.byref(gamma), _stream(stream)))
+    return packed, float(gamma.value)
+
+
+def unpack_ternary(packed: torch.Tensor, d_out: int, d_in: int, stream=None) -> torch.Tensor:
+    T = torch.empty((d_out, d_in), dtype=torch.int8, device=packed.device)
+    _check("hgf_unpack_ternary", lib().hgf_unpack_ternary(_ptr(packed), d_out, d_in, _ptr(T), _stream(stream)))
+    return T
+
+
+def workspace_bytes(M: int, d_in: int, d_out: int, r: int, flags: int = 0) -> int:
+    return int(lib().hgf_workspace_bytes(M, d_in, d_out, r, flags))
+
+
+def act_quant(x: torch.Tensor, stream=None):
+    """x: CUDA bf16 [M][d_in] -> (xq int8 [M][d_in], gamma_x fp32 [M], row_sum int32 [M])."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    M, K = x.shape
+    xq = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    gx = torch.empty(M, dtype=torch.float32, device=x.device)
+    rs = torch.empty(M, dtype=torch.int32, device=x.device)
+    _check("hgf_act_quant", lib().hgf_act_quant(_ptr(x), M, K, _ptr(xq), _ptr(gx), _ptr(rs), _stream(stream)))
+    return xq, gx, rs
+
+
+def linear_forward(x, packed, gamma, d_in, d_out, At=None, Bt=None, gate=None, *, y=None, workspace=None,
+                   debug=False, flags=0, stream=None):
+    """Enqueue one layer forward.  Returns y, or (y, dbg dict of device tensors) with debug=True.
+
+    x bf16 [M][d_in]; packed uint8 from pack_ternary; At fp16 [r][d_in]; Bt fp16 [d_out][r];
+    gate fp32 [d_out]; y fp32 (or bf16 with FLAG_OUT_BF16) [M][d_out].
+    """
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    M = x.shape[0]
+    r = 0 if At is None else At.shape[0]
+    if y is None:
+        y = torch.empty((M, d_out), dtype=torch.bfloat16 if flags & FLAG_OUT_BF16 else torch.float32,
+                        device=x.device)
+    if workspace is None:
+        workspace = torch.empty(workspace_bytes(M, d_in, d_out, r, flags), dtype=torch.uint8, device=x.device)
+    dbg_struct, dbg = None, None
+    if debug:
+        dbg = {"xq": torch.empty((M, d_in), dtype=torch.int8, device=x.device),
+               "gamma_x": torch.empty(M, dtype=torch.float32, device=x.device),
+               "y_int": torch.empty((M, d_out), dtype=torch.int32, device=x.device),
+               "h": torch.empty((M, max(r, 1)), dtype=torch.float32, device=x.device)}
+        dbg_struct = DebugOut(dbg["xq"].data_ptr(), dbg["gamma_x"].data_ptr(), dbg["y_int"].data_ptr(),
+                              dbg["h"].data_ptr())
+    st = lib().hgf_linear_forward(_ptr(x), M, _ptr(packed), ctypes.c_float(gamma), d_in, d_out, _ptr(At), _ptr(Bt),
+                                  r, _ptr(gate), _ptr(y), _ptr(workspace), workspace.numel(),
+                                  ctypes.byref(dbg_struct) if dbg_struct is not None else None, flags,
+                                  _stream(stream))
+    _check("hgf_linear_forward", st)
+    if debug:
+        dbg["h"] = dbg["h"][:, :r]
+        return y, dbg
+    return y
+
+
+def check_status(stream=None) -> None:
+    """Synchronise and raise if a bounded device-side wait gave up since the last check."""
+    _check("hgf_check_status", lib().hgf_check_status(_stream(stream)))
+
+
+def tmax_tokens_per_s(bmem_bytes_per_s: float, params: float, bits: float) -> float:
+    return float(lib().hgf_tmax_tokens_per_s(bmem_bytes_per_s, params, bits))
+
+
+def launch_count() -> int:
+    return int(lib().hgf_launch_count())
