@@ -378,6 +378,30 @@ def run_reference(args):
     }))
 
 
+def run_profile_case(spec: str, reps: int):
+    """Plain launches of one layer problem, for use under a profiler: `kind:KxNxM[xr][:bf16]`.
+    The printed time is wall-clock context only, never a benchmark value."""
+    import torch
+
+    from paper_2602_05269_b200 import hgf, inputs as syn
+
+    parts = spec.split(":")
+    dims = [int(v) for v in parts[1].split("x")]
+    K, N, M = dims[:3]
+    r = dims[3] if len(dims) > 3 else 32
+    flags = hgf.FLAG_OUT_BF16 if (len(parts) > 2 and parts[2] == "bf16") else 0
+    copies = int(parts[3]) if len(parts) > 3 else 1
+    torch.cuda.set_device(0)
+    stream = torch.cuda.Stream()
+    w = Workload(hgf, torch, [syn.LayerShape("p", K, N, r)], M, copies, flags=flags)
+    with torch.cuda.stream(stream):
+        for _ in range(reps):
+            w.enqueue(stream)
+        stream.synchronize()
+    hgf.check_status(stream)
+    print(json.dumps({"profile_case": spec, "reps": reps, "launches": hgf.launch_count()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -386,7 +410,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline measurement only")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
+    ap.add_argument("--profile", default=None,
+                    help="run plain launches of one case for a profiler, e.g. prefill:2048x5632x8192x32:bf16")
+    ap.add_argument("--reps", type=int, default=3)
     args = ap.parse_args()
+    if args.profile:
+        run_profile_case(args.profile, args.reps)
+        return
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

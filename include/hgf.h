@@ -46,6 +46,8 @@ typedef enum {
 #define HGF_FLAG_NO_SILU 0x2u  /* correction is (x A) B, without the SiLU the paper defines */
 #define HGF_FLAG_FORCE_GEMM 0x4u /* route to the tensor-core GEMM path even when M <= 16 (testing) */
 
+#define HGF_FLAG_NO_PDL 0x8u     /* do not use programmatic dependent launch (see hgf_linear_forward) */
+
 /* Largest token count the register-resident decode path handles; above it the GEMM path runs. */
 #define HGF_DECODE_MAX_M 16
 
@@ -108,12 +110,51 @@ size_t hgf_workspace_bytes(int64_t M, int64_t d_in, int64_t d_out, int32_t r, ui
  * pointers.  M <= HGF_DECODE_MAX_M runs the bandwidth-bound GEMV path, larger M the tcgen05
  * int8 GEMM path (which additionally needs d_in % 128 == 0 and d_out % 8 == 0).
  * Calls on the same workspace must not overlap on the device.
+ * Launch overlap: the decode kernels are launched with programmatic stream serialization and start
+ * fetching `packed` before the preceding work on `stream` has finished (they wait for that work
+ * before touching x, the workspace or y).  packed, At, Bt and gate must therefore not be written
+ * by work still pending on `stream`; pass HGF_FLAG_NO_PDL if they might be.
  */
 hgf_status hgf_linear_forward(const void *x, int64_t M, const void *packed, float gamma,
                               int64_t d_in, int64_t d_out, const void *At, const void *Bt,
                               int32_t r, const float *gate, void *y, void *workspace,
                               size_t workspace_bytes, const hgf_debug_out *dbg, uint32_t flags,
                               void *stream);
+
+/*
+ * A group of independent decode-sized layer problems served by one pair of launches.  The paper's
+ * blocks evaluate several HGF layers on the same or on unrelated inputs with no dependency between
+ * them (Section 2.4, Definition "HGF Attention Projections": Q, K and V are three HGF layers of the
+ * same X; the MLP's two up-projections likewise), and each is small against the launch latency,
+ * so a group streams all their packed weights in one pass.  Each problem is exactly one
+ * hgf_linear_forward with M <= HGF_DECODE_MAX_M (same argument meaning, same requirements).
+ *
+ * hgf_group_create records the problems (pointers are kept, not the data: x, y and the weights
+ * stay owned by the caller and must stay valid) and allocates the group's descriptors and
+ * workspace on the current device; it is a set-up call, not for the hot path.
+ * hgf_group_forward only enqueues: one prologue launch and one GEMV launch for the whole group.
+ * Forward calls of one group must not overlap on the device.  hgf_group_destroy frees the group
+ * (the caller makes sure no forward is still running).
+ */
+typedef struct {
+    const void *x;      /* [M][d_in] bf16 */
+    int64_t M;
+    const void *packed; /* from hgf_pack_ternary */
+    float gamma;
+    int64_t d_in, d_out;
+    const void *At;     /* [r][d_in] fp16, nullable */
+    const void *Bt;     /* [d_out][r] fp16, nullable */
+    int32_t r;
+    const float *gate;  /* [d_out] fp32, nullable */
+    void *y;            /* [M][d_out] fp32, or bf16 with HGF_FLAG_OUT_BF16 */
+} hgf_problem;
+
+typedef struct hgf_group hgf_group;
+
+hgf_status hgf_group_create(const hgf_problem *problems /* host array */, int32_t n, uint32_t flags,
+                            hgf_group **out);
+hgf_status hgf_group_forward(hgf_group *group, void *stream);
+void hgf_group_destroy(hgf_group *group);
 
 /*
  * Step a1 alone (paper, Definition "Dynamic Activation Quantization"): xq, gamma_x and the row

@@ -2,6 +2,8 @@
 // path (M <= 16) and the tcgen05 GEMM path.  No compute happens on the host and there is no CPU
 // fallback: without a CUDA device every forward call fails with HGF_ERR_CUDA.
 #include <atomic>
+#include <new>
+#include <vector>
 
 #include "hgf_common.cuh"
 
@@ -56,64 +58,95 @@ extern "C" hgf_status hgf_act_quant(const void *x, int64_t M, int64_t d_in, int8
     return launch_quant(pp, (cudaStream_t)stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
 }
 
+namespace hgf {
+
+// Validates one layer problem.  On HGF_OK, *r_eff is the rank actually used (0 for a pure
+// ternary layer) and *gemm tells which path the problem takes.
+static hgf_status validate_problem(const void *x, int64_t M, const void *packed, int64_t d_in, int64_t d_out,
+                                   const void *At, const void *Bt, int32_t r, const float *gate, const void *y,
+                                   uint32_t flags, int32_t *r_eff, bool *gemm) {
+    if (!x || !packed || !y || M <= 0 || d_in <= 0 || d_out <= 0 || r < 0) return HGF_ERR_INVALID_ARG;
+    if (flags & ~(HGF_FLAG_OUT_BF16 | HGF_FLAG_NO_SILU | HGF_FLAG_FORCE_GEMM | HGF_FLAG_NO_PDL)) return HGF_ERR_INVALID_ARG;
+    if (!At || !Bt || !gate) r = 0;  // pure ternary layer
+    if (d_in % 64 != 0 || d_in > 65536 || d_out > (1 << 24) || M > (1 << 22)) return HGF_ERR_UNSUPPORTED_SHAPE;
+    if (r != 0 && r != 16 && r != 32 && r != 48 && r != 64) return HGF_ERR_UNSUPPORTED_SHAPE;
+    *gemm = M > HGF_DECODE_MAX_M || (flags & HGF_FLAG_FORCE_GEMM);
+    if (*gemm && (d_out % 8 != 0)) return HGF_ERR_UNSUPPORTED_SHAPE;
+    if (misaligned(x) || misaligned(packed) || misaligned(y) || misaligned(At) || misaligned(Bt) || misaligned(gate))
+        return HGF_ERR_MISALIGNED;
+    *r_eff = r;
+    return HGF_OK;
+}
+
+static void fill_params(const void *x, int64_t M, const void *packed, float gamma, int64_t d_in, int64_t d_out,
+                        const void *At, const void *Bt, int32_t r, const float *gate, void *y, char *ws,
+                        const WsLayout &L, bool gemm, const hgf_debug_out *dbg, uint32_t flags, PrologueParams *pp,
+                        DecodeProblem *dp) {
+    *pp = PrologueParams{};
+    pp->x = (const __nv_bfloat16 *)x;
+    pp->At = r ? (const __half *)At : nullptr;
+    pp->xq = (int8_t *)(ws + L.xq);
+    pp->gamma_x = (float *)(ws + L.gamma_x);
+    pp->row_sum = (int32_t *)(ws + L.row_sum);
+    pp->h = (float *)(ws + L.h);
+    pp->h16 = gemm ? (__half *)(ws + L.h16) : nullptr;
+    pp->dbg_xq = dbg ? dbg->xq : nullptr;
+    pp->dbg_gamma_x = dbg ? dbg->gamma_x : nullptr;
+    pp->dbg_h = (dbg && r) ? dbg->h : nullptr;
+    pp->M = (int)M;
+    pp->K = (int)d_in;
+    pp->r = r;
+    pp->flags = flags;
+    if (dp) {
+        *dp = DecodeProblem{};
+        dp->packed = (const uint8_t *)packed;
+        dp->xq = pp->xq;
+        dp->gamma_x = pp->gamma_x;
+        dp->row_sum = pp->row_sum;
+        dp->h = pp->h;
+        dp->Bt = (const __half *)Bt;
+        dp->gate = gate;
+        dp->y = y;
+        dp->dbg_y_int = dbg ? dbg->y_int : nullptr;
+        dp->gw_over_127 = (float)((double)gamma / 127.0);
+        dp->M = (int)M;
+        dp->K = (int)d_in;
+        dp->N = (int)d_out;
+        dp->r = r;
+        dp->flags = flags;
+        dp->tile_begin = 0;
+    }
+}
+
+}  // namespace hgf
+
 extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *packed, float gamma, int64_t d_in,
                                          int64_t d_out, const void *At, const void *Bt, int32_t r,
                                          const float *gate, void *y, void *workspace, size_t workspace_bytes,
                                          const hgf_debug_out *dbg, uint32_t flags, void *stream_) {
-    if (!x || !packed || !y || M <= 0 || d_in <= 0 || d_out <= 0 || r < 0) return HGF_ERR_INVALID_ARG;
-    if (flags & ~(HGF_FLAG_OUT_BF16 | HGF_FLAG_NO_SILU | HGF_FLAG_FORCE_GEMM)) return HGF_ERR_INVALID_ARG;
-    if (!At || !Bt || !gate) r = 0;  // pure ternary layer
-    if (d_in % 64 != 0 || d_in > 65536 || d_out > (1 << 24) || M > (1 << 22)) return HGF_ERR_UNSUPPORTED_SHAPE;
-    if (r != 0 && r != 16 && r != 32 && r != 48 && r != 64) return HGF_ERR_UNSUPPORTED_SHAPE;
-    const bool gemm = M > HGF_DECODE_MAX_M || (flags & HGF_FLAG_FORCE_GEMM);
-    if (gemm && (d_out % 8 != 0)) return HGF_ERR_UNSUPPORTED_SHAPE;
-    if (misaligned(x) || misaligned(packed) || misaligned(y) || misaligned(At) || misaligned(Bt) || misaligned(gate))
-        return HGF_ERR_MISALIGNED;
+    bool gemm = false;
+    hgf_status st = validate_problem(x, M, packed, d_in, d_out, At, Bt, r, gate, y, flags, &r, &gemm);
+    if (st != HGF_OK) return st;
     if (dbg && (misaligned(dbg->xq) || misaligned(dbg->gamma_x) || misaligned(dbg->y_int) || misaligned(dbg->h)))
         return HGF_ERR_MISALIGNED;
     const WsLayout L = ws_layout(M, d_in, r, gemm);
     if (!workspace || workspace_bytes < L.total) return HGF_ERR_WORKSPACE;
     if (((uintptr_t)workspace) & 255u) return HGF_ERR_MISALIGNED;
     cudaStream_t stream = (cudaStream_t)stream_;
-    char *ws = (char *)workspace;
+    const bool pdl = !(flags & HGF_FLAG_NO_PDL);
 
-    PrologueParams pp = {};
-    pp.x = (const __nv_bfloat16 *)x;
-    pp.At = r ? (const __half *)At : nullptr;
-    pp.xq = (int8_t *)(ws + L.xq);
-    pp.gamma_x = (float *)(ws + L.gamma_x);
-    pp.row_sum = (int32_t *)(ws + L.row_sum);
-    pp.h = (float *)(ws + L.h);
-    pp.h16 = gemm ? (__half *)(ws + L.h16) : nullptr;
-    pp.dbg_xq = dbg ? dbg->xq : nullptr;
-    pp.dbg_gamma_x = dbg ? dbg->gamma_x : nullptr;
-    pp.dbg_h = (dbg && r) ? dbg->h : nullptr;
-    pp.M = (int)M;
-    pp.K = (int)d_in;
-    pp.r = r;
-    pp.flags = flags;
-
-    const float gw = (float)((double)gamma / 127.0);
+    PrologueParams pp;
+    DecodeProblem dp;
+    fill_params(x, M, packed, gamma, d_in, d_out, At, Bt, r, gate, y, (char *)workspace, L, gemm, dbg, flags, &pp, &dp);
 
     if (!gemm) {
-        if (launch_decode_prologue(pp, stream) != cudaSuccess) return HGF_ERR_CUDA;
-        DecodeParams dp = {};
-        dp.packed = (const uint8_t *)packed;
-        dp.xq = pp.xq;
-        dp.gamma_x = pp.gamma_x;
-        dp.row_sum = pp.row_sum;
-        dp.h = pp.h;
-        dp.Bt = (const __half *)Bt;
-        dp.gate = gate;
-        dp.y = y;
-        dp.dbg_y_int = dbg ? dbg->y_int : nullptr;
-        dp.gw_over_127 = gw;
-        dp.M = (int)M;
-        dp.K = (int)d_in;
-        dp.N = (int)d_out;
-        dp.r = r;
-        dp.flags = flags;
-        return launch_decode_gemv(dp, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
+        if (launch_decode_prologue(pp, pdl, stream) != cudaSuccess) return HGF_ERR_CUDA;
+        DecodeLaunch dl = {};
+        dl.probs = nullptr;
+        dl.n_probs = 1;
+        dl.total_tiles = (int)((d_out + 15) / 16);
+        return launch_decode_gemv(dl, &dp, (int)M, (int)((d_in + 255) / 256), pdl, stream) == cudaSuccess ? HGF_OK
+                                                                                                       : HGF_ERR_CUDA;
     }
 
     if (launch_quant(pp, stream) != cudaSuccess) return HGF_ERR_CUDA;
@@ -128,13 +161,102 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
     gp.gate = gate;
     gp.y = y;
     gp.dbg_y_int = dbg ? dbg->y_int : nullptr;
-    gp.gw_over_127 = gw;
+    gp.gw_over_127 = dp.gw_over_127;
     gp.M = (int)M;
     gp.K = (int)d_in;
     gp.N = (int)d_out;
     gp.r = r;
     gp.flags = flags;
     return launch_prefill_gemm(gp, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
+}
+
+// ---- groups of independent decode problems --------------------------------------------------------
+struct hgf_group {
+    int n, total_tiles, total_blocks, max_M, min_steps, device;
+    uint32_t flags;
+    void *d_mem;              // one allocation: descriptors, block offsets, workspaces
+    DecodeProblem *d_probs;
+    PrologueParams *d_pps;
+    int *d_blk_begin;
+};
+
+extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, uint32_t flags, hgf_group **out) {
+    if (!problems || !out || n <= 0 || n > 65536) return HGF_ERR_INVALID_ARG;
+    if (flags & HGF_FLAG_FORCE_GEMM) return HGF_ERR_INVALID_ARG;
+    *out = nullptr;
+    std::vector<PrologueParams> pps((size_t)n);
+    std::vector<DecodeProblem> dps((size_t)n);
+    std::vector<int> blk((size_t)n + 1);
+    std::vector<WsLayout> lay((size_t)n);
+    std::vector<int32_t> ranks((size_t)n);
+    size_t ws_total = 0;
+    int tiles = 0, blocks = 0, max_M = 0, min_steps = 1 << 30;
+    for (int i = 0; i < n; ++i) {
+        const hgf_problem &q = problems[i];
+        bool gemm = false;
+        int32_t r = q.r;
+        hgf_status st = validate_problem(q.x, q.M, q.packed, q.d_in, q.d_out, q.At, q.Bt, q.r, q.gate, q.y, flags, &r, &gemm);
+        if (st != HGF_OK) return st;
+        if (gemm) return HGF_ERR_UNSUPPORTED_SHAPE;  // groups hold decode-sized problems only
+        ranks[i] = r;
+        lay[i] = ws_layout(q.M, q.d_in, r, false);
+        ws_total += lay[i].total;
+        if (tiles > (1 << 30) - (1 << 21)) return HGF_ERR_UNSUPPORTED_SHAPE;
+    }
+    const size_t off_probs = 0;
+    const size_t off_pps = align_up(off_probs + sizeof(DecodeProblem) * (size_t)n, 256);
+    const size_t off_blk = align_up(off_pps + sizeof(PrologueParams) * (size_t)n, 256);
+    const size_t off_ws = align_up(off_blk + sizeof(int) * ((size_t)n + 1), 256);
+    void *mem = nullptr;
+    if (cudaMalloc(&mem, off_ws + ws_total) != cudaSuccess) return HGF_ERR_CUDA;
+    char *ws = (char *)mem + off_ws;
+    for (int i = 0; i < n; ++i) {
+        const hgf_problem &q = problems[i];
+        fill_params(q.x, q.M, q.packed, q.gamma, q.d_in, q.d_out, q.At, q.Bt, ranks[i], q.gate, q.y, ws, lay[i], false,
+                    nullptr, flags, &pps[i], &dps[i]);
+        ws += lay[i].total;
+        dps[i].tile_begin = tiles;
+        blk[i] = blocks;
+        tiles += (int)((q.d_out + 15) / 16);
+        blocks += (int)q.M + ranks[i];
+        max_M = q.M > max_M ? (int)q.M : max_M;
+        const int steps = (int)((q.d_in + 255) / 256);
+        min_steps = steps < min_steps ? steps : min_steps;
+    }
+    blk[n] = blocks;
+    hgf_group *g = new (std::nothrow) hgf_group();
+    if (!g) { cudaFree(mem); return HGF_ERR_CUDA; }
+    g->n = n; g->total_tiles = tiles; g->total_blocks = blocks; g->max_M = max_M; g->min_steps = min_steps;
+    g->flags = flags; g->d_mem = mem;
+    g->d_probs = (DecodeProblem *)((char *)mem + off_probs);
+    g->d_pps = (PrologueParams *)((char *)mem + off_pps);
+    g->d_blk_begin = (int *)((char *)mem + off_blk);
+    cudaGetDevice(&g->device);
+    bool ok = cudaMemcpy(g->d_probs, dps.data(), sizeof(DecodeProblem) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
+              cudaMemcpy(g->d_pps, pps.data(), sizeof(PrologueParams) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
+              cudaMemcpy(g->d_blk_begin, blk.data(), sizeof(int) * ((size_t)n + 1), cudaMemcpyHostToDevice) == cudaSuccess;
+    if (!ok) { cudaFree(mem); delete g; return HGF_ERR_CUDA; }
+    *out = g;
+    return HGF_OK;
+}
+
+extern "C" hgf_status hgf_group_forward(hgf_group *g, void *stream_) {
+    if (!g) return HGF_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const bool pdl = !(g->flags & HGF_FLAG_NO_PDL);
+    if (launch_decode_prologue_group(g->d_pps, g->d_blk_begin, g->n, g->total_blocks, pdl, stream) != cudaSuccess)
+        return HGF_ERR_CUDA;
+    DecodeLaunch dl = {};
+    dl.probs = g->d_probs;
+    dl.n_probs = g->n;
+    dl.total_tiles = g->total_tiles;
+    return launch_decode_gemv(dl, nullptr, g->max_M, g->min_steps, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
+}
+
+extern "C" void hgf_group_destroy(hgf_group *g) {
+    if (!g) return;
+    cudaFree(g->d_mem);
+    delete g;
 }
 
 extern "C" hgf_status hgf_check_status(void *stream) {

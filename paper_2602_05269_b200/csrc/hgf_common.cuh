@@ -60,7 +60,9 @@ struct PrologueParams {
     uint32_t flags;
 };
 
-struct DecodeParams {
+// One layer problem of a decode launch (M <= 16).  tile_begin = index of its first 16-row tile in
+// the launch-wide tile numbering.
+struct DecodeProblem {
     const uint8_t *packed;   // [N][K/4]
     const int8_t *xq;        // [M][K]
     const float *gamma_x;    // [M]
@@ -73,13 +75,24 @@ struct DecodeParams {
     float gw_over_127;       // gamma_W / 127
     int M, K, N, r;
     uint32_t flags;
+    int tile_begin;
+};
+
+struct DecodeLaunch {
+    const DecodeProblem *probs;  // device array, or null for a single problem passed by value
+    int n_probs;
+    int total_tiles;
+    int S;                       // K slices per row tile (chosen by the launcher)
 };
 
 // host-side launchers (each enqueues on `stream` and returns the CUDA error of the launch)
 cudaError_t launch_quant(const PrologueParams &p, cudaStream_t stream);
-cudaError_t launch_decode_prologue(const PrologueParams &p, cudaStream_t stream);
+cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream_t stream);
+cudaError_t launch_decode_prologue_group(const PrologueParams *d_pps, const int *d_blk_begin, int n, int total_blocks,
+                                         bool pdl, cudaStream_t stream);
 cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream);
-cudaError_t launch_decode_gemv(const DecodeParams &p, cudaStream_t stream);
+cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, int max_M, int min_steps, bool pdl,
+                               cudaStream_t stream);
 
 struct GemmParams {
     const int8_t *xq;        // [M][K]

@@ -147,12 +147,36 @@ __global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p)
     quant_row(p, blockIdx.x);
 }
 
+// Programmatic dependent launch: no-ops when the launch carries no such attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+
 // Decode prologue: blocks [0, M) quantise one token each, blocks [M, M + r) compute one column of H.
 __global__ void __launch_bounds__(kThreads) decode_prologue_kernel(const PrologueParams p) {
+    pdl_launch_dependents();  // the GEMV that follows may start streaming its weights
+    pdl_wait();               // x, and the workspace this kernel overwrites, belong to earlier work
     if ((int)blockIdx.x < p.M)
         quant_row(p, blockIdx.x);
     else
         lora_down_column(p, blockIdx.x - p.M);
+}
+
+// The same for a group of problems: blk_begin[i] = first block of problem i (n + 1 entries).
+__global__ void __launch_bounds__(kThreads) decode_prologue_group_kernel(const PrologueParams *pps, const int *blk_begin,
+                                                                         int n) {
+    pdl_launch_dependents();
+    pdl_wait();
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (blk_begin[mid] <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
+    }
+    const PrologueParams p = pps[lo];
+    const int b = blockIdx.x - blk_begin[lo];
+    if (b < p.M)
+        quant_row(p, b);
+    else
+        lora_down_column(p, b - p.M);
 }
 
 // ---- GEMM-path LoRA down-projection on tensor cores (legacy warp MMA, tf32 inputs) -----------
@@ -261,10 +285,33 @@ cudaError_t launch_quant(const PrologueParams &p, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_decode_prologue(const PrologueParams &p, cudaStream_t stream) {
-    decode_prologue_kernel<<<p.M + p.r, kThreads, 0, stream>>>(p);
+static cudaLaunchConfig_t prologue_cfg(int blocks, bool pdl, cudaStream_t stream, cudaLaunchAttribute *attr) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cfg;
+}
+
+cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream_t stream) {
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = prologue_cfg(p.M + p.r, pdl, stream, attr);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_prologue_kernel, p);
     count_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_decode_prologue_group(const PrologueParams *d_pps, const int *d_blk_begin, int n, int total_blocks,
+                                         bool pdl, cudaStream_t stream) {
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = prologue_cfg(total_blocks, pdl, stream, attr);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_prologue_group_kernel, d_pps, d_blk_begin, n);
+    count_launch();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream) {

@@ -17,18 +17,27 @@ HGF_OK = 0
 FLAG_OUT_BF16 = 0x1
 FLAG_NO_SILU = 0x2
 FLAG_FORCE_GEMM = 0x4
+FLAG_NO_PDL = 0x8
 DECODE_MAX_M = 16
 
 # every symbol include/hgf.h declares
 EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_workspace_bytes",
            "hgf_linear_forward", "hgf_act_quant", "hgf_check_status", "hgf_tmax_tokens_per_s",
-           "hgf_launch_count", "hgf_status_string"]
+           "hgf_launch_count", "hgf_status_string", "hgf_group_create", "hgf_group_forward",
+           "hgf_group_destroy"]
 
 
 class HgfError(RuntimeError):
     def __init__(self, call: str, status: int):
         self.status = status
         super().__init__(f"{call} failed: status {status} ({status_string(status)})")
+
+
+class Problem(ctypes.Structure):
+    _fields_ = [("x", ctypes.c_void_p), ("M", ctypes.c_int64), ("packed", ctypes.c_void_p),
+                ("gamma", ctypes.c_float), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64),
+                ("At", ctypes.c_void_p), ("Bt", ctypes.c_void_p), ("r", ctypes.c_int32),
+                ("gate", ctypes.c_void_p), ("y", ctypes.c_void_p)]
 
 
 class DebugOut(ctypes.Structure):
@@ -68,6 +77,12 @@ def lib() -> ctypes.CDLL:
         L.hgf_tmax_tokens_per_s.argtypes = [c.c_double] * 3
         L.hgf_launch_count.restype = c.c_uint64
         L.hgf_launch_count.argtypes = []
+        L.hgf_group_create.restype = c.c_int
+        L.hgf_group_create.argtypes = [c.POINTER(Problem), i32, u32, c.POINTER(vp)]
+        L.hgf_group_forward.restype = c.c_int
+        L.hgf_group_forward.argtypes = [vp, vp]
+        L.hgf_group_destroy.restype = None
+        L.hgf_group_destroy.argtypes = [vp]
         L.hgf_status_string.restype = c.c_char_p
         L.hgf_status_string.argtypes = [c.c_int]
         _lib = L
@@ -163,6 +178,38 @@ def linear_forward(x, packed, gamma, d_in, d_out, At=None, Bt=None, gate=None, *
         dbg["h"] = dbg["h"][:, :r]
         return y, dbg
     return y
+
+
+class Group:
+    """A group of independent decode-sized problems (hgf_group_*).  `problems` is a list of dicts
+    with keys x, packed, gamma, d_in, d_out, y and optionally At, Bt, gate (device tensors);
+    the tensors are kept alive by this object."""
+
+    def __init__(self, problems, flags: int = 0):
+        self._keep = problems
+        arr = (Problem * len(problems))()
+        for i, q in enumerate(problems):
+            At = q.get("At")
+            arr[i] = Problem(q["x"].data_ptr(), q["x"].shape[0], q["packed"].data_ptr(), float(q["gamma"]),
+                             q["d_in"], q["d_out"], None if At is None else At.data_ptr(),
+                             None if q.get("Bt") is None else q["Bt"].data_ptr(), 0 if At is None else At.shape[0],
+                             None if q.get("gate") is None else q["gate"].data_ptr(), q["y"].data_ptr())
+        self._handle = ctypes.c_void_p()
+        _check("hgf_group_create", lib().hgf_group_create(arr, len(problems), flags, ctypes.byref(self._handle)))
+
+    def forward(self, stream=None) -> None:
+        _check("hgf_group_forward", lib().hgf_group_forward(self._handle, _stream(stream)))
+
+    def close(self) -> None:
+        if self._handle:
+            lib().hgf_group_destroy(self._handle)
+            self._handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def check_status(stream=None) -> None:

@@ -226,3 +226,53 @@ def test_config4_prefill_sampled_tokens(hgf):
     for i, shape in enumerate(syn.distinct_shapes(4)):
         check_layer(hgf, shape, 4096, config=4, layer=i, sample=32, flags=hgf.FLAG_OUT_BF16)
     check_layer(hgf, syn.distinct_shapes(4)[0], 4096, config=4, layer=0, sample=32, tol2=TOL_GEMM)
+
+
+# ----------------------------------------------------------------------------------------- groups
+def _group_problem(hgf, shape, M, config, layer, lora=True):
+    packed, gamma, T = packed_layer(hgf, shape, config, layer)
+    x = syn.make_x(M, shape.d_in, config=config, layer=layer)
+    q = {"x": dev(x, torch.bfloat16), "packed": packed, "gamma": float(gamma), "d_in": shape.d_in,
+         "d_out": shape.d_out, "y": torch.zeros((M, shape.d_out), dtype=torch.float32, device="cuda")}
+    host = {"x": x, "T": T, "gamma": gamma, "At": None, "Bt": None, "gate": None}
+    if lora and shape.r:
+        At, Bt, gate = syn.make_lora(shape.d_in, shape.d_out, shape.r, config=config, layer=layer)
+        q.update(At=dev(At, torch.float16), Bt=dev(Bt, torch.float16), gate=dev(gate))
+        host.update(At=At, Bt=Bt, gate=gate)
+    return q, host
+
+
+@pytest.mark.parametrize("M", [1, 4, 16])
+def test_group_of_independent_layers_matches_oracle_and_single_calls(hgf, M):
+    shapes = [(s, M, True) for s in syn.distinct_shapes(1)]
+    shapes += [(syn.LayerShape("ragged", 448, 72, 16), max(1, M // 2), True),
+               (syn.LayerShape("pure", 1024, 512, 32), M, False),
+               (syn.LayerShape("r64", 3200, 328, 64), min(M, 3), True)]
+    probs, hosts = zip(*[_group_problem(hgf, s, m, 12, i, lora) for i, (s, m, lora) in enumerate(shapes)])
+    group = hgf.Group(list(probs))
+    group.forward()
+    group.forward()          # a second pass over the same buffers must give the same result
+    hgf.check_status()
+    for q, h, (s, m, lora) in zip(probs, hosts, shapes):
+        ref = oracle.forward(h["x"], h["T"], h["gamma"], h["At"], h["Bt"], h["gate"])
+        yg = q["y"].cpu().numpy().astype(np.float64)
+        err = np.abs(yg - ref["y"]).max() / np.abs(ref["y"]).max()
+        assert err <= TOL_DECODE, (s, err)
+        y_single = hgf.linear_forward(q["x"], q["packed"], q["gamma"], s.d_in, s.d_out, q.get("At"), q.get("Bt"),
+                                      q.get("gate"))
+        assert torch.equal(y_single, q["y"]), s     # same kernels, same arithmetic order
+    group.close()
+
+
+def test_group_rejects_gemm_sized_problem(hgf):
+    q, _ = _group_problem(hgf, syn.LayerShape("big", 256, 256, 16), 17, 12, 50)
+    with pytest.raises(hgf.HgfError) as e:
+        hgf.Group([q])
+    assert e.value.status == 2
+
+
+def test_no_pdl_flag_gives_identical_results(hgf):
+    shape = syn.LayerShape("p", 2048, 2048, 32)
+    _, y1, _ = check_layer(hgf, shape, 4, config=13, tol2=TOL_DECODE)
+    _, y2, _ = check_layer(hgf, shape, 4, config=13, flags=hgf.FLAG_NO_PDL, tol2=TOL_DECODE)
+    assert torch.equal(y1, y2)
