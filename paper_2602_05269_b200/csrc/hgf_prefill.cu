@@ -11,8 +11,8 @@
 //               tcgen05.ld, combine, and write through shared memory with TMA stores
 //   warps 6-9   expand the 2-bit codes of a packed tile into the int8, K-major, 128-byte-swizzled
 //               operand layout the tensor core reads from shared memory
-// The tile is 128 tokens (MMA M) x 256 output channels (MMA N).  Codes are c = t + 1 (unsigned
-// operand); sum_k t x~ = sum_k c x~ - sum_k x~ is restored in the epilogue from the row sums.
+// The tile is 128 tokens (MMA M) x 256 output channels (MMA N).  Codes are c = t + 1 (both operands
+// are declared signed 8-bit; 0, 1, 2 read the same either way); sum_k t x~ = sum_k c x~ - sum_k x~ is restored in the epilogue from the row sums.
 //
 // Every wait is bounded: when one gives up, the CTA records it in the device status word, all
 // roles leave their loops, in-flight bulk copies are drained, tensor memory is freed and the
@@ -51,7 +51,8 @@ enum { BAR_FULL = 0, BAR_EMPTY = BAR_FULL + XSTAGES, BAR_BFULL = BAR_EMPTY + XST
        BAR_LORAFULL, BAR_COUNT };
 static_assert(BAR_COUNT * 8 + 16 <= 256, "barrier block too small");
 
-constexpr uint32_t kSpinLimit = 1u << 22;  // bounded waits: about a second at worst
+constexpr uint32_t kSpinLimit = 1u << 22;            // polls of a drain loop
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // bounded waits give up after two seconds
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -76,12 +77,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false if it gave up or another role already aborted.
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after kWaitLimitNs of wall time (and at the latest after kSpinLimit polls
+// past the first clock reading).  Returns false if it gave up or another role already aborted.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           unsigned int *status, unsigned int code) {
+    unsigned long long t0 = 0;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 255u && *abort_flag) return false;
+        if ((i & 127u) == 127u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
+        }
     }
     *abort_flag = 1;
     atomicExch(status, code);
@@ -150,7 +163,7 @@ __device__ __forceinline__ uint64_t make_sw128_desc(uint32_t saddr) {
 }
 // Instruction descriptor: D format (bits 4-5), A format (7-9), B format (10-12), K-major A and B,
 // N >> 3 (17-22), M >> 4 (24-28).
-constexpr uint32_t IDESC_I8 = (2u << 4) /*s32*/ | (1u << 7) /*A signed*/ | (0u << 10) /*B unsigned*/ |
+constexpr uint32_t IDESC_I8 = (2u << 4) /*s32*/ | (1u << 7) /*A s8*/ | (1u << 10) /*B s8: the codes 0..2 read the same*/ |
                               ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
 constexpr uint32_t IDESC_F16 = (1u << 4) /*f32*/ | (0u << 7) /*A f16*/ | (0u << 10) /*B f16*/ |
                                ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
