@@ -84,45 +84,56 @@ void oracle_ternarise(const float *W, int64_t d_out, int64_t d_in, float gamma, 
 }
 
 /* ---- packed layout (the paper only says "1.58-bit"; two bits per weight are used) ------------ */
-/* Row n of the matrix occupies d_in/4 bytes starting at byte n*d_in/4.  A row is a sequence of
- * little-endian 32-bit words; word i holds the 16 weights k = 16 i .. 16 i + 15.  Writing
- * k = 16 i + 4 j + b with j, b in 0..3, the weight's code c = t + 1 (0, 1 or 2; 3 is never
- * written) sits in bits 8 b + 2 j and 8 b + 2 j + 1 of word i. */
-int64_t oracle_packed_bytes(int64_t d_out, int64_t d_in) { return d_out * d_in / 4; }
+/* The matrix is cut into tiles of 16 output rows by 256 input columns; d_out is padded up to a
+ * multiple of 16 and d_in up to a multiple of 256 with zero weights.  A tile is 1024 bytes: its 16
+ * rows one after the other, 64 bytes per row.  Tiles are stored with the column-tile index
+ * running fastest: tile (R, C) starts at byte (R * (d_in_padded / 256) + C) * 1024.  The 64 bytes
+ * of a row are 16 little-endian 32-bit words; word i holds the 16 weights whose column inside
+ * the tile is 16 i .. 16 i + 15.  Writing that column as 16 i + 4 j + b with j, b in 0..3, the
+ * weight's code c = t + 1 (0, 1 or 2; 3 is never written) sits in bits 8 b + 2 j and 8 b + 2 j + 1
+ * of word i. */
+static int64_t padded_cols(int64_t d_in) { return (d_in + 255) / 256 * 256; }
+static int64_t padded_rows(int64_t d_out) { return (d_out + 15) / 16 * 16; }
+
+int64_t oracle_packed_bytes(int64_t d_out, int64_t d_in) { return padded_rows(d_out) * padded_cols(d_in) / 4; }
+
+/* Byte offset of the word that holds weight (n, k), and the bit position of its code in it. */
+static int64_t word_offset(int64_t n, int64_t k, int64_t d_in, int *shift) {
+    int64_t col_tiles = padded_cols(d_in) / 256;
+    int64_t R = n / 16, row = n % 16, C = k / 256, col = k % 256;
+    int64_t i = col / 16, j = (col % 16) / 4, b = col % 4;
+    *shift = (int)(8 * b + 2 * j);
+    return (R * col_tiles + C) * 1024 + row * 64 + i * 4;
+}
 
 void oracle_pack(const int8_t *T, int64_t d_out, int64_t d_in, uint8_t *packed) {
-    int64_t words_per_row = d_in / 16;
-    for (int64_t n = 0; n < d_out; ++n)
-        for (int64_t i = 0; i < words_per_row; ++i) {
-            uint32_t word = 0;
-            for (int j = 0; j < 4; ++j)
-                for (int b = 0; b < 4; ++b) {
-                    int t = T[n * d_in + 16 * i + 4 * j + b];
-                    uint32_t c = (uint32_t)(t + 1);
-                    word |= c << (8 * b + 2 * j);
-                }
-            uint8_t *dst = packed + (n * words_per_row + i) * 4;
-            dst[0] = (uint8_t)(word & 0xff);
-            dst[1] = (uint8_t)((word >> 8) & 0xff);
-            dst[2] = (uint8_t)((word >> 16) & 0xff);
-            dst[3] = (uint8_t)((word >> 24) & 0xff);
+    int64_t rows = padded_rows(d_out), cols = padded_cols(d_in);
+    memset(packed, 0, (size_t)(rows * cols / 4));
+    for (int64_t n = 0; n < rows; ++n)
+        for (int64_t k = 0; k < cols; ++k) {
+            int t = (n < d_out && k < d_in) ? T[n * d_in + k] : 0; /* padding is weight 0 */
+            int shift;
+            int64_t off = word_offset(n, k, d_in, &shift);
+            uint32_t c = (uint32_t)(t + 1) << shift;
+            packed[off + 0] |= (uint8_t)(c & 0xff);
+            packed[off + 1] |= (uint8_t)((c >> 8) & 0xff);
+            packed[off + 2] |= (uint8_t)((c >> 16) & 0xff);
+            packed[off + 3] |= (uint8_t)((c >> 24) & 0xff);
         }
 }
 
-/* Returns the number of invalid codes (value 3) met; those decode to 0. */
+/* Returns the number of invalid codes (value 3) met inside the matrix; those decode to 0. */
 int64_t oracle_unpack(const uint8_t *packed, int64_t d_out, int64_t d_in, int8_t *T) {
-    int64_t words_per_row = d_in / 16, bad = 0;
+    int64_t bad = 0;
     for (int64_t n = 0; n < d_out; ++n)
-        for (int64_t i = 0; i < words_per_row; ++i) {
-            const uint8_t *src = packed + (n * words_per_row + i) * 4;
-            uint32_t word = (uint32_t)src[0] | ((uint32_t)src[1] << 8) | ((uint32_t)src[2] << 16) |
-                            ((uint32_t)src[3] << 24);
-            for (int j = 0; j < 4; ++j)
-                for (int b = 0; b < 4; ++b) {
-                    uint32_t c = (word >> (8 * b + 2 * j)) & 3u;
-                    if (c == 3u) { ++bad; c = 1u; }
-                    T[n * d_in + 16 * i + 4 * j + b] = (int8_t)((int)c - 1);
-                }
+        for (int64_t k = 0; k < d_in; ++k) {
+            int shift;
+            int64_t off = word_offset(n, k, d_in, &shift);
+            uint32_t word = (uint32_t)packed[off] | ((uint32_t)packed[off + 1] << 8) |
+                            ((uint32_t)packed[off + 2] << 16) | ((uint32_t)packed[off + 3] << 24);
+            uint32_t c = (word >> shift) & 3u;
+            if (c == 3u) { ++bad; c = 1u; }
+            T[n * d_in + k] = (int8_t)((int)c - 1);
         }
     return bad;
 }

@@ -100,8 +100,6 @@ def packed_bytes(d_out: int, d_in: int) -> int:
 def pack(T) -> np.ndarray:
     T = _arr(T, np.int8)
     d_out, d_in = T.shape
-    if d_in % 16:
-        raise ValueError("d_in must be a multiple of 16")
     out = np.zeros(packed_bytes(d_out, d_in), np.uint8)
     _load().oracle_pack(_p(T), d_out, d_in, _p(out))
     return out

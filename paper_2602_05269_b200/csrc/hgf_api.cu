@@ -32,15 +32,21 @@ unsigned int *device_status_word() {
 
 static bool misaligned(const void *p) { return p && (((uintptr_t)p) & 15u); }
 
+// The decode path keeps a problem's quantised activations in shared memory; problems too large
+// for that (and every M > 16) take the GEMM path.
+static bool takes_gemm_path(int64_t M, int64_t d_in, uint32_t flags) {
+    if (M > HGF_DECODE_MAX_M || (flags & HGF_FLAG_FORCE_GEMM)) return true;
+    return decode_xq_smem_bytes((int)M, (int)d_in) > decode_xq_smem_limit();
+}
+
 }  // namespace hgf
 
 using namespace hgf;
 
 extern "C" size_t hgf_workspace_bytes(int64_t M, int64_t d_in, int64_t d_out, int32_t r, uint32_t flags) {
     (void)d_out;
-    if (M <= 0 || d_in <= 0 || r < 0) return 256;
-    const bool gemm = M > HGF_DECODE_MAX_M || (flags & HGF_FLAG_FORCE_GEMM);
-    return ws_layout(M, d_in, r, gemm).total;
+    if (M <= 0 || d_in <= 0 || d_in > 65536 || r < 0) return 256;
+    return ws_layout(M, d_in, r, takes_gemm_path(M, d_in, flags)).total;
 }
 
 extern "C" hgf_status hgf_act_quant(const void *x, int64_t M, int64_t d_in, int8_t *xq, float *gamma_x,
@@ -70,7 +76,7 @@ static hgf_status validate_problem(const void *x, int64_t M, const void *packed,
     if (!At || !Bt || !gate) r = 0;  // pure ternary layer
     if (d_in % 64 != 0 || d_in > 65536 || d_out > (1 << 24) || M > (1 << 22)) return HGF_ERR_UNSUPPORTED_SHAPE;
     if (r != 0 && r != 16 && r != 32 && r != 48 && r != 64) return HGF_ERR_UNSUPPORTED_SHAPE;
-    *gemm = M > HGF_DECODE_MAX_M || (flags & HGF_FLAG_FORCE_GEMM);
+    *gemm = takes_gemm_path(M, d_in, flags);
     if (*gemm && (d_out % 8 != 0)) return HGF_ERR_UNSUPPORTED_SHAPE;
     if (misaligned(x) || misaligned(packed) || misaligned(y) || misaligned(At) || misaligned(Bt) || misaligned(gate))
         return HGF_ERR_MISALIGNED;
@@ -89,6 +95,8 @@ static void fill_params(const void *x, int64_t M, const void *packed, float gamm
     pp->gamma_x = (float *)(ws + L.gamma_x);
     pp->row_sum = (int32_t *)(ws + L.row_sum);
     pp->h = (float *)(ws + L.h);
+    pp->h_hi = gemm ? nullptr : (__half *)(ws + L.h_hi);
+    pp->h_lo = gemm ? nullptr : (__half *)(ws + L.h_lo);
     pp->h16 = gemm ? (__half *)(ws + L.h16) : nullptr;
     pp->dbg_xq = dbg ? dbg->xq : nullptr;
     pp->dbg_gamma_x = dbg ? dbg->gamma_x : nullptr;
@@ -103,7 +111,8 @@ static void fill_params(const void *x, int64_t M, const void *packed, float gamm
         dp->xq = pp->xq;
         dp->gamma_x = pp->gamma_x;
         dp->row_sum = pp->row_sum;
-        dp->h = pp->h;
+        dp->h_hi = pp->h_hi;
+        dp->h_lo = pp->h_lo;
         dp->Bt = (const __half *)Bt;
         dp->gate = gate;
         dp->y = y;
@@ -115,6 +124,7 @@ static void fill_params(const void *x, int64_t M, const void *packed, float gamm
         dp->r = r;
         dp->flags = flags;
         dp->tile_begin = 0;
+        dp->cost_begin = 0;
     }
 }
 
@@ -144,9 +154,11 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
         DecodeLaunch dl = {};
         dl.probs = nullptr;
         dl.n_probs = 1;
-        dl.total_tiles = (int)((d_out + 15) / 16);
-        return launch_decode_gemv(dl, &dp, (int)M, (int)((d_in + 255) / 256), pdl, stream) == cudaSuccess ? HGF_OK
-                                                                                                       : HGF_ERR_CUDA;
+        dl.total_tiles = (int)row_tiles(d_out);
+        dl.total_cost = (long long)dl.total_tiles * (long long)(padded_k(d_in) / 256);
+        dl.max_M = (int)M;
+        dl.xq_smem_bytes = decode_xq_smem_bytes((int)M, (int)d_in);
+        return launch_decode_gemv(dl, &dp, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
     }
 
     if (launch_quant(pp, stream) != cudaSuccess) return HGF_ERR_CUDA;
@@ -172,7 +184,8 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
 
 // ---- groups of independent decode problems --------------------------------------------------------
 struct hgf_group {
-    int n, total_tiles, total_blocks, max_M, min_steps, device;
+    int n, total_tiles, total_blocks, max_M, xq_smem_bytes, device;
+    long long total_cost;
     uint32_t flags;
     void *d_mem;              // one allocation: descriptors, block offsets, workspaces
     DecodeProblem *d_probs;
@@ -190,7 +203,8 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     std::vector<WsLayout> lay((size_t)n);
     std::vector<int32_t> ranks((size_t)n);
     size_t ws_total = 0;
-    int tiles = 0, blocks = 0, max_M = 0, min_steps = 1 << 30;
+    int tiles = 0, blocks = 0, max_M = 0, xq_smem = 0;
+    long long cost = 0;
     for (int i = 0; i < n; ++i) {
         const hgf_problem &q = problems[i];
         bool gemm = false;
@@ -216,17 +230,20 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
                     nullptr, flags, &pps[i], &dps[i]);
         ws += lay[i].total;
         dps[i].tile_begin = tiles;
+        dps[i].cost_begin = cost;
         blk[i] = blocks;
-        tiles += (int)((q.d_out + 15) / 16);
-        blocks += (int)q.M + ranks[i];
+        tiles += (int)row_tiles(q.d_out);
+        cost += (long long)row_tiles(q.d_out) * (long long)(padded_k(q.d_in) / 256);
+        blocks += (int)q.M + ranks[i] / 16;
         max_M = q.M > max_M ? (int)q.M : max_M;
-        const int steps = (int)((q.d_in + 255) / 256);
-        min_steps = steps < min_steps ? steps : min_steps;
+        const int xb = decode_xq_smem_bytes((int)q.M, (int)q.d_in);
+        xq_smem = xb > xq_smem ? xb : xq_smem;
     }
     blk[n] = blocks;
     hgf_group *g = new (std::nothrow) hgf_group();
     if (!g) { cudaFree(mem); return HGF_ERR_CUDA; }
-    g->n = n; g->total_tiles = tiles; g->total_blocks = blocks; g->max_M = max_M; g->min_steps = min_steps;
+    g->n = n; g->total_tiles = tiles; g->total_blocks = blocks; g->max_M = max_M; g->xq_smem_bytes = xq_smem;
+    g->total_cost = cost;
     g->flags = flags; g->d_mem = mem;
     g->d_probs = (DecodeProblem *)((char *)mem + off_probs);
     g->d_pps = (PrologueParams *)((char *)mem + off_pps);
@@ -250,7 +267,10 @@ extern "C" hgf_status hgf_group_forward(hgf_group *g, void *stream_) {
     dl.probs = g->d_probs;
     dl.n_probs = g->n;
     dl.total_tiles = g->total_tiles;
-    return launch_decode_gemv(dl, nullptr, g->max_M, g->min_steps, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
+    dl.total_cost = g->total_cost;
+    dl.max_M = g->max_M;
+    dl.xq_smem_bytes = g->xq_smem_bytes;
+    return launch_decode_gemv(dl, nullptr, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
 }
 
 extern "C" void hgf_group_destroy(hgf_group *g) {

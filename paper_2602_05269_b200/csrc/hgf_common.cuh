@@ -19,15 +19,24 @@ namespace hgf {
 void count_launch(int n = 1);
 unsigned int *device_status_word();  // per-device word in global memory; nonzero = a wait gave up
 
+// ---- packed weight layout ---------------------------------------------------------------------
+// Tiles of 16 output rows x 256 input columns, 1 KiB each, row-major inside the tile (64 bytes per
+// row), tiles ordered with the column-tile index fastest.  d_in is padded to a multiple of 256 and
+// d_out to a multiple of 16 with code 1 (weight 0).
+static inline int64_t padded_k(int64_t d_in) { return (d_in + 255) / 256 * 256; }
+static inline int64_t row_tiles(int64_t d_out) { return (d_out + 15) / 16; }
+
 // ---- workspace layout (all sections 256-byte aligned) --------------------------------------
 //   xq       [M][d_in]   int8     quantised activations
 //   gamma_x  [M]         float    per-token scales (floored at 1e-5)
 //   row_sum  [M]         int32    sum_k xq[m][k]  (the packed codes are t + 1, so
 //                                 sum_k t*xq = sum_k c*xq - row_sum)
 //   h        [M][r]      float    SiLU(x A)
-//   h16      [M][64]     half     the same, fp16 and zero-padded to 64 columns (GEMM path only)
+//   h_hi     [M][r]      half     fp16 rounding of h          (decode path only)
+//   h_lo     [M][r]      half     fp16 rounding of h - h_hi   (decode path only)
+//   h16      [M][64]     half     h in fp16, zero-padded to 64 columns (GEMM path only)
 struct WsLayout {
-    size_t xq, gamma_x, row_sum, h, h16, total;
+    size_t xq, gamma_x, row_sum, h, h_hi, h_lo, h16, total;
 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -35,10 +44,13 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 static inline WsLayout ws_layout(int64_t M, int64_t d_in, int32_t r, bool gemm_path) {
     WsLayout L;
     size_t off = 0;
+    const size_t rr = (size_t)(r > 0 ? r : 1);
     L.xq = off;      off += align_up((size_t)M * (size_t)d_in, 256);
     L.gamma_x = off; off += align_up((size_t)M * 4, 256);
     L.row_sum = off; off += align_up((size_t)M * 4, 256);
-    L.h = off;       off += align_up((size_t)M * (size_t)(r > 0 ? r : 1) * 4, 256);
+    L.h = off;       off += align_up((size_t)M * rr * 4, 256);
+    L.h_hi = off;    off += gemm_path ? 0 : align_up((size_t)M * rr * 2, 256);
+    L.h_lo = off;    off += gemm_path ? 0 : align_up((size_t)M * rr * 2, 256);
     L.h16 = off;     off += gemm_path ? align_up((size_t)M * 64 * 2, 256) : 0;
     L.total = off ? off : 256;
     return L;
@@ -52,7 +64,8 @@ struct PrologueParams {
     float *gamma_x;          // [M]
     int32_t *row_sum;        // [M], nullable
     float *h;                // [M][r]
-    __half *h16;             // [M][64] or null
+    __half *h_hi, *h_lo;     // [M][r] each (decode path) or null
+    __half *h16;             // [M][64] (GEMM path) or null
     int8_t *dbg_xq;          // nullable debug copies
     float *dbg_gamma_x;
     float *dbg_h;
@@ -61,13 +74,14 @@ struct PrologueParams {
 };
 
 // One layer problem of a decode launch (M <= 16).  tile_begin = index of its first 16-row tile in
-// the launch-wide tile numbering.
+// the launch-wide tile numbering; cost_begin = number of 1 KiB weight tiles of all earlier problems.
 struct DecodeProblem {
-    const uint8_t *packed;   // [N][K/4]
+    const uint8_t *packed;   // tiled layout, see above
     const int8_t *xq;        // [M][K]
     const float *gamma_x;    // [M]
     const int32_t *row_sum;  // [M]
-    const float *h;          // [M][r]
+    const __half *h_hi;      // [M][r]
+    const __half *h_lo;      // [M][r]
     const __half *Bt;        // [N][r]
     const float *gate;       // [N]
     void *y;                 // [M][N] fp32 or bf16
@@ -76,13 +90,16 @@ struct DecodeProblem {
     int M, K, N, r;
     uint32_t flags;
     int tile_begin;
+    long long cost_begin;
 };
 
 struct DecodeLaunch {
     const DecodeProblem *probs;  // device array, or null for a single problem passed by value
     int n_probs;
     int total_tiles;
-    int S;                       // K slices per row tile (chosen by the launcher)
+    long long total_cost;        // 1 KiB weight tiles of all problems
+    int max_M;                   // largest token count of any problem
+    int xq_smem_bytes;           // shared memory for the largest problem's activations
 };
 
 // host-side launchers (each enqueues on `stream` and returns the CUDA error of the launch)
@@ -91,12 +108,14 @@ cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream
 cudaError_t launch_decode_prologue_group(const PrologueParams *d_pps, const int *d_blk_begin, int n, int total_blocks,
                                          bool pdl, cudaStream_t stream);
 cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream);
-cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, int max_M, int min_steps, bool pdl,
-                               cudaStream_t stream);
+cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream);
+// Shared memory the decode kernel needs for one problem's activations, and the largest it accepts.
+int decode_xq_smem_bytes(int M, int K);
+int decode_xq_smem_limit();
 
 struct GemmParams {
     const int8_t *xq;        // [M][K]
-    const uint8_t *packed;   // [N][K/4]
+    const uint8_t *packed;   // tiled layout, see above
     const float *gamma_x;    // [M]
     const int32_t *row_sum;  // [M]
     const __half *h16;       // [M][64]
@@ -108,7 +127,6 @@ struct GemmParams {
     int M, K, N, r;
     uint32_t flags;
 };
-// Returns cudaSuccess or an error; *status distinguishes tensor-map failures.
 cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream);
 
 // ---- small device helpers ---------------------------------------------------------------------

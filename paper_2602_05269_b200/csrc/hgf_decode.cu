@@ -2,24 +2,58 @@
 // with the dequantisation (step 4), the LoRA up-projection (step 7) and the gated fusion (step 8)
 // fused into the epilogue.  One launch serves one layer or a group of independent layers.
 //
-// The kernel is bound by the packed-weight stream from HBM.  A work item is 16 consecutive
-// output rows of one layer (optionally one of S interleaved K slices of them) and belongs to one
-// warp.  Each lane fetches 128-bit pieces of two weight rows, four steps (4 x 256 k) ahead of
-// their use, expands the 2-bit codes in registers with one AND per register and feeds them to the
-// warp-level int8 tensor-core MMA (m16n8k32, u8 x s8 -> s32): the 16-row operand holds weight
-// rows, the 8-column operand holds the tokens.  The AND masks keep the codes in place, i.e. scaled
+// The kernel is bound by the packed-weight stream from HBM, so it is built around keeping that
+// stream busy.  One persistent CTA of 16 warps per SM.  The weights of all problems of the launch
+// form one long sequence of 1 KiB tiles (16 output rows x 256 input columns); it is cut into equal
+// contiguous shares, one per CTA.  Every warp owns a private ring of 1 KiB shared-memory slots
+// that one of its lanes keeps filled with bulk asynchronous copies (cp.async.bulk, completion on an
+// mbarrier), several tiles ahead of their use and across row-tile, layer and (under programmatic
+// dependent launch) kernel boundaries, so the number of bytes in flight does not depend on what
+// the math is doing.  A warp consumes a row tile (16 output rows, all of K or a K slice of it):
+// per 1 KiB tile two 128-bit shared-memory loads per lane bring the 2-bit codes in the register
+// layout of the warp-level int8 MMA (m16n8k32, u8 x s8 -> s32; the 16-row operand holds weight
+// rows, the 8-column operand the tokens), one AND per register isolates the codes in place (scaled
 // by 1, 4, 16 or 64; each scale has its own accumulator and the exact quotients are added at the
-// end.  Codes are t + 1, so sum_k t x~ = sum_k c x~ - sum_k x~ (the row sums come from the
-// quantisation kernel).  Before an item's epilogue the warp already has the first loads of its
-// next item in flight, so the weight stream does not pause.
+// end).  Codes are t + 1, so sum_k t x~ = sum_k c x~ - sum_k x~ (the row sums come from the
+// quantisation kernel).  The quantised activations of the layer at hand sit in shared memory.
+// The epilogue runs the rank-r up-projection on the same MMA unit (f16 inputs; SiLU(x A) enters as
+// an fp16 value plus an fp16 residual, so nothing is lost against fp32), in the accumulator layout
+// of the integer result, and writes y.
 #include "hgf_common.cuh"
 
 namespace hgf {
 
-constexpr int kDecThreads = 256;
-constexpr int kDecWarps = kDecThreads / 32;
-constexpr int kTileRows = 16;
-constexpr int kDepth = 4;  // steps of weight loads in flight per warp
+constexpr int kDecWarps = 16;
+constexpr int kDecThreads = kDecWarps * 32;
+constexpr int kSlots = 6;            // 1 KiB slots per warp ring
+constexpr int kSlotBytes = 1024;
+constexpr int kXqPad = 64;           // row padding of the activations in shared memory (bank spread)
+constexpr int kHPitch = 72;          // halves per row of H in shared memory (r <= 64, + 8 bank spread)
+
+// shared-memory map
+constexpr int kOffRing = 0;
+constexpr int kOffBars = kOffRing + kDecWarps * kSlots * kSlotBytes;
+constexpr int kOffSmall = kOffBars + kDecWarps * kSlots * 8;
+struct SegSmall {                    // per-problem values the epilogue needs
+    float scale[16];                 // gamma_x[m] * gamma_W / 127
+    int row_sum[16];
+    __half h_hi[16][kHPitch];
+    __half h_lo[16][kHPitch];
+};
+constexpr int kOffRed = kOffSmall + 2 * (int)sizeof(SegSmall);
+constexpr int kRedBytes = kDecWarps * 8 * 32 * 4;  // per warp: up to 8 accumulator registers per lane
+constexpr int kOffFlags = kOffRed + kRedBytes;
+constexpr int kOffXq = kOffFlags + 64;
+constexpr int kSmemLimit = 227 * 1024;
+constexpr int kXqLimit = (kSmemLimit - kOffXq) / 1024 * 1024;
+
+constexpr unsigned long long kDecWaitLimitNs = 2000000000ull;  // bounded waits give up after two seconds
+
+int decode_xq_smem_bytes(int M, int K) { return M * ((int)padded_k(K) + kXqPad); }
+int decode_xq_smem_limit() { return kXqLimit; }
+
+// ---- PTX wrappers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t dsmem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -29,245 +63,444 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
         : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-
-__device__ __forceinline__ uint4 ld_stream_u4(const void *ptr) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(ptr));
-    return v;
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void dmbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ bool dmbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// One bulk copy global -> shared of `bytes` (a multiple of 16; both addresses 16-byte aligned),
+// completing on the mbarrier.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void prefetch_l2(const void *ptr) {
     asm volatile("prefetch.global.L2 [%0];\n" ::"l"(ptr));
+}
+__device__ __forceinline__ unsigned long long dec_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+    return t;
 }
 // Programmatic dependent launch: both are no-ops when the launch carries no such attribute.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 
+// ---- work decomposition -------------------------------------------------------------------------
+// A segment is the run of row tiles of one problem that falls into this CTA's share.  Its tiles are
+// dealt to the 16 warps in rounds of 16 whole tiles; a last round with fewer tiles than warps
+// splits each tile's K range into slices so that every warp has work, and the slices are added
+// through shared memory.
+struct Seg {
+    int p;                   // problem index
+    int lo, hi;              // launch-wide tile range [lo, hi) of the segment
+    int tile_begin;          // first launch-wide tile of the problem
+    int nsteps;              // 1 KiB tiles per row tile (padded K / 256)
+    const uint8_t *packed;
+};
 struct Item {
-    const uint8_t *wA, *wB;  // this lane's two weight rows, already offset by 16 t bytes
-    const int8_t *xq;        // activations of token g, already offset by 64 t
-    int K, M, first_step, nsteps, prob, n0;
+    int tile_local;          // row tile inside the problem
+    int ks0, ks1;            // column tiles [ks0, ks1)
+    int S, slice;            // number of K slices of the row tile, and this warp's
+    bool valid;
 };
 
-__device__ __forceinline__ const DecodeProblem &problem_of(const DecodeLaunch &L, const DecodeProblem &single,
-                                                           int prob) {
-    return L.probs ? L.probs[prob] : single;
+__device__ __forceinline__ const DecodeProblem &problem_of(const DecodeLaunch &L, const DecodeProblem &single, int p) {
+    return L.probs ? L.probs[p] : single;
+}
+__device__ __forceinline__ int steps_of(int K) { return (K + 255) >> 8; }
+__device__ __forceinline__ int tiles_of(int N) { return (N + 15) >> 4; }
+
+// Smallest launch-wide tile index whose first 1 KiB tile has sequence number >= cost.
+__device__ int tile_of_cost(const DecodeLaunch &L, const DecodeProblem &single, long long cost) {
+    int lo = 0, hi = L.n_probs - 1;
+    while (lo < hi) {  // last problem with cost_begin <= cost
+        const int mid = (lo + hi + 1) >> 1;
+        if (problem_of(L, single, mid).cost_begin <= cost) lo = mid; else hi = mid - 1;
+    }
+    const DecodeProblem &P = problem_of(L, single, lo);
+    const int steps = steps_of(P.K), tiles = tiles_of(P.N);
+    long long local = (cost - P.cost_begin + steps - 1) / steps;
+    if (local > tiles) local = tiles;
+    return P.tile_begin + (int)local;
 }
 
-// Work item `tile` (a global row-tile index over all problems of the launch), K slice ks of S.
-__device__ __forceinline__ Item make_item(const DecodeLaunch &L, const DecodeProblem &single, int tile, int ks,
-                                          int S, int g, int t) {
-    Item it;
-    it.nsteps = 0;
-    it.prob = -1;
-    if (tile >= L.total_tiles) return it;
-    int prob = 0;
-    if (L.probs) {  // last problem whose tile_begin <= tile
+// First segment (first = true) or the one after `s`, inside the CTA's tile range [t0, t1).
+__device__ bool next_segment(const DecodeLaunch &L, const DecodeProblem &single, int t0, int t1, bool first, Seg &s) {
+    if (t0 >= t1) return false;
+    int p;
+    if (first) {
         int lo = 0, hi = L.n_probs - 1;
-        while (lo < hi) {
+        while (lo < hi) {  // last problem with tile_begin <= t0
             const int mid = (lo + hi + 1) >> 1;
-            if (L.probs[mid].tile_begin <= tile) lo = mid; else hi = mid - 1;
+            if (problem_of(L, single, mid).tile_begin <= t0) lo = mid; else hi = mid - 1;
         }
-        prob = lo;
+        p = lo;
+    } else {
+        p = s.p + 1;
     }
-    const DecodeProblem &P = problem_of(L, single, prob);
-    const int K = P.K, N = P.N;
-    const int n0 = (tile - P.tile_begin) * kTileRows;
-    const size_t row_bytes = (size_t)K / 4;
-    it.wA = P.packed + (size_t)min(n0 + g, N - 1) * row_bytes + 16 * t;
-    it.wB = P.packed + (size_t)min(n0 + g + 8, N - 1) * row_bytes + 16 * t;
-    it.xq = P.xq + (size_t)g * K + 64 * t;
-    it.K = K;
-    it.M = P.M;
-    it.first_step = ks;
-    const int total = (K + 255) / 256;
-    it.nsteps = ks < total ? (total - ks + S - 1) / S : 0;
-    it.prob = prob;
-    it.n0 = n0;
+    for (; p < L.n_probs; ++p) {
+        const DecodeProblem &P = problem_of(L, single, p);
+        const int tb = P.tile_begin, te = tb + tiles_of(P.N);
+        if (tb >= t1) return false;
+        const int lo = t0 > tb ? t0 : tb, hi = t1 < te ? t1 : te;
+        if (lo < hi) {
+            s.p = p; s.lo = lo; s.hi = hi; s.tile_begin = tb; s.nsteps = steps_of(P.K); s.packed = P.packed;
+            return true;
+        }
+    }
+    return false;
+}
+__device__ __forceinline__ int seg_rounds(const Seg &s) { return (s.hi - s.lo + kDecWarps - 1) / kDecWarps; }
+
+__device__ __forceinline__ Item seg_item(const Seg &s, int round, int warp) {
+    const int n = s.hi - s.lo, full = n / kDecWarps, rem = n % kDecWarps;
+    Item it;
+    if (round < full) {
+        it.tile_local = s.lo - s.tile_begin + round * kDecWarps + warp;
+        it.ks0 = 0; it.ks1 = s.nsteps; it.S = 1; it.slice = 0; it.valid = true;
+    } else {
+        int S = kDecWarps / rem;
+        S = S < s.nsteps ? S : s.nsteps;
+        const int tix = warp / S, sl = warp - tix * S;
+        it.valid = tix < rem;
+        it.tile_local = s.lo - s.tile_begin + full * kDecWarps + tix;
+        it.ks0 = sl * s.nsteps / S; it.ks1 = (sl + 1) * s.nsteps / S;
+        it.S = S; it.slice = sl;
+    }
     return it;
 }
 
+// The copy-issuing side of a warp's ring: walks the same item sequence as the consumer, one 1 KiB
+// tile per call.  All lanes keep the (warp-uniform) state; lane 0 issues.
+struct Producer {
+    Seg seg;
+    int round, rounds, ks, ks1;
+    const uint8_t *src;      // next 1 KiB tile of the current item
+    bool have_item, done;
+    uint32_t seq;            // tiles issued so far
+};
+
 // NT = number of 8-token tiles (1: M <= 8, 2: M <= 16).
 template <int NT>
-__global__ void __launch_bounds__(kDecThreads, 2) decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single) {
-    __shared__ int s_red[kDecWarps][kTileRows][8 * NT];
+__global__ void __launch_bounds__(kDecThreads, 1)
+decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned int *status) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    uint8_t *ring = smem + kOffRing + warp * kSlots * kSlotBytes;
+    const uint32_t ring_u32 = dsmem_u32(ring);
+    const uint32_t bars_u32 = dsmem_u32(smem + kOffBars) + warp * kSlots * 8;
+    SegSmall *small = reinterpret_cast<SegSmall *>(smem + kOffSmall);
+    int *red = reinterpret_cast<int *>(smem + kOffRed);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffFlags);
+    int8_t *xq_s = reinterpret_cast<int8_t *>(smem + kOffXq);
 
     pdl_launch_dependents();
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-    const int S = L.S;                       // K slices per row tile: 1, 2, 4 or 8
-    const int tiles_per_cta = kDecWarps / S;
-    const int my_tile = warp / S, ks = warp % S;
-    const int n_cta_items = (L.total_tiles + tiles_per_cta - 1) / tiles_per_cta;
+    if (tid == 0) *abort_flag = 0;
+    if (lane == 0) {
+        for (int s = 0; s < kSlots; ++s) dmbar_init(bars_u32 + 8 * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncthreads();
 
-    uint4 ringA[kDepth], ringB[kDepth];
-    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+    // this CTA's share of the launch-wide tile sequence
+    const long long c0 = L.total_cost * (long long)blockIdx.x / (long long)gridDim.x;
+    const long long c1 = L.total_cost * (long long)(blockIdx.x + 1) / (long long)gridDim.x;
+    const int t0 = tile_of_cost(L, single, c0);
+    const int t1 = (blockIdx.x + 1 == gridDim.x) ? L.total_tiles : tile_of_cost(L, single, c1);
 
-    auto fetch = [&](const Item &it, int i, uint4 &a, uint4 &b) {
-        // step i of the item; K % 64 == 0, so a lane's 64-wide piece is either whole or absent
-        const int step = it.first_step + i * S;
-        const bool valid = i < it.nsteps && step * 256 + 64 * t < it.K;
-        a = valid ? ld_stream_u4(it.wA + (size_t)step * 64) : zero4;
-        b = valid ? ld_stream_u4(it.wB + (size_t)step * 64) : zero4;
+    // ---- producer ------------------------------------------------------------------------------
+    Producer pr;
+    pr.seq = 0; pr.have_item = false; pr.round = 0; pr.rounds = 0; pr.ks = pr.ks1 = 0; pr.src = nullptr;
+    pr.done = !next_segment(L, single, t0, t1, true, pr.seg);
+    if (!pr.done) { pr.rounds = seg_rounds(pr.seg); pr.round = -1; }
+
+    auto produce = [&]() {
+        // move to the next 1 KiB tile of this warp's sequence, if any, and issue its copy
+        while (!pr.done && (!pr.have_item || pr.ks >= pr.ks1)) {
+            pr.have_item = false;
+            if (++pr.round >= pr.rounds) {
+                if (!next_segment(L, single, t0, t1, false, pr.seg)) { pr.done = true; break; }
+                pr.rounds = seg_rounds(pr.seg);
+                pr.round = 0;
+            }
+            const Item it = seg_item(pr.seg, pr.round, warp);
+            if (it.valid && it.ks0 < it.ks1) {
+                pr.have_item = true;
+                pr.ks = it.ks0; pr.ks1 = it.ks1;
+                pr.src = pr.seg.packed + ((size_t)it.tile_local * pr.seg.nsteps + it.ks0) * kSlotBytes;
+                if (lane == 0 && it.slice == 0) {  // the rows of B^T and the gates this item's epilogue will read
+                    const DecodeProblem &P = problem_of(L, single, pr.seg.p);
+                    if (P.r > 0) {
+                        const int n0 = it.tile_local * 16, rows = P.N - n0 < 16 ? P.N - n0 : 16;
+                        bulk_prefetch_l2(P.Bt + (size_t)n0 * P.r, (uint32_t)(rows * P.r * 2));
+                        prefetch_l2(P.gate + n0);
+                    }
+                }
+            }
+        }
+        if (pr.done) return;
+        if (lane == 0) {
+            const uint32_t slot = pr.seq % kSlots;
+            bulk_load(ring_u32 + slot * kSlotBytes, pr.src, kSlotBytes, bars_u32 + 8 * slot);
+        }
+        pr.src += kSlotBytes;
+        ++pr.ks;
+        ++pr.seq;
     };
-
-    int ci = blockIdx.x;
-    Item cur = make_item(L, single, ci < n_cta_items ? ci * tiles_per_cta + my_tile : L.total_tiles, ks, S, g, t);
-#pragma unroll
-    for (int j = 0; j < kDepth; ++j) fetch(cur, j, ringA[j], ringB[j]);
+#pragma unroll 1
+    for (int i = 0; i < kSlots; ++i) produce();
 
     // everything above reads only weights; the activations come from the preceding launch
     pdl_wait();
 
-    for (; ci < n_cta_items; ci += gridDim.x) {
-        int acc[NT][4][4];
-#pragma unroll
-        for (int a = 0; a < NT; ++a)
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-#pragma unroll
-                for (int c = 0; c < 4; ++c) acc[a][b][c] = 0;
+    // ---- consumer ------------------------------------------------------------------------------
+    uint32_t cseq = 0;  // tiles consumed so far
+    bool ok = true;     // false once a wait gave up (this warp stops computing but keeps the barriers)
+    Seg seg;
+    int seg_idx = 0;
+    for (bool more = next_segment(L, single, t0, t1, true, seg); more;
+         more = next_segment(L, single, t0, t1, false, seg), ++seg_idx) {
+        const DecodeProblem &P = problem_of(L, single, seg.p);
+        const int K = P.K, M = P.M, N = P.N, r = P.r;
+        const int Kp = seg.nsteps * 256, pitch = Kp + kXqPad;
+        SegSmall &sm = small[seg_idx & 1];
 
-        for (int s0 = 0; s0 < cur.nsteps; s0 += kDepth) {
+        // stage the problem's activations and per-token values (all reads of the previous
+        // segment's activations ended at the barrier that closed it)
+        {
+            const int units_per_row = Kp >> 4;
+            for (int u = tid; u < M * units_per_row; u += kDecThreads) {
+                const int m = u / units_per_row, q = u - m * units_per_row;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (16 * q < K) v = *reinterpret_cast<const uint4 *>(P.xq + (size_t)m * K + 16 * q);
+                // inside each 256-byte group the sixteen 16-byte units are stored transposed (4 x 4),
+                // so that the four units a lane reads for one tile are 64 bytes apart
+                const int ql = q & 15, qt = (ql >> 2) + ((ql & 3) << 2);
+                *reinterpret_cast<uint4 *>(xq_s + (size_t)m * pitch + ((q >> 4) << 8) + (qt << 4)) = v;
+            }
+            if (tid < 16) {
+                sm.scale[tid] = tid < M ? P.gamma_x[tid] * P.gw_over_127 : 0.0f;
+                sm.row_sum[tid] = tid < M ? P.row_sum[tid] : 0;
+            }
+            const int words = r >> 1;  // 32-bit words per row of H
+            for (int u = tid; u < M * words; u += kDecThreads) {
+                const int m = u / words, w = u - m * words;
+                reinterpret_cast<uint32_t *>(&sm.h_hi[m][0])[w] = reinterpret_cast<const uint32_t *>(P.h_hi + (size_t)m * r)[w];
+                reinterpret_cast<uint32_t *>(&sm.h_lo[m][0])[w] = reinterpret_cast<const uint32_t *>(P.h_lo + (size_t)m * r)[w];
+            }
+        }
+        __syncthreads();
+
+        // Epilogue of one row tile: dequantise, add the gated rank-r correction, store.  v holds
+        // sum_k c x~ in the MMA accumulator layout: register c of token tile nt is row g + 8 (c >> 1),
+        // token 8 nt + 2 t + (c & 1).
+        auto epilogue = [&](int n0, const int (&v)[NT][4]) {
+            float corr[NT][4];
 #pragma unroll
-            for (int j = 0; j < kDepth; ++j) {
-                const int i = s0 + j;
-                if (i < cur.nsteps) {  // warp-uniform
-                    const uint32_t pw[4] = {ringA[j].x, ringA[j].y, ringA[j].z, ringA[j].w};
-                    const uint32_t qw[4] = {ringB[j].x, ringB[j].y, ringB[j].z, ringB[j].w};
-                    const int k = (cur.first_step + i * S) * 256;  // + 64 t is folded into cur.xq
-                    const bool kvalid = k + 64 * t < cur.K;
-                    fetch(cur, i + kDepth, ringA[j], ringB[j]);
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) corr[nt][c] = 0.0f;
+            const int nA = n0 + g < N ? n0 + g : N - 1, nB = n0 + g + 8 < N ? n0 + g + 8 : N - 1;
+            if (r > 0) {
+                // B^T rows are the 16-row operand, H^T (fp16 value + fp16 residual) the 8-column one
+                const uint32_t *bA = reinterpret_cast<const uint32_t *>(P.Bt + (size_t)nA * r);
+                const uint32_t *bB = reinterpret_cast<const uint32_t *>(P.Bt + (size_t)nB * r);
+                for (int kk = 0; kk < (r >> 4); ++kk) {
+                    const uint32_t a0 = __ldg(bA + 8 * kk + t), a1 = __ldg(bB + 8 * kk + t);
+                    const uint32_t a2 = __ldg(bA + 8 * kk + 4 + t), a3 = __ldg(bB + 8 * kk + 4 + t);
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        uint32_t xw[4][4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            uint4 v = zero4;
-                            if (kvalid && 8 * nt + g < cur.M)
-                                v = *reinterpret_cast<const uint4 *>(cur.xq + (size_t)(8 * nt) * cur.K + k + 16 * u);
-                            xw[u][0] = v.x; xw[u][1] = v.y; xw[u][2] = v.z; xw[u][3] = v.w;
+                        uint32_t h0 = 0, h1 = 0, l0 = 0, l1 = 0;
+                        if (g + 8 * nt < M) {
+                            const uint32_t *hh = reinterpret_cast<const uint32_t *>(&sm.h_hi[g + 8 * nt][0]);
+                            const uint32_t *hl = reinterpret_cast<const uint32_t *>(&sm.h_lo[g + 8 * nt][0]);
+                            h0 = hh[8 * kk + t]; h1 = hh[8 * kk + 4 + t];
+                            l0 = hl[8 * kk + t]; l1 = hl[8 * kk + 4 + t];
                         }
-#pragma unroll
-                        for (int jj = 0; jj < 4; ++jj) {
-                            const uint32_t mask = 0x03030303u << (2 * jj);
-#pragma unroll
-                            for (int h = 0; h < 2; ++h)
-                                mma_u8s8(acc[nt][jj], pw[2 * h] & mask, qw[2 * h] & mask, pw[2 * h + 1] & mask,
-                                         qw[2 * h + 1] & mask, xw[2 * h][jj], xw[2 * h + 1][jj]);
-                        }
+                        mma_f16(corr[nt], a0, a1, a2, a3, h0, h1);
+                        mma_f16(corr[nt], a0, a1, a2, a3, l0, l1);
                     }
                 }
             }
-        }
-
-        // start the next item's weight stream before this item's epilogue
-        const int cn = ci + gridDim.x;
-        const Item nxt = make_item(L, single, cn < n_cta_items ? cn * tiles_per_cta + my_tile : L.total_tiles, ks, S, g, t);
+            const float gA = r > 0 ? __ldg(P.gate + nA) : 0.0f, gB = r > 0 ? __ldg(P.gate + nB) : 0.0f;
 #pragma unroll
-        for (int j = 0; j < kDepth; ++j) fetch(nxt, j, ringA[j], ringB[j]);
-
-        // exact rescale of the four accumulators
-        int v[NT][4];
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                v[nt][c] = acc[nt][0][c] + (acc[nt][1][c] >> 2) + (acc[nt][2][c] >> 4) + (acc[nt][3][c] >> 6);
+                for (int c = 0; c < 4; ++c) {
+                    const int m = 8 * nt + 2 * t + (c & 1), n = n0 + g + 8 * (c >> 1);
+                    if (m < M && n < N) {
+                        const int y_int = v[nt][c] - sm.row_sum[m];
+                        const float y = fmaf(c >> 1 ? gB : gA, corr[nt][c], (float)y_int * sm.scale[m]);
+                        const size_t o = (size_t)m * N + n;
+                        if (P.flags & HGF_FLAG_OUT_BF16)
+                            reinterpret_cast<__nv_bfloat16 *>(P.y)[o] = __float2bfloat16_rn(y);
+                        else
+                            reinterpret_cast<float *>(P.y)[o] = y;
+                        if (P.dbg_y_int) P.dbg_y_int[o] = y_int;
+                    }
+                }
+        };
 
-        if (S > 1) {  // sum the K slices of a row tile through shared memory
-            __syncthreads();  // previous item's readers are done
+        const int rounds = seg_rounds(seg);
+        const int full_rounds = (seg.hi - seg.lo) / kDecWarps;
+        Item last_it;
+        last_it.valid = false;
+        int v_last[NT][4];
+
+        for (int round = 0; round < rounds; ++round) {
+            const Item it = seg_item(seg, round, warp);
+            if (!it.valid || it.ks0 >= it.ks1) { if (round >= full_rounds) last_it = it; continue; }
+
+            int acc[NT][4][4];
+#pragma unroll
+            for (int a = 0; a < NT; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) acc[a][b][c] = 0;
+
+            // this lane's activation bytes of column tile ks: token (g + 8 nt), units t, t+4, t+8, t+12
+            const int8_t *xrow[NT];
+            bool tok_ok[NT];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                s_red[warp][g][8 * nt + 2 * t] = v[nt][0];
-                s_red[warp][g][8 * nt + 2 * t + 1] = v[nt][1];
-                s_red[warp][g + 8][8 * nt + 2 * t] = v[nt][2];
-                s_red[warp][g + 8][8 * nt + 2 * t + 1] = v[nt][3];
+                tok_ok[nt] = g + 8 * nt < M;
+                xrow[nt] = xq_s + (size_t)(tok_ok[nt] ? g + 8 * nt : 0) * pitch + 16 * t;
             }
-            __syncthreads();
-            if (ks == 0) {
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    int s0 = 0, s1 = 0, s2 = 0, s3 = 0;
-                    for (int w = 0; w < S; ++w) {
-                        s0 += s_red[warp + w][g][8 * nt + 2 * t];
-                        s1 += s_red[warp + w][g][8 * nt + 2 * t + 1];
-                        s2 += s_red[warp + w][g + 8][8 * nt + 2 * t];
-                        s3 += s_red[warp + w][g + 8][8 * nt + 2 * t + 1];
+
+            for (int ks = it.ks0; ks < it.ks1; ++ks) {
+                const uint32_t slot = cseq % kSlots, parity = (cseq / kSlots) & 1u;
+                if (ok) {
+                    unsigned long long t_start = 0;
+                    uint32_t polls = 0;
+                    while (!dmbar_try_wait(bars_u32 + 8 * slot, parity)) {
+                        if ((++polls & 255u) == 0) {
+                            const unsigned long long now = dec_timer_ns();
+                            if (t_start == 0) t_start = now;
+                            else if (now - t_start > kDecWaitLimitNs || *abort_flag) { ok = false; break; }
+                        }
                     }
-                    v[nt][0] = s0; v[nt][1] = s1; v[nt][2] = s2; v[nt][3] = s3;
+                    if (!ok) { *abort_flag = 1; if (lane == 0) atomicExch(status, 0x500u + (unsigned)warp); }
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) continue;  // stop computing and copying; tiles cseq .. pr.seq - 1 stay outstanding
+                ++cseq;
+                const uint4 pq = *reinterpret_cast<const uint4 *>(ring + slot * kSlotBytes + 16 * lane);
+                const uint4 qq = *reinterpret_cast<const uint4 *>(ring + slot * kSlotBytes + 512 + 16 * lane);
+                __syncwarp();
+                produce();  // refill the slot just read
+                const uint32_t pw[4] = {pq.x, pq.y, pq.z, pq.w};
+                const uint32_t qw[4] = {qq.x, qq.y, qq.z, qq.w};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t xa[NT][4], xb[NT][4];
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        uint4 va = make_uint4(0u, 0u, 0u, 0u), vb = va;
+                        if (tok_ok[nt]) {
+                            va = *reinterpret_cast<const uint4 *>(xrow[nt] + ks * 256 + 64 * (2 * h));
+                            vb = *reinterpret_cast<const uint4 *>(xrow[nt] + ks * 256 + 64 * (2 * h + 1));
+                        }
+                        xa[nt][0] = va.x; xa[nt][1] = va.y; xa[nt][2] = va.z; xa[nt][3] = va.w;
+                        xb[nt][0] = vb.x; xb[nt][1] = vb.y; xb[nt][2] = vb.z; xb[nt][3] = vb.w;
+                    }
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const uint32_t mask = 0x03030303u << (2 * jj);
+                        const uint32_t a0 = pw[2 * h] & mask, a1 = qw[2 * h] & mask;
+                        const uint32_t a2 = pw[2 * h + 1] & mask, a3 = qw[2 * h + 1] & mask;
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) mma_u8s8(acc[nt][jj], a0, a1, a2, a3, xa[nt][jj], xb[nt][jj]);
+                    }
                 }
             }
+
+            // exact rescale of the four accumulators
+            int v[NT][4];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    v[nt][c] = acc[nt][0][c] + (acc[nt][1][c] >> 2) + (acc[nt][2][c] >> 4) + (acc[nt][3][c] >> 6);
+
+            if (it.S > 1) {  // K slices of a row tile: park the partial sums, add them after the barrier
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) red[(warp * 8 + nt * 4 + c) * 32 + lane] = v[nt][c];
+                last_it = it;
+                continue;
+            }
+            if (round >= full_rounds) {  // last round without slicing: its epilogue also runs after the barrier
+                last_it = it;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) v_last[nt][c] = v[nt][c];
+                continue;
+            }
+            if (ok) epilogue(it.tile_local * 16, v);
         }
 
-        // epilogue: lane l handles output row l / 2 and one half of the rank-r dot product
-        if (ks == 0 && cur.prob >= 0) {
-            const DecodeProblem &P = problem_of(L, single, cur.prob);
-            const int row = lane >> 1, half = lane & 1, n = cur.n0 + row, r = P.r, hr = r >> 1;
-            const bool n_ok = n < P.N;
-            const int nc = n_ok ? n : P.N - 1;
-            uint4 bq[4];  // this lane's half of row n of B^T, as fp16 pairs
+        __syncthreads();  // partial sums are parked; every read of this segment's activations is done
+
+        // ---- epilogue of the last round (after adding K slices) ----------------------------------
+        if (ok && last_it.valid && last_it.slice == 0 && last_it.ks0 < last_it.ks1) {
+            int v[NT][4];
+            if (last_it.S > 1) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                bq[q] = q * 8 < hr ? *reinterpret_cast<const uint4 *>(P.Bt + (size_t)nc * r + half * hr + q * 8) : zero4;
-            const float gate = r > 0 ? P.gate[nc] : 0.0f;
-            const int owner_base = (row & 7) * 4;
+                for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-                for (int mm = 0; mm < 8; ++mm) {
-                    const int m = 8 * nt + mm;
-                    if (m < P.M) {  // warp-uniform
-                        // C[row][m] lives in lane (row % 8) * 4 + mm / 2, register (row / 8) * 2 + mm % 2
-                        const int src = owner_base + (mm >> 1);
-                        const int lo = __shfl_sync(0xffffffffu, v[nt][mm & 1], src);
-                        const int hi = __shfl_sync(0xffffffffu, v[nt][2 + (mm & 1)], src);
-                        const int y_int = (row < 8 ? lo : hi) - P.row_sum[m];
-                        float corr = 0.0f;
-                        if (r > 0) {
-                            const float4 *hv = reinterpret_cast<const float4 *>(P.h + (size_t)m * r + half * hr);
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                if (q * 8 < hr) {
-                                    const __half2 *b2 = reinterpret_cast<const __half2 *>(&bq[q]);
-                                    const float4 h0 = hv[2 * q], h1 = hv[2 * q + 1];
-                                    const float2 f0 = __half22float2(b2[0]), f1 = __half22float2(b2[1]);
-                                    const float2 f2 = __half22float2(b2[2]), f3 = __half22float2(b2[3]);
-                                    corr = fmaf(h0.x, f0.x, corr); corr = fmaf(h0.y, f0.y, corr);
-                                    corr = fmaf(h0.z, f1.x, corr); corr = fmaf(h0.w, f1.y, corr);
-                                    corr = fmaf(h1.x, f2.x, corr); corr = fmaf(h1.y, f2.y, corr);
-                                    corr = fmaf(h1.z, f3.x, corr); corr = fmaf(h1.w, f3.y, corr);
-                                }
-                            }
-                        }
-                        corr += __shfl_xor_sync(0xffffffffu, corr, 1);
-                        if (half == 0 && n_ok) {
-                            const float y = fmaf(gate, corr, (float)y_int * (P.gamma_x[m] * P.gw_over_127));
-                            const size_t o = (size_t)m * P.N + n;
-                            if (P.flags & HGF_FLAG_OUT_BF16)
-                                reinterpret_cast<__nv_bfloat16 *>(P.y)[o] = __float2bfloat16_rn(y);
-                            else
-                                reinterpret_cast<float *>(P.y)[o] = y;
-                            if (P.dbg_y_int) P.dbg_y_int[o] = y_int;
-                        }
+                    for (int c = 0; c < 4; ++c) {
+                        int s = 0;
+                        for (int w = 0; w < last_it.S; ++w) s += red[((warp + w) * 8 + nt * 4 + c) * 32 + lane];
+                        v[nt][c] = s;
                     }
-                }
+            } else {
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) v[nt][c] = v_last[nt][c];
             }
+            epilogue(last_it.tile_local * 16, v);
         }
-        cur = nxt;
+    }
+
+    // A warp that stopped early still has copies in flight: wait (bounded) for them before leaving.
+    if (!ok) {
+        for (uint32_t q = cseq; q < pr.seq; ++q) {
+            const uint32_t slot = q % kSlots, parity = (q / kSlots) & 1u;
+            for (uint32_t i = 0; i < (1u << 20) && !dmbar_try_wait(bars_u32 + 8 * slot, parity); ++i) {}
+        }
     }
 }
 
-// K slices per row tile: enough items to give every resident warp one, at least one step each.
-static int choose_slices(int total_tiles, int min_steps, int warp_slots) {
-    int S = 1;
-    while (S < kDecWarps && total_tiles * S < warp_slots && min_steps >= 2 * S) S *= 2;
-    return S;
-}
-
-cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *single, int max_M, int min_steps,
-                               bool pdl, cudaStream_t stream) {
+cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream) {
     static int sm_count = 0;
+    static bool attr_set = false;
     if (!sm_count) {
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
@@ -275,27 +508,32 @@ cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *si
         e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
     }
-    DecodeLaunch L = L_in;
-    const int warp_slots = sm_count * 2 * kDecWarps;
-    L.S = choose_slices(L.total_tiles, min_steps, warp_slots);
-    const int tiles_per_cta = kDecWarps / L.S;
-    const int n_cta_items = (L.total_tiles + tiles_per_cta - 1) / tiles_per_cta;
-    const int grid = n_cta_items < sm_count * 2 ? n_cta_items : sm_count * 2;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(decode_gemv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(decode_gemv_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    if (L.xq_smem_bytes > kXqLimit) return cudaErrorInvalidValue;
+    unsigned int *status = device_status_word();
+    if (!status) return cudaErrorMemoryAllocation;
+    const int grid = L.total_tiles < sm_count ? L.total_tiles : sm_count;
     DecodeProblem dummy = {};
     const DecodeProblem &sp = single ? *single : dummy;
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kDecThreads);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = (size_t)(kOffXq + L.xq_smem_bytes);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    cudaError_t e = max_M <= 8 ? cudaLaunchKernelEx(&cfg, decode_gemv_kernel<1>, L, sp)
-                               : cudaLaunchKernelEx(&cfg, decode_gemv_kernel<2>, L, sp);
+    cudaError_t e = L.max_M <= 8 ? cudaLaunchKernelEx(&cfg, decode_gemv_kernel<1>, L, sp, status)
+                                 : cudaLaunchKernelEx(&cfg, decode_gemv_kernel<2>, L, sp, status);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -26,39 +26,62 @@ __global__ void __launch_bounds__(kAbsThreads) abs_sum_partial_kernel(const floa
     if (threadIdx.x == 0) partials[blockIdx.x] = red[0];
 }
 
-// Stage 2: one thread adds the partials in index order and rounds the mean once to fp32.
+// Stage 2: one warp adds the partials (fixed order: lane-strided, then a fixed shuffle tree) and
+// rounds the mean once to fp32.
 __global__ void abs_sum_final_kernel(const double *partials, int n, double count, float *gamma) {
-    if (threadIdx.x == 0 && blockIdx.x == 0) {
-        double acc = 0.0;
-        for (int i = 0; i < n; ++i) acc += partials[i];
-        *gamma = (float)(acc / count);
-    }
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n; i += 32) acc += partials[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (threadIdx.x == 0) *gamma = (float)(acc / count);
 }
 
-// Stage 3: one thread per 32-bit packed word (16 weights).  Weight k = 16 i + 4 j + b of a row
-// goes to bits 8 b + 2 j of word i; code = t + 1; t = sign(w) * [|w| > gamma/2].
-__global__ void __launch_bounds__(256) ternarise_pack_kernel(const float4 *W4, size_t n_words,
-                                                             const float *gamma, uint32_t *packed) {
+// Decomposition of a packed word index into its place in the matrix.  Words are numbered in storage
+// order: 16 per row segment, 16 row segments per tile, column tiles fastest, then row tiles.
+struct WordPos {
+    int64_t n, k0;  // output row and first of the 16 input columns the word covers
+};
+__device__ __forceinline__ WordPos word_pos(size_t w, int64_t steps) {
+    const int64_t kw = (int64_t)(w & 15), r = (int64_t)((w >> 4) & 15);
+    const int64_t tile = (int64_t)(w >> 8);
+    WordPos p;
+    p.n = (tile / steps) * 16 + r;
+    p.k0 = (tile % steps) * 256 + kw * 16;
+    return p;
+}
+
+// Stage 3: one thread per 32-bit packed word (16 weights).  Weight k0 + 4 j + b goes to bits
+// 8 b + 2 j of the word; code = t + 1; t = sign(w) * [|w| > gamma/2].  Padding words hold code 1.
+__global__ void __launch_bounds__(256) ternarise_pack_kernel(const float *W, int64_t N, int64_t K, int64_t steps,
+                                                             size_t n_words, const float *gamma, uint32_t *packed) {
     size_t w = (size_t)blockIdx.x * 256 + threadIdx.x;
     if (w >= n_words) return;
-    const float half = 0.5f * *gamma;  // exact
-    uint32_t word = 0;
+    const WordPos p = word_pos(w, steps);
+    uint32_t word = 0x55555555u;
+    if (p.n < N && p.k0 < K) {
+        const float half = 0.5f * *gamma;  // exact
+        const float4 *src = reinterpret_cast<const float4 *>(W + p.n * K + p.k0);
+        word = 0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        float4 v = W4[w * 4 + j];
-        float e[4] = {v.x, v.y, v.z, v.w};
+        for (int j = 0; j < 4; ++j) {
+            float4 v = src[j];
+            float e[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            uint32_t c = e[b] > half ? 2u : (e[b] < -half ? 0u : 1u);
-            word |= c << (8 * b + 2 * j);
+            for (int b = 0; b < 4; ++b) {
+                uint32_t c = e[b] > half ? 2u : (e[b] < -half ? 0u : 1u);
+                word |= c << (8 * b + 2 * j);
+            }
         }
     }
     packed[w] = word;
 }
 
-__global__ void __launch_bounds__(256) unpack_kernel(const uint32_t *packed, size_t n_words, uint4 *T16) {
+__global__ void __launch_bounds__(256) unpack_kernel(const uint32_t *packed, int64_t N, int64_t K, int64_t steps,
+                                                     size_t n_words, int8_t *T) {
     size_t w = (size_t)blockIdx.x * 256 + threadIdx.x;
     if (w >= n_words) return;
+    const WordPos p = word_pos(w, steps);
+    if (p.n >= N || p.k0 >= K) return;
     uint32_t word = packed[w];
     uint32_t o[4];
 #pragma unroll
@@ -73,7 +96,7 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t *packed, siz
         }
         o[j] = r;
     }
-    T16[w] = make_uint4(o[0], o[1], o[2], o[3]);
+    *reinterpret_cast<uint4 *>(T + p.n * K + p.k0) = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 }  // namespace hgf
@@ -82,7 +105,7 @@ using namespace hgf;
 
 extern "C" size_t hgf_packed_bytes(int64_t d_out, int64_t d_in) {
     if (d_out <= 0 || d_in <= 0 || d_in % 64 != 0) return 0;
-    return (size_t)d_out * (size_t)d_in / 4;
+    return (size_t)row_tiles(d_out) * 16 * (size_t)padded_k(d_in) / 4;
 }
 
 extern "C" hgf_status hgf_pack_ternary(const float *W, int64_t d_out, int64_t d_in, void *packed,
@@ -98,9 +121,10 @@ extern "C" hgf_status hgf_pack_ternary(const float *W, int64_t d_out, int64_t d_
     float *gamma_dev = (float *)((char *)tmp + kAbsBlocks * sizeof(double));
     abs_sum_partial_kernel<<<kAbsBlocks, kAbsThreads, 0, stream>>>((const float4 *)W, n / 4, partials);
     abs_sum_final_kernel<<<1, 32, 0, stream>>>(partials, kAbsBlocks, (double)n, gamma_dev);
-    size_t n_words = n / 16;
-    ternarise_pack_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, stream>>>(
-        (const float4 *)W, n_words, gamma_dev, (uint32_t *)packed);
+    const int64_t steps = padded_k(d_in) / 256;
+    size_t n_words = (size_t)row_tiles(d_out) * (size_t)steps * 256;
+    ternarise_pack_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, stream>>>(W, d_out, d_in, steps, n_words, gamma_dev,
+                                                                                 (uint32_t *)packed);
     count_launch(3);
     cudaError_t e = cudaMemcpyAsync(gamma_out, gamma_dev, sizeof(float), cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
@@ -114,9 +138,10 @@ extern "C" hgf_status hgf_unpack_ternary(const void *packed, int64_t d_out, int6
     if (!packed || !T || d_out <= 0 || d_in <= 0) return HGF_ERR_INVALID_ARG;
     if (d_in % 64 != 0) return HGF_ERR_UNSUPPORTED_SHAPE;
     if (((uintptr_t)T | (uintptr_t)packed) & 15) return HGF_ERR_MISALIGNED;
-    size_t n_words = (size_t)d_out * (size_t)d_in / 16;
-    unpack_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, (cudaStream_t)stream_>>>(
-        (const uint32_t *)packed, n_words, (uint4 *)T);
+    const int64_t steps = padded_k(d_in) / 256;
+    size_t n_words = (size_t)row_tiles(d_out) * (size_t)steps * 256;
+    unpack_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, (cudaStream_t)stream_>>>((const uint32_t *)packed, d_out, d_in,
+                                                                                        steps, n_words, T);
     count_launch(1);
     return cudaGetLastError() == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
 }

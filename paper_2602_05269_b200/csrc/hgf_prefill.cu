@@ -5,7 +5,8 @@
 //
 // One persistent CTA per SM, 10 warps with fixed roles:
 //   warp 0      TMA producer: per 128-wide k block, the int8 activation tile (128 tokens x 128 B,
-//               128-byte swizzle) and the packed weight tile (256 rows x 32 B)
+//               128-byte swizzle) and the packed weight tile (256 rows x 32 B, gathered
+//               from 16 consecutive row tiles of the tiled weight layout)
 //   warp 1      allocates tensor memory; one lane issues the MMAs and commits to mbarriers
 //   warps 2-5   epilogue: stage the LoRA operands of the tile, then read both accumulators with
 //               tcgen05.ld, combine, and write through shared memory with TMA stores
@@ -105,6 +106,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int x, int y, uint32_t src) {
@@ -226,7 +233,9 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     if (!(ok = mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x100u + s))) break;
                     mbar_arrive_expect_tx(bar(BAR_FULL + s), X_TILE_BYTES + P_TILE_BYTES);
                     tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, m0, bar(BAR_FULL + s));
-                    tma_load_2d(sbase + OFF_P + s * P_TILE_BYTES, &tmap_w, kb * (KBLK / 4), n0, bar(BAR_FULL + s));
+                    // packed weights: bytes 32 (kb % 2) .. + 31 of the 16 rows of column tile kb / 2, for 16 row tiles
+                    tma_load_4d(sbase + OFF_P + s * P_TILE_BYTES, &tmap_w, (kb & 1) * 32, 0, kb >> 1, n0 >> 4,
+                                bar(BAR_FULL + s));
                     ++issued[s];
                     if (++s == XSTAGES) { s = 0; ph ^= 1u; }
                 }
@@ -490,9 +499,19 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
     if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.xq, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.K, KBLK, TILE_M,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;
-    if (!make_map_2d(&mw, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.packed, (uint64_t)p.K / 4, (uint64_t)p.N, (uint64_t)p.K / 4,
-                     KBLK / 4, TILE_N, CU_TENSOR_MAP_SWIZZLE_NONE))
-        return cudaErrorInvalidValue;
+    {   // packed weights as a 4-D byte tensor: (byte in row: 64, row in tile: 16, column tile, row tile)
+        EncodeTiledFn fn = get_encode_fn();
+        if (!fn) return cudaErrorInvalidValue;
+        const uint64_t steps = (uint64_t)padded_k(p.K) / 256;
+        cuuint64_t dims[4] = {64, 16, steps, (uint64_t)row_tiles(p.N)};
+        cuuint64_t strides[3] = {64, 1024, steps * 1024};
+        cuuint32_t box[4] = {KBLK / 4, 16, 1, TILE_N / 16};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (fn(&mw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<uint8_t *>(p.packed), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
     if (!make_map_2d(&my, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, p.y, (uint64_t)p.N,
                      (uint64_t)p.M, (uint64_t)p.N * (bf16 ? 2 : 4), bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;

@@ -89,58 +89,111 @@ __device__ void quant_row(const PrologueParams &p, int m) {
     }
 }
 
-// One block computes column j of H for up to 16 tokens: H[m][j] = act(sum_k x[m][k] A[k][j]).
-// fp32 accumulation of exact bf16 x fp16 products.
-__device__ void lora_down_column(const PrologueParams &p, int j) {
-    __shared__ float s_part[kWarps][HGF_DECODE_MAX_M];
-    const int K = p.K, M = p.M, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint4 *av = reinterpret_cast<const uint4 *>(p.At + (size_t)j * K);
-    const int nv = K / 8;
-    float acc[HGF_DECODE_MAX_M];
-#pragma unroll
-    for (int m = 0; m < HGF_DECODE_MAX_M; ++m) acc[m] = 0.0f;
+__device__ __forceinline__ void mma_tf32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                         uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint4 ldg_nc_u4(const void *ptr) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(ptr));
+    return v;
+}
 
-    for (int i = tid; i < nv; i += kThreads) {
-        uint4 a4 = av[i];
-        float a[8];
-        {
-            const __half2 *h2 = reinterpret_cast<const __half2 *>(&a4);
+// One block computes 16 columns of H (rows 16 jt .. 16 jt + 15 of A^T) for up to 16 tokens:
+// H[m][j] = act(sum_k x[m][k] A[k][j]) on the warp-level tf32 MMA.  bf16 and fp16 values are both
+// exactly representable in tf32 (8 exponent, 10 mantissa bits), so the products are formed from
+// exact inputs and accumulated in fp32.  The rows of A^T are the 16-row operand, the tokens the
+// 8-column operand; the warps split K in 32-element chunks and their partial sums are added in a
+// fixed order through shared memory.  NT = number of 8-token tiles.
+template <int NT>
+__device__ void lora_down_tile(const PrologueParams &p, int jt) {
+    __shared__ float s_red[kWarps][NT * 4][32];
+    const int K = p.K, M = p.M, r = p.r, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    const __half *rowA = p.At + (size_t)(16 * jt + g) * K + 8 * t;
+    const __half *rowB = rowA + (size_t)8 * K;
+    const __nv_bfloat16 *xr[NT];
+    bool tok_ok[NT];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                float2 f = __half22float2(h2[q]);
-                a[2 * q] = f.x;
-                a[2 * q + 1] = f.y;
+    for (int nt = 0; nt < NT; ++nt) {
+        tok_ok[nt] = g + 8 * nt < M;
+        xr[nt] = p.x + (size_t)(tok_ok[nt] ? g + 8 * nt : 0) * K + 8 * t;
+    }
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[nt][c] = 0.0f;
+
+    const int nchunks = K / 32;
+    constexpr int U = 4;  // chunks in flight per warp
+    for (int c0 = warp; c0 < nchunks; c0 += U * kWarps) {
+        uint4 av[U], bv[U], xv[U][NT];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int c = c0 + u * kWarps;
+            av[u] = bv[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (c < nchunks) {
+                av[u] = ldg_nc_u4(rowA + 32 * c);
+                bv[u] = ldg_nc_u4(rowB + 32 * c);
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                xv[u][nt] = make_uint4(0u, 0u, 0u, 0u);
+                if (c < nchunks && tok_ok[nt]) xv[u][nt] = *reinterpret_cast<const uint4 *>(xr[nt] + 32 * c);
             }
         }
 #pragma unroll
-        for (int m = 0; m < HGF_DECODE_MAX_M; ++m) {
-            if (m < M) {
-                uint4 x4 = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K)[i];
-                uint32_t w[4] = {x4.x, x4.y, x4.z, x4.w};
-                float s = acc[m];
+        for (int u = 0; u < U; ++u) {
+            const uint32_t aw[4] = {av[u].x, av[u].y, av[u].z, av[u].w};
+            const uint32_t bw[4] = {bv[u].x, bv[u].y, bv[u].z, bv[u].w};
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    s = fmaf(bf16lo_to_float(w[q]), a[2 * q], s);
-                    s = fmaf(bf16hi_to_float(w[q]), a[2 * q + 1], s);
+            for (int i = 0; i < 4; ++i) {
+                // elements 2 i and 2 i + 1 of this lane's eight take the k slots t and t + 4 of the MMA
+                const float2 fa = __half22float2(*reinterpret_cast<const __half2 *>(&aw[i]));
+                const float2 fb = __half22float2(*reinterpret_cast<const __half2 *>(&bw[i]));
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint32_t xw = (&xv[u][nt].x)[i];
+                    mma_tf32(acc[nt], __float_as_uint(fa.x), __float_as_uint(fb.x), __float_as_uint(fa.y),
+                             __float_as_uint(fb.y), xw << 16, xw & 0xffff0000u);
                 }
-                acc[m] = s;
             }
         }
     }
 #pragma unroll
-    for (int m = 0; m < HGF_DECODE_MAX_M; ++m) {
-        float v = warp_sum_f(acc[m]);
-        if (lane == 0) s_part[warp][m] = v;
-    }
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) s_red[warp][nt * 4 + c][lane] = acc[nt][c];
     __syncthreads();
-    if (tid < M) {
+    if (tid < NT * 4 * 32) {
+        const int idx = tid >> 5, ln = tid & 31, nt = idx >> 2, c = idx & 3;
         float z = 0.0f;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) z += s_part[w][tid];
-        float h = (p.flags & HGF_FLAG_NO_SILU) ? z : silu_f(z);
-        p.h[(size_t)tid * p.r + j] = h;
-        if (p.dbg_h) p.dbg_h[(size_t)tid * p.r + j] = h;
+        for (int w = 0; w < kWarps; ++w) z += s_red[w][idx][ln];
+        // accumulator register c of lane (g, t): row g + 8 (c >> 1), token 8 nt + 2 t + (c & 1)
+        const int j = 16 * jt + (ln >> 2) + 8 * (c >> 1), m = 8 * nt + 2 * (ln & 3) + (c & 1);
+        if (m < M) {
+            const float h = (p.flags & HGF_FLAG_NO_SILU) ? z : silu_f(z);
+            const size_t o = (size_t)m * r + j;
+            p.h[o] = h;
+            if (p.dbg_h) p.dbg_h[o] = h;
+            if (p.h_hi) {
+                const __half hi = __float2half_rn(h);
+                p.h_hi[o] = hi;
+                p.h_lo[o] = __float2half_rn(h - __half2float(hi));
+            }
+        }
     }
+}
+
+__device__ __forceinline__ void lora_down_block(const PrologueParams &p, int jt) {
+    if (p.M <= 8) lora_down_tile<1>(p, jt); else lora_down_tile<2>(p, jt);
 }
 
 __global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p) {
@@ -151,14 +204,14 @@ __global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p)
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 
-// Decode prologue: blocks [0, M) quantise one token each, blocks [M, M + r) compute one column of H.
+// Decode prologue: blocks [0, M) quantise one token each, blocks [M, M + r / 16) compute 16 columns of H.
 __global__ void __launch_bounds__(kThreads) decode_prologue_kernel(const PrologueParams p) {
     pdl_launch_dependents();  // the GEMV that follows may start streaming its weights
     pdl_wait();               // x, and the workspace this kernel overwrites, belong to earlier work
     if ((int)blockIdx.x < p.M)
         quant_row(p, blockIdx.x);
     else
-        lora_down_column(p, blockIdx.x - p.M);
+        lora_down_block(p, blockIdx.x - p.M);
 }
 
 // The same for a group of problems: blk_begin[i] = first block of problem i (n + 1 entries).
@@ -176,7 +229,7 @@ __global__ void __launch_bounds__(kThreads) decode_prologue_group_kernel(const P
     if (b < p.M)
         quant_row(p, b);
     else
-        lora_down_column(p, b - p.M);
+        lora_down_block(p, b - p.M);
 }
 
 // ---- GEMM-path LoRA down-projection on tensor cores (legacy warp MMA, tf32 inputs) -----------
@@ -186,15 +239,6 @@ __global__ void __launch_bounds__(kThreads) decode_prologue_group_kernel(const P
 // partial sums are reduced through shared memory.
 constexpr int kLdThreads = 128;
 constexpr int kLdTokens = 32;
-
-__device__ __forceinline__ void mma_tf32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                         uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};\n"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 
 template <int JT>  // r = 8 * JT column tiles
 __global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const PrologueParams p) {
@@ -299,7 +343,7 @@ static cudaLaunchConfig_t prologue_cfg(int blocks, bool pdl, cudaStream_t stream
 
 cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream_t stream) {
     cudaLaunchAttribute attr[1];
-    cudaLaunchConfig_t cfg = prologue_cfg(p.M + p.r, pdl, stream, attr);
+    cudaLaunchConfig_t cfg = prologue_cfg(p.M + p.r / 16, pdl, stream, attr);
     cudaError_t e = cudaLaunchKernelEx(&cfg, decode_prologue_kernel, p);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();

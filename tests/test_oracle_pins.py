@@ -74,38 +74,55 @@ def test_ternary_ties_at_half_gamma_round_to_zero():
 # ------------------------------------------------------------------------------- packed format
 def test_pack_roundtrip_random_and_constant():
     rng = np.random.default_rng(0)
-    for shape in [(1, 16), (3, 64), (17, 208), (64, 512)]:
+    for shape in [(1, 16), (3, 64), (17, 208), (64, 512), (40, 8640 // 8)]:
         T = rng.integers(-1, 2, size=shape, dtype=np.int8)
         P = oracle.pack(T)
-        assert P.size == shape[0] * shape[1] // 4 == oracle.packed_bytes(*shape)
+        rows, cols = -(-shape[0] // 16) * 16, -(-shape[1] // 256) * 256
+        assert P.size == rows * cols // 4 == oracle.packed_bytes(*shape)
         T2, bad = oracle.unpack(P, *shape, return_bad=True)
         assert bad == 0 and np.array_equal(T, T2)
     for v, byte in [(-1, 0x00), (0, 0x55), (1, 0xAA)]:
-        T = np.full((4, 64), v, np.int8)
+        T = np.full((32, 512), v, np.int8)           # exactly 2 x 2 tiles, no padding
         P = oracle.pack(T)
         assert np.all(P == byte)
-        assert np.array_equal(oracle.unpack(P, 4, 64), T)
+        assert np.array_equal(oracle.unpack(P, 32, 512), T)
+    # padding rows and columns hold weight 0 (code 1 -> byte 0x55)
+    T = np.full((3, 64), 1, np.int8)
+    P = oracle.pack(T).reshape(16, 64)               # one tile: 16 rows of 64 bytes
+    assert np.all(P[:3, :16] == 0xAA) and np.all(P[:3, 16:] == 0x55) and np.all(P[3:] == 0x55)
 
 
-def test_pack_every_single_position_of_a_16_byte_group():
-    # one 16-byte group = 64 weights; weight k = 16 i + 4 j + b lives in byte 4 i + b, bits 2 j, 2 j + 1
-    for k in range(64):
-        for v in (-1, 1):
-            T = np.zeros((1, 64), np.int8)
-            T[0, k] = v
+def test_pack_every_single_position_of_two_tiles_and_tile_order():
+    # inside a tile: row n at byte 64 n; column c = 16 i + 4 j + b in byte 4 i + b, bits 2 j, 2 j + 1
+    for n in (0, 5, 15):
+        for k in range(512):
+            v = 1 if (n + k) % 2 else -1
+            T = np.zeros((16, 512), np.int8)
+            T[n, k] = v
             P = oracle.pack(T)
-            i, j, b = k // 16, (k % 16) // 4, k % 4
-            expect = np.full(16, 0x55, np.uint8)
-            expect[4 * i + b] = (0x55 & ~(3 << (2 * j))) | ((v + 1) << (2 * j))
-            assert np.array_equal(P, expect), k
-            assert np.array_equal(oracle.unpack(P, 1, 64), T)
+            tile, c = k // 256, k % 256
+            i, j, b = c // 16, (c % 16) // 4, c % 4
+            expect = np.full(2048, 0x55, np.uint8)
+            expect[tile * 1024 + n * 64 + 4 * i + b] = (0x55 & ~(3 << (2 * j))) | ((v + 1) << (2 * j))
+            assert np.array_equal(P, expect), (n, k)
+            assert np.array_equal(oracle.unpack(P, 16, 512), T)
+    # tiles: column tiles of one row tile are adjacent, the next row tile follows them
+    T = np.zeros((33, 520), np.int8)                 # 3 row tiles x 3 column tiles
+    T[32, 519] = 1                                   # row tile 2, row 0; column tile 2, column 7
+    P = oracle.pack(T)
+    assert P.size == 48 * 768 // 4
+    (pos,) = np.nonzero(P != 0x55)
+    assert pos.tolist() == [(2 * 3 + 2) * 1024 + 0 * 64 + 0 * 4 + 3] and P[pos[0]] == (0x55 & ~(3 << 2)) | (2 << 2)
 
 
 def test_unpack_flags_invalid_code():
-    P = np.full(16, 0x55, np.uint8)
-    P[5] = 0x55 | 0x0C  # code 3 in slot j = 1
+    P = np.full(1024, 0x55, np.uint8)
+    P[5] = 0x55 | 0x0C  # code 3 in slot j = 1 of row 0, word 1
     T, bad = oracle.unpack(P, 1, 64, return_bad=True)
     assert bad == 1 and np.all(T == 0)
+    P[64 * 7] = 0xFF    # row 7 is padding for a one-row matrix: not counted
+    T, bad = oracle.unpack(P, 1, 64, return_bad=True)
+    assert bad == 1
 
 
 # ------------------------------------------------------------------------ activation quantisation
