@@ -100,6 +100,7 @@ struct DecodeLaunch {
     long long total_cost;        // 1 KiB weight tiles of all problems
     int max_M;                   // largest token count of any problem
     int xq_smem_bytes;           // shared memory for the largest problem's activations
+    int ring_slots;              // weight-ring slots per warp (set by the launcher)
 };
 
 // host-side launchers (each enqueues on `stream` and returns the CUDA error of the launch)

@@ -25,27 +25,34 @@ namespace hgf {
 
 constexpr int kDecWarps = 16;
 constexpr int kDecThreads = kDecWarps * 32;
-constexpr int kSlots = 6;            // 1 KiB slots per warp ring
-constexpr int kSlotBytes = 1024;
+constexpr int kTileBytes = 1024;     // one 16 x 256 weight tile
+constexpr int kSlotTiles = 2;        // tiles per ring slot
+constexpr int kSlotBytes = kSlotTiles * kTileBytes;
+constexpr int kMaxSlots = 4;         // slots per warp ring (fewer when the activations need the room)
+constexpr int kMinSlots = 3;
 constexpr int kXqPad = 64;           // row padding of the activations in shared memory (bank spread)
 constexpr int kHPitch = 72;          // halves per row of H in shared memory (r <= 64, + 8 bank spread)
 
-// shared-memory map
-constexpr int kOffRing = 0;
-constexpr int kOffBars = kOffRing + kDecWarps * kSlots * kSlotBytes;
-constexpr int kOffSmall = kOffBars + kDecWarps * kSlots * 8;
+// shared-memory map: fixed part, then the activations, then the rings
+constexpr int kOffBars = 0;
+constexpr int kOffSmall = kOffBars + kDecWarps * kMaxSlots * 8;
 struct SegSmall {                    // per-problem values the epilogue needs
     float scale[16];                 // gamma_x[m] * gamma_W / 127
     int row_sum[16];
     __half h_hi[16][kHPitch];
     __half h_lo[16][kHPitch];
+    void *y;
+    int32_t *dbg_y_int;
+    const float *gate;
+    uint32_t flags;
+    int pad;
 };
 constexpr int kOffRed = kOffSmall + 2 * (int)sizeof(SegSmall);
 constexpr int kRedBytes = kDecWarps * 8 * 32 * 4;  // per warp: up to 8 accumulator registers per lane
 constexpr int kOffFlags = kOffRed + kRedBytes;
-constexpr int kOffXq = kOffFlags + 64;
+constexpr int kOffXq = (kOffFlags + 64 + 127) / 128 * 128;
 constexpr int kSmemLimit = 227 * 1024;
-constexpr int kXqLimit = (kSmemLimit - kOffXq) / 1024 * 1024;
+constexpr int kXqLimit = (kSmemLimit - kOffXq - kMinSlots * kDecWarps * kSlotBytes) / 128 * 128;
 
 constexpr unsigned long long kDecWaitLimitNs = 2000000000ull;  // bounded waits give up after two seconds
 
@@ -193,14 +200,16 @@ __device__ __forceinline__ Item seg_item(const Seg &s, int round, int warp) {
     return it;
 }
 
-// The copy-issuing side of a warp's ring: walks the same item sequence as the consumer, one 1 KiB
-// tile per call.  All lanes keep the (warp-uniform) state; lane 0 issues.
+// The copy-issuing side of a warp's ring: walks the same item sequence as the consumer.  All
+// lanes keep the (warp-uniform) state; lane 0 issues.
 struct Producer {
     Seg seg;
-    int round, rounds, ks, ks1;
-    const uint8_t *src;      // next 1 KiB tile of the current item
-    bool have_item, done;
-    uint32_t seq;            // tiles issued so far
+    int round, rounds;
+    int left;                // 1 KiB tiles of the current item not yet requested
+    const uint8_t *src;      // the next of them
+    const __half *bt_src;    // rows of B^T the item's epilogue reads (requested after its last tile)
+    int bt_bytes;            // 0 when the item has no epilogue of its own or the layer has no correction
+    bool done;
 };
 
 // NT = number of 8-token tiles (1: M <= 8, 2: M <= 16).
@@ -209,9 +218,10 @@ __global__ void __launch_bounds__(kDecThreads, 1)
 decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned int *status) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-    uint8_t *ring = smem + kOffRing + warp * kSlots * kSlotBytes;
+    const int slots = L.ring_slots;  // slots of this warp's ring, kSlotBytes each
+    uint8_t *ring = smem + kOffXq + ((L.xq_smem_bytes + 127) & ~127) + warp * slots * kSlotBytes;
     const uint32_t ring_u32 = dsmem_u32(ring);
-    const uint32_t bars_u32 = dsmem_u32(smem + kOffBars) + warp * kSlots * 8;
+    const uint32_t bars_u32 = dsmem_u32(smem + kOffBars) + warp * kMaxSlots * 8;
     SegSmall *small = reinterpret_cast<SegSmall *>(smem + kOffSmall);
     int *red = reinterpret_cast<int *>(smem + kOffRed);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffFlags);
@@ -220,7 +230,7 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
     pdl_launch_dependents();
     if (tid == 0) *abort_flag = 0;
     if (lane == 0) {
-        for (int s = 0; s < kSlots; ++s) dmbar_init(bars_u32 + 8 * s, 1);
+        for (int s = 0; s < slots; ++s) dmbar_init(bars_u32 + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     __syncthreads();
@@ -232,15 +242,15 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
     const int t1 = (blockIdx.x + 1 == gridDim.x) ? L.total_tiles : tile_of_cost(L, single, c1);
 
     // ---- producer ------------------------------------------------------------------------------
+    // A slot receives up to kSlotTiles consecutive tiles of one item; items are cut into slots from
+    // their first tile on, so the consumer knows each slot's size from its own position.
     Producer pr;
-    pr.seq = 0; pr.have_item = false; pr.round = 0; pr.rounds = 0; pr.ks = pr.ks1 = 0; pr.src = nullptr;
+    pr.left = 0; pr.round = -1; pr.rounds = 0; pr.src = nullptr; pr.bt_src = nullptr; pr.bt_bytes = 0;
     pr.done = !next_segment(L, single, t0, t1, true, pr.seg);
-    if (!pr.done) { pr.rounds = seg_rounds(pr.seg); pr.round = -1; }
+    if (!pr.done) pr.rounds = seg_rounds(pr.seg);
 
-    auto produce = [&]() {
-        // move to the next 1 KiB tile of this warp's sequence, if any, and issue its copy
-        while (!pr.done && (!pr.have_item || pr.ks >= pr.ks1)) {
-            pr.have_item = false;
+    auto next_item = [&]() {  // slow path of the producer: find this warp's next item with work
+        while (!pr.done && pr.left == 0) {
             if (++pr.round >= pr.rounds) {
                 if (!next_segment(L, single, t0, t1, false, pr.seg)) { pr.done = true; break; }
                 pr.rounds = seg_rounds(pr.seg);
@@ -248,104 +258,148 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
             }
             const Item it = seg_item(pr.seg, pr.round, warp);
             if (it.valid && it.ks0 < it.ks1) {
-                pr.have_item = true;
-                pr.ks = it.ks0; pr.ks1 = it.ks1;
-                pr.src = pr.seg.packed + ((size_t)it.tile_local * pr.seg.nsteps + it.ks0) * kSlotBytes;
-                if (lane == 0 && it.slice == 0) {  // the rows of B^T and the gates this item's epilogue will read
+                pr.left = it.ks1 - it.ks0;
+                pr.src = pr.seg.packed + ((size_t)it.tile_local * pr.seg.nsteps + it.ks0) * kTileBytes;
+                if (it.slice == 0) {  // this warp runs the row tile's epilogue
                     const DecodeProblem &P = problem_of(L, single, pr.seg.p);
-                    if (P.r > 0) {
-                        const int n0 = it.tile_local * 16, rows = P.N - n0 < 16 ? P.N - n0 : 16;
-                        bulk_prefetch_l2(P.Bt + (size_t)n0 * P.r, (uint32_t)(rows * P.r * 2));
-                        prefetch_l2(P.gate + n0);
-                    }
+                    const int r = P.r, n0 = it.tile_local * 16, rows = P.N - n0 < 16 ? P.N - n0 : 16;
+                    pr.bt_bytes = rows * r * 2;
+                    pr.bt_src = P.Bt + (size_t)n0 * r;
                 }
             }
         }
-        if (pr.done) return;
-        if (lane == 0) {
-            const uint32_t slot = pr.seq % kSlots;
-            bulk_load(ring_u32 + slot * kSlotBytes, pr.src, kSlotBytes, bars_u32 + 8 * slot);
+    };
+    // Request the next slot's worth of this warp's sequence into `slot`: up to kSlotTiles consecutive
+    // tiles of an item, or (after the item's last tile) the rows of B^T for its epilogue.
+    auto produce = [&](int slot) {
+        const uint32_t dst = ring_u32 + slot * kSlotBytes, bar = bars_u32 + 8 * slot;
+        if (pr.left == 0) {
+            if (pr.bt_bytes) {
+                if (lane == 0) bulk_load(dst, pr.bt_src, (uint32_t)pr.bt_bytes, bar);
+                pr.bt_bytes = 0;
+                return;
+            }
+            next_item();
+            if (pr.done) return;
         }
-        pr.src += kSlotBytes;
-        ++pr.ks;
-        ++pr.seq;
+        const int n = pr.left < kSlotTiles ? pr.left : kSlotTiles;
+        if (lane == 0) bulk_load(dst, pr.src, (uint32_t)(n * kTileBytes), bar);
+        pr.src += n * kTileBytes;
+        pr.left -= n;
     };
 #pragma unroll 1
-    for (int i = 0; i < kSlots; ++i) produce();
+    for (int i = 0; i < slots; ++i) produce(i);
 
     // everything above reads only weights; the activations come from the preceding launch
     pdl_wait();
 
     // ---- consumer ------------------------------------------------------------------------------
-    uint32_t cseq = 0;  // tiles consumed so far
-    bool ok = true;     // false once a wait gave up (this warp stops computing but keeps the barriers)
+    int cslot = 0;          // slot the next tiles arrive in
+    uint32_t cpar = 0;      // and its mbarrier phase
+    bool ok = true;         // false once a wait gave up (this warp stops computing but keeps the barriers)
     Seg seg;
     int seg_idx = 0;
     for (bool more = next_segment(L, single, t0, t1, true, seg); more;
          more = next_segment(L, single, t0, t1, false, seg), ++seg_idx) {
-        const DecodeProblem &P = problem_of(L, single, seg.p);
-        const int K = P.K, M = P.M, N = P.N, r = P.r;
+        const DecodeProblem &Pg = problem_of(L, single, seg.p);
+        const int K = Pg.K, M = Pg.M, N = Pg.N, r = Pg.r;
         const int Kp = seg.nsteps * 256, pitch = Kp + kXqPad;
         SegSmall &sm = small[seg_idx & 1];
 
         // stage the problem's activations and per-token values (all reads of the previous
         // segment's activations ended at the barrier that closed it)
         {
+            const int8_t *xq_g = Pg.xq;
             const int units_per_row = Kp >> 4;
             for (int u = tid; u < M * units_per_row; u += kDecThreads) {
                 const int m = u / units_per_row, q = u - m * units_per_row;
                 uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (16 * q < K) v = *reinterpret_cast<const uint4 *>(P.xq + (size_t)m * K + 16 * q);
+                if (16 * q < K) v = *reinterpret_cast<const uint4 *>(xq_g + (size_t)m * K + 16 * q);
                 // inside each 256-byte group the sixteen 16-byte units are stored transposed (4 x 4),
                 // so that the four units a lane reads for one tile are 64 bytes apart
                 const int ql = q & 15, qt = (ql >> 2) + ((ql & 3) << 2);
                 *reinterpret_cast<uint4 *>(xq_s + (size_t)m * pitch + ((q >> 4) << 8) + (qt << 4)) = v;
             }
             if (tid < 16) {
-                sm.scale[tid] = tid < M ? P.gamma_x[tid] * P.gw_over_127 : 0.0f;
-                sm.row_sum[tid] = tid < M ? P.row_sum[tid] : 0;
+                sm.scale[tid] = tid < M ? Pg.gamma_x[tid] * Pg.gw_over_127 : 0.0f;
+                sm.row_sum[tid] = tid < M ? Pg.row_sum[tid] : 0;
             }
+            if (tid == 32) { sm.y = Pg.y; sm.dbg_y_int = Pg.dbg_y_int; sm.gate = Pg.gate; sm.flags = Pg.flags; }
             const int words = r >> 1;  // 32-bit words per row of H
+            const uint32_t *hi_g = reinterpret_cast<const uint32_t *>(Pg.h_hi), *lo_g = reinterpret_cast<const uint32_t *>(Pg.h_lo);
             for (int u = tid; u < M * words; u += kDecThreads) {
                 const int m = u / words, w = u - m * words;
-                reinterpret_cast<uint32_t *>(&sm.h_hi[m][0])[w] = reinterpret_cast<const uint32_t *>(P.h_hi + (size_t)m * r)[w];
-                reinterpret_cast<uint32_t *>(&sm.h_lo[m][0])[w] = reinterpret_cast<const uint32_t *>(P.h_lo + (size_t)m * r)[w];
+                reinterpret_cast<uint32_t *>(&sm.h_hi[m][0])[w] = hi_g[u];
+                reinterpret_cast<uint32_t *>(&sm.h_lo[m][0])[w] = lo_g[u];
             }
         }
         __syncthreads();
 
+        // Bounded wait for the slot the next part of this warp's sequence arrives in.
+        auto wait_slot = [&]() -> bool {
+            const uint32_t bar = bars_u32 + 8 * cslot;
+            bool got = dmbar_try_wait(bar, cpar);
+            if (__all_sync(0xffffffffu, got)) return true;  // the whole warp takes the same path
+            unsigned long long t_start = 0;
+            uint32_t polls = 0;
+            while (!got && !(got = dmbar_try_wait(bar, cpar))) {
+                if ((++polls & 255u) == 0) {
+                    const unsigned long long now = dec_timer_ns();
+                    if (t_start == 0) t_start = now;
+                    else if (now - t_start > kDecWaitLimitNs || *abort_flag) break;
+                }
+            }
+            if (!got) { *abort_flag = 1; if (lane == 0) atomicExch(status, 0x500u + (unsigned)warp); }
+            return __all_sync(0xffffffffu, got);
+        };
+        auto release_slot = [&]() {  // every lane has read the slot: refill it, move on
+            __syncwarp();
+            produce(cslot);
+            if (++cslot == slots) { cslot = 0; cpar ^= 1u; }
+        };
         // Epilogue of one row tile: dequantise, add the gated rank-r correction, store.  v holds
         // sum_k c x~ in the MMA accumulator layout: register c of token tile nt is row g + 8 (c >> 1),
-        // token 8 nt + 2 t + (c & 1).
-        auto epilogue = [&](int n0, const int (&v)[NT][4]) {
+        // token 8 nt + 2 t + (c & 1).  The correction runs on the f16 MMA: the tile's rows of B^T (which
+        // arrive in a ring slot of their own) are the 16-row operand, H^T (fp16 value + fp16 residual)
+        // the 8-column operand.  Returns false if the wait for B^T gave up.
+        auto epilogue = [&](int n0, const int (&v)[NT][4]) -> bool {
             float corr[NT][4];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                 for (int c = 0; c < 4; ++c) corr[nt][c] = 0.0f;
-            const int nA = n0 + g < N ? n0 + g : N - 1, nB = n0 + g + 8 < N ? n0 + g + 8 : N - 1;
+            float gA = 0.0f, gB = 0.0f;
             if (r > 0) {
-                // B^T rows are the 16-row operand, H^T (fp16 value + fp16 residual) the 8-column one
-                const uint32_t *bA = reinterpret_cast<const uint32_t *>(P.Bt + (size_t)nA * r);
-                const uint32_t *bB = reinterpret_cast<const uint32_t *>(P.Bt + (size_t)nB * r);
-                for (int kk = 0; kk < (r >> 4); ++kk) {
-                    const uint32_t a0 = __ldg(bA + 8 * kk + t), a1 = __ldg(bB + 8 * kk + t);
-                    const uint32_t a2 = __ldg(bA + 8 * kk + 4 + t), a3 = __ldg(bB + 8 * kk + 4 + t);
+                const float *gate = sm.gate;
+                gA = __ldg(gate + (n0 + g < N ? n0 + g : N - 1));
+                gB = __ldg(gate + (n0 + g + 8 < N ? n0 + g + 8 : N - 1));
+                if (!wait_slot()) return false;
+                const int rows = N - n0 < 16 ? N - n0 : 16;
+                const uint32_t *bA = reinterpret_cast<const uint32_t *>(ring + cslot * kSlotBytes) + (g < rows ? g : rows - 1) * (r >> 1) + t;
+                const uint32_t *bB = reinterpret_cast<const uint32_t *>(ring + cslot * kSlotBytes) + (g + 8 < rows ? g + 8 : rows - 1) * (r >> 1) + t;
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        uint32_t h0 = 0, h1 = 0, l0 = 0, l1 = 0;
-                        if (g + 8 * nt < M) {
-                            const uint32_t *hh = reinterpret_cast<const uint32_t *>(&sm.h_hi[g + 8 * nt][0]);
-                            const uint32_t *hl = reinterpret_cast<const uint32_t *>(&sm.h_lo[g + 8 * nt][0]);
-                            h0 = hh[8 * kk + t]; h1 = hh[8 * kk + 4 + t];
-                            l0 = hl[8 * kk + t]; l1 = hl[8 * kk + 4 + t];
+                for (int kk = 0; kk < 4; ++kk) {
+                    if (16 * kk < r) {
+                        const uint32_t a0 = bA[8 * kk], a1 = bB[8 * kk], a2 = bA[8 * kk + 4], a3 = bB[8 * kk + 4];
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            uint32_t h0 = 0, h1 = 0, l0 = 0, l1 = 0;
+                            if (g + 8 * nt < M) {
+                                const uint32_t *hh = reinterpret_cast<const uint32_t *>(&sm.h_hi[g + 8 * nt][0]);
+                                const uint32_t *hl = reinterpret_cast<const uint32_t *>(&sm.h_lo[g + 8 * nt][0]);
+                                h0 = hh[8 * kk + t]; h1 = hh[8 * kk + 4 + t];
+                                l0 = hl[8 * kk + t]; l1 = hl[8 * kk + 4 + t];
+                            }
+                            mma_f16(corr[nt], a0, a1, a2, a3, h0, h1);
+                            mma_f16(corr[nt], a0, a1, a2, a3, l0, l1);
                         }
-                        mma_f16(corr[nt], a0, a1, a2, a3, h0, h1);
-                        mma_f16(corr[nt], a0, a1, a2, a3, l0, l1);
                     }
                 }
+                release_slot();
             }
-            const float gA = r > 0 ? __ldg(P.gate + nA) : 0.0f, gB = r > 0 ? __ldg(P.gate + nB) : 0.0f;
+            void *y_out = sm.y;
+            int32_t *dbg_y_int = sm.dbg_y_int;
+            const bool out_bf16 = (sm.flags & HGF_FLAG_OUT_BF16) != 0;
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -355,24 +409,32 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
                         const int y_int = v[nt][c] - sm.row_sum[m];
                         const float y = fmaf(c >> 1 ? gB : gA, corr[nt][c], (float)y_int * sm.scale[m]);
                         const size_t o = (size_t)m * N + n;
-                        if (P.flags & HGF_FLAG_OUT_BF16)
-                            reinterpret_cast<__nv_bfloat16 *>(P.y)[o] = __float2bfloat16_rn(y);
+                        if (out_bf16)
+                            reinterpret_cast<__nv_bfloat16 *>(y_out)[o] = __float2bfloat16_rn(y);
                         else
-                            reinterpret_cast<float *>(P.y)[o] = y;
-                        if (P.dbg_y_int) P.dbg_y_int[o] = y_int;
+                            reinterpret_cast<float *>(y_out)[o] = y;
+                        if (dbg_y_int) dbg_y_int[o] = y_int;
                     }
                 }
+            return true;
         };
 
         const int rounds = seg_rounds(seg);
         const int full_rounds = (seg.hi - seg.lo) / kDecWarps;
-        Item last_it;
-        last_it.valid = false;
-        int v_last[NT][4];
+        int last_tile = -1, last_S = 1;  // the row tile whose epilogue this warp runs after the barrier
+
+        // this lane's activation bytes: token g + 8 nt, 16-byte units t, t + 4, t + 8, t + 12 of each tile
+        const int8_t *xrow[NT];
+        bool tok_ok[NT];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            tok_ok[nt] = g + 8 * nt < M;
+            xrow[nt] = xq_s + (size_t)(tok_ok[nt] ? g + 8 * nt : 0) * pitch + 16 * t;
+        }
 
         for (int round = 0; round < rounds; ++round) {
             const Item it = seg_item(seg, round, warp);
-            if (!it.valid || it.ks0 >= it.ks1) { if (round >= full_rounds) last_it = it; continue; }
+            if (!it.valid || it.ks0 >= it.ks1) continue;
 
             int acc[NT][4][4];
 #pragma unroll
@@ -382,60 +444,42 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
 #pragma unroll
                     for (int c = 0; c < 4; ++c) acc[a][b][c] = 0;
 
-            // this lane's activation bytes of column tile ks: token (g + 8 nt), units t, t+4, t+8, t+12
-            const int8_t *xrow[NT];
-            bool tok_ok[NT];
+            for (int ks = it.ks0; ks < it.ks1 && ok; ks += kSlotTiles) {
+                if (!(ok = wait_slot())) break;  // stop computing and copying; requested slots stay outstanding
+                const uint8_t *sl = ring + cslot * kSlotBytes + 16 * lane;
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                tok_ok[nt] = g + 8 * nt < M;
-                xrow[nt] = xq_s + (size_t)(tok_ok[nt] ? g + 8 * nt : 0) * pitch + 16 * t;
-            }
-
-            for (int ks = it.ks0; ks < it.ks1; ++ks) {
-                const uint32_t slot = cseq % kSlots, parity = (cseq / kSlots) & 1u;
-                if (ok) {
-                    unsigned long long t_start = 0;
-                    uint32_t polls = 0;
-                    while (!dmbar_try_wait(bars_u32 + 8 * slot, parity)) {
-                        if ((++polls & 255u) == 0) {
-                            const unsigned long long now = dec_timer_ns();
-                            if (t_start == 0) t_start = now;
-                            else if (now - t_start > kDecWaitLimitNs || *abort_flag) { ok = false; break; }
+                for (int j = 0; j < kSlotTiles; ++j) {
+                    if (ks + j < it.ks1) {
+                        const uint4 pq = *reinterpret_cast<const uint4 *>(sl + j * kTileBytes);
+                        const uint4 qq = *reinterpret_cast<const uint4 *>(sl + j * kTileBytes + 512);
+                        const uint32_t pw[4] = {pq.x, pq.y, pq.z, pq.w};
+                        const uint32_t qw[4] = {qq.x, qq.y, qq.z, qq.w};
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            uint32_t xa[NT][4], xb[NT][4];
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                uint4 va = make_uint4(0u, 0u, 0u, 0u), vb = va;
+                                if (tok_ok[nt]) {
+                                    va = *reinterpret_cast<const uint4 *>(xrow[nt] + (ks + j) * 256 + 64 * (2 * h));
+                                    vb = *reinterpret_cast<const uint4 *>(xrow[nt] + (ks + j) * 256 + 64 * (2 * h + 1));
+                                }
+                                xa[nt][0] = va.x; xa[nt][1] = va.y; xa[nt][2] = va.z; xa[nt][3] = va.w;
+                                xb[nt][0] = vb.x; xb[nt][1] = vb.y; xb[nt][2] = vb.z; xb[nt][3] = vb.w;
+                            }
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj) {
+                                const uint32_t mask = 0x03030303u << (2 * jj);
+                                const uint32_t a0 = pw[2 * h] & mask, a1 = qw[2 * h] & mask;
+                                const uint32_t a2 = pw[2 * h + 1] & mask, a3 = qw[2 * h + 1] & mask;
+#pragma unroll
+                                for (int nt = 0; nt < NT; ++nt)
+                                    mma_u8s8(acc[nt][jj], a0, a1, a2, a3, xa[nt][jj], xb[nt][jj]);
+                            }
                         }
                     }
-                    if (!ok) { *abort_flag = 1; if (lane == 0) atomicExch(status, 0x500u + (unsigned)warp); }
                 }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) continue;  // stop computing and copying; tiles cseq .. pr.seq - 1 stay outstanding
-                ++cseq;
-                const uint4 pq = *reinterpret_cast<const uint4 *>(ring + slot * kSlotBytes + 16 * lane);
-                const uint4 qq = *reinterpret_cast<const uint4 *>(ring + slot * kSlotBytes + 512 + 16 * lane);
-                __syncwarp();
-                produce();  // refill the slot just read
-                const uint32_t pw[4] = {pq.x, pq.y, pq.z, pq.w};
-                const uint32_t qw[4] = {qq.x, qq.y, qq.z, qq.w};
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t xa[NT][4], xb[NT][4];
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        uint4 va = make_uint4(0u, 0u, 0u, 0u), vb = va;
-                        if (tok_ok[nt]) {
-                            va = *reinterpret_cast<const uint4 *>(xrow[nt] + ks * 256 + 64 * (2 * h));
-                            vb = *reinterpret_cast<const uint4 *>(xrow[nt] + ks * 256 + 64 * (2 * h + 1));
-                        }
-                        xa[nt][0] = va.x; xa[nt][1] = va.y; xa[nt][2] = va.z; xa[nt][3] = va.w;
-                        xb[nt][0] = vb.x; xb[nt][1] = vb.y; xb[nt][2] = vb.z; xb[nt][3] = vb.w;
-                    }
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        const uint32_t mask = 0x03030303u << (2 * jj);
-                        const uint32_t a0 = pw[2 * h] & mask, a1 = qw[2 * h] & mask;
-                        const uint32_t a2 = pw[2 * h + 1] & mask, a3 = qw[2 * h + 1] & mask;
-#pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) mma_u8s8(acc[nt][jj], a0, a1, a2, a3, xa[nt][jj], xb[nt][jj]);
-                    }
-                }
+                release_slot();
             }
 
             // exact rescale of the four accumulators
@@ -446,59 +490,45 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
                 for (int c = 0; c < 4; ++c)
                     v[nt][c] = acc[nt][0][c] + (acc[nt][1][c] >> 2) + (acc[nt][2][c] >> 4) + (acc[nt][3][c] >> 6);
 
-            if (it.S > 1) {  // K slices of a row tile: park the partial sums, add them after the barrier
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) red[(warp * 8 + nt * 4 + c) * 32 + lane] = v[nt][c];
-                last_it = it;
+            if (round < full_rounds) {  // a whole row tile: its epilogue runs right away
+                if (ok) ok = epilogue(it.tile_local * 16, v);
                 continue;
             }
-            if (round >= full_rounds) {  // last round without slicing: its epilogue also runs after the barrier
-                last_it = it;
+            // last round: park the sums (K slices are added after the barrier)
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) v_last[nt][c] = v[nt][c];
-                continue;
-            }
-            if (ok) epilogue(it.tile_local * 16, v);
+                for (int c = 0; c < 4; ++c) red[(warp * 8 + nt * 4 + c) * 32 + lane] = v[nt][c];
+            if (it.slice == 0) { last_tile = it.tile_local; last_S = it.S; }
         }
 
         __syncthreads();  // partial sums are parked; every read of this segment's activations is done
 
         // ---- epilogue of the last round (after adding K slices) ----------------------------------
-        if (ok && last_it.valid && last_it.slice == 0 && last_it.ks0 < last_it.ks1) {
+        if (ok && last_tile >= 0) {
             int v[NT][4];
-            if (last_it.S > 1) {
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        int s = 0;
-                        for (int w = 0; w < last_it.S; ++w) s += red[((warp + w) * 8 + nt * 4 + c) * 32 + lane];
-                        v[nt][c] = s;
-                    }
-            } else {
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) v[nt][c] = v_last[nt][c];
-            }
-            epilogue(last_it.tile_local * 16, v);
+                for (int c = 0; c < 4; ++c) {
+                    int s = 0;
+                    for (int w = 0; w < last_S; ++w) s += red[((warp + w) * 8 + nt * 4 + c) * 32 + lane];
+                    v[nt][c] = s;
+                }
+            ok = epilogue(last_tile * 16, v);
         }
     }
 
     // A warp that stopped early still has copies in flight: wait (bounded) for them before leaving.
     if (!ok) {
-        for (uint32_t q = cseq; q < pr.seq; ++q) {
-            const uint32_t slot = q % kSlots, parity = (q / kSlots) & 1u;
-            for (uint32_t i = 0; i < (1u << 20) && !dmbar_try_wait(bars_u32 + 8 * slot, parity); ++i) {}
+        for (int q = 0; q < slots; ++q) {
+            for (uint32_t i = 0; i < (1u << 16) && !dmbar_try_wait(bars_u32 + 8 * cslot, cpar); ++i) {}
+            if (++cslot == slots) { cslot = 0; cpar ^= 1u; }
         }
     }
 }
 
-cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream) {
+cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *single, bool pdl, cudaStream_t stream) {
     static int sm_count = 0;
     static bool attr_set = false;
     if (!sm_count) {
@@ -515,9 +545,15 @@ cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *singl
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    if (L.xq_smem_bytes > kXqLimit) return cudaErrorInvalidValue;
+    if (L_in.xq_smem_bytes > kXqLimit) return cudaErrorInvalidValue;
     unsigned int *status = device_status_word();
     if (!status) return cudaErrorMemoryAllocation;
+    DecodeLaunch L = L_in;
+    // as many ring slots as shared memory allows beside the activations
+    const int xq_bytes = (L.xq_smem_bytes + 127) & ~127;
+    int slots = (kSmemLimit - kOffXq - xq_bytes) / (kDecWarps * kSlotBytes);
+    slots = slots > kMaxSlots ? kMaxSlots : slots;
+    L.ring_slots = slots;
     const int grid = L.total_tiles < sm_count ? L.total_tiles : sm_count;
     DecodeProblem dummy = {};
     const DecodeProblem &sp = single ? *single : dummy;
@@ -525,7 +561,7 @@ cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *singl
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kDecThreads);
-    cfg.dynamicSmemBytes = (size_t)(kOffXq + L.xq_smem_bytes);
+    cfg.dynamicSmemBytes = (size_t)(kOffXq + xq_bytes + kDecWarps * slots * kSlotBytes);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
