@@ -26,7 +26,7 @@ namespace hgf {
 constexpr int kDecWarps = 16;
 constexpr int kDecThreads = kDecWarps * 32;
 constexpr int kTileBytes = 1024;     // one 16 x 256 weight tile
-constexpr int kSlotTiles = 2;        // tiles per ring slot
+constexpr int kSlotTiles = 2;        // tiles per ring slot (the consumer loop is written for 2)
 constexpr int kSlotBytes = kSlotTiles * kTileBytes;
 constexpr int kMaxSlots = 4;         // slots per warp ring (fewer when the activations need the room)
 constexpr int kMinSlots = 3;
@@ -56,7 +56,9 @@ constexpr int kXqLimit = (kSmemLimit - kOffXq - kMinSlots * kDecWarps * kSlotByt
 
 constexpr unsigned long long kDecWaitLimitNs = 2000000000ull;  // bounded waits give up after two seconds
 
-int decode_xq_smem_bytes(int M, int K) { return M * ((int)padded_k(K) + kXqPad); }
+// Rows of activations kept in shared memory: the M tokens, plus one row of zeros that stands in for
+// the absent tokens of the 8-token tiles.
+int decode_xq_smem_bytes(int M, int K) { return (M + (M < 16 ? 1 : 0)) * ((int)padded_k(K) + kXqPad); }
 int decode_xq_smem_limit() { return kXqLimit; }
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -310,15 +312,27 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
         // segment's activations ended at the barrier that closed it)
         {
             const int8_t *xq_g = Pg.xq;
-            const int units_per_row = Kp >> 4;
-            for (int u = tid; u < M * units_per_row; u += kDecThreads) {
-                const int m = u / units_per_row, q = u - m * units_per_row;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (16 * q < K) v = *reinterpret_cast<const uint4 *>(xq_g + (size_t)m * K + 16 * q);
-                // inside each 256-byte group the sixteen 16-byte units are stored transposed (4 x 4),
-                // so that the four units a lane reads for one tile are 64 bytes apart
-                const int ql = q & 15, qt = (ql >> 2) + ((ql & 3) << 2);
-                *reinterpret_cast<uint4 *>(xq_s + (size_t)m * pitch + ((q >> 4) << 8) + (qt << 4)) = v;
+            // Shared-memory order of a token's bytes, per 256-column tile: the lane with t = lane % 4
+            // owns columns 64 t .. 64 t + 63; of each 32 of them (4-byte groups G0 .. G7) it reads two
+            // 16-byte units, [G0 G4 G1 G5] and [G2 G6 G3 G7], so that the two registers one MMA takes
+            // (columns c .. c + 3 and c + 16 .. c + 19) come out of one load next to each other.  Unit
+            // u = 0 .. 3 of lane t sits at byte 64 u + 16 t of the tile: the four lanes of a token read
+            // 64 consecutive bytes, and the row padding puts the next token on the other banks.
+            const int groups_per_row = Kp >> 5;
+            if (M < 16)  // the row of zeros
+                for (int u = tid; u < (Kp >> 4); u += kDecThreads)
+                    *reinterpret_cast<uint4 *>(xq_s + (size_t)M * pitch + 16 * u) = make_uint4(0u, 0u, 0u, 0u);
+            for (int u = tid; u < M * groups_per_row; u += kDecThreads) {
+                const int m = u / groups_per_row, q = u - m * groups_per_row;
+                uint4 v0 = make_uint4(0u, 0u, 0u, 0u), v1 = v0;
+                if (32 * q < K) {
+                    v0 = *reinterpret_cast<const uint4 *>(xq_g + (size_t)m * K + 32 * q);
+                    v1 = *reinterpret_cast<const uint4 *>(xq_g + (size_t)m * K + 32 * q + 16);
+                }
+                const int tq = q & 7, tt = tq >> 1, h = tq & 1;
+                int8_t *dst = xq_s + (size_t)m * pitch + ((q >> 3) << 8) + 16 * tt + 128 * h;
+                *reinterpret_cast<uint4 *>(dst) = make_uint4(v0.x, v1.x, v0.y, v1.y);
+                *reinterpret_cast<uint4 *>(dst + 64) = make_uint4(v0.z, v1.z, v0.w, v1.w);
             }
             if (tid < 16) {
                 sm.scale[tid] = tid < M ? Pg.gamma_x[tid] * Pg.gw_over_127 : 0.0f;
@@ -423,14 +437,11 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
         const int full_rounds = (seg.hi - seg.lo) / kDecWarps;
         int last_tile = -1, last_S = 1;  // the row tile whose epilogue this warp runs after the barrier
 
-        // this lane's activation bytes: token g + 8 nt, 16-byte units t, t + 4, t + 8, t + 12 of each tile
+        // this lane's activation bytes: token g + 8 nt (an absent token reads the row of zeros), units
+        // at bytes 16 t + 64 u of each tile
         const int8_t *xrow[NT];
-        bool tok_ok[NT];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            tok_ok[nt] = g + 8 * nt < M;
-            xrow[nt] = xq_s + (size_t)(tok_ok[nt] ? g + 8 * nt : 0) * pitch + 16 * t;
-        }
+        for (int nt = 0; nt < NT; ++nt) xrow[nt] = xq_s + (size_t)(g + 8 * nt < M ? g + 8 * nt : M) * pitch + 16 * t;
 
         for (int round = 0; round < rounds; ++round) {
             const Item it = seg_item(seg, round, warp);
@@ -444,42 +455,54 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
 #pragma unroll
                     for (int c = 0; c < 4; ++c) acc[a][b][c] = 0;
 
-            for (int ks = it.ks0; ks < it.ks1 && ok; ks += kSlotTiles) {
-                if (!(ok = wait_slot())) break;  // stop computing and copying; requested slots stay outstanding
-                const uint8_t *sl = ring + cslot * kSlotBytes + 16 * lane;
+            // one 16 x 256 tile at shared-memory address `wt` against the activations at `xt`
+            auto compute_tile = [&](const uint8_t *wt, const int8_t *const (&xt)[NT]) {
+                const uint4 pq = *reinterpret_cast<const uint4 *>(wt);
+                const uint4 qq = *reinterpret_cast<const uint4 *>(wt + 512);
+                const uint32_t pw[4] = {pq.x, pq.y, pq.z, pq.w};
+                const uint32_t qw[4] = {qq.x, qq.y, qq.z, qq.w};
 #pragma unroll
-                for (int j = 0; j < kSlotTiles; ++j) {
-                    if (ks + j < it.ks1) {
-                        const uint4 pq = *reinterpret_cast<const uint4 *>(sl + j * kTileBytes);
-                        const uint4 qq = *reinterpret_cast<const uint4 *>(sl + j * kTileBytes + 512);
-                        const uint32_t pw[4] = {pq.x, pq.y, pq.z, pq.w};
-                        const uint32_t qw[4] = {qq.x, qq.y, qq.z, qq.w};
+                for (int h = 0; h < 2; ++h) {
+                    uint4 xa[NT], xb[NT];
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            uint32_t xa[NT][4], xb[NT][4];
+                    for (int nt = 0; nt < NT; ++nt) {
+                        xa[nt] = *reinterpret_cast<const uint4 *>(xt[nt] + 64 * (2 * h));
+                        xb[nt] = *reinterpret_cast<const uint4 *>(xt[nt] + 64 * (2 * h + 1));
+                    }
 #pragma unroll
-                            for (int nt = 0; nt < NT; ++nt) {
-                                uint4 va = make_uint4(0u, 0u, 0u, 0u), vb = va;
-                                if (tok_ok[nt]) {
-                                    va = *reinterpret_cast<const uint4 *>(xrow[nt] + (ks + j) * 256 + 64 * (2 * h));
-                                    vb = *reinterpret_cast<const uint4 *>(xrow[nt] + (ks + j) * 256 + 64 * (2 * h + 1));
-                                }
-                                xa[nt][0] = va.x; xa[nt][1] = va.y; xa[nt][2] = va.z; xa[nt][3] = va.w;
-                                xb[nt][0] = vb.x; xb[nt][1] = vb.y; xb[nt][2] = vb.z; xb[nt][3] = vb.w;
-                            }
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const uint32_t mask = 0x03030303u << (2 * jj);
+                        const uint32_t a0 = pw[2 * h] & mask, a1 = qw[2 * h] & mask;
+                        const uint32_t a2 = pw[2 * h + 1] & mask, a3 = qw[2 * h + 1] & mask;
 #pragma unroll
-                            for (int jj = 0; jj < 4; ++jj) {
-                                const uint32_t mask = 0x03030303u << (2 * jj);
-                                const uint32_t a0 = pw[2 * h] & mask, a1 = qw[2 * h] & mask;
-                                const uint32_t a2 = pw[2 * h + 1] & mask, a3 = qw[2 * h + 1] & mask;
-#pragma unroll
-                                for (int nt = 0; nt < NT; ++nt)
-                                    mma_u8s8(acc[nt][jj], a0, a1, a2, a3, xa[nt][jj], xb[nt][jj]);
-                            }
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const uint4 &xv = jj < 2 ? xa[nt] : xb[nt];
+                            if (jj & 1) mma_u8s8(acc[nt][jj], a0, a1, a2, a3, xv.z, xv.w);
+                            else mma_u8s8(acc[nt][jj], a0, a1, a2, a3, xv.x, xv.y);
                         }
                     }
                 }
+            };
+            const int8_t *xt[NT];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) xt[nt] = xrow[nt] + it.ks0 * 256;
+            const int ntiles = it.ks1 - it.ks0;
+            for (int i = ntiles >> 1; i > 0 && ok; --i) {  // full slots
+                if (!(ok = wait_slot())) break;  // stop computing and copying; requested slots stay outstanding
+                const uint8_t *sl = ring + cslot * kSlotBytes + 16 * lane;
+                compute_tile(sl, xt);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) xt[nt] += 256;
+                compute_tile(sl + kTileBytes, xt);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) xt[nt] += 256;
                 release_slot();
+            }
+            if ((ntiles & 1) && ok) {  // a last slot with one tile
+                if ((ok = wait_slot())) {
+                    compute_tile(ring + cslot * kSlotBytes + 16 * lane, xt);
+                    release_slot();
+                }
             }
 
             // exact rescale of the four accumulators
