@@ -60,13 +60,19 @@ typedef struct {
 } hgf_debug_out;
 
 /*
- * Size in bytes of the packed form of a d_out x d_in ternary matrix: d_out * d_in / 4.
+ * Size in bytes of the packed form of a d_out x d_in ternary matrix.
  * Packed layout (the paper fixes none; it only states 1.58 bits of information per weight):
- * two bits per weight, code c = t + 1 in {0,1,2}.  Row n occupies d_in/4 bytes from byte
- * n * d_in / 4.  A row is a sequence of little-endian 32-bit words; word i holds weights
- * k = 16 i .. 16 i + 15, and with k = 16 i + 4 j + b (j, b in 0..3) the code of weight k is in
- * bits 8 b + 2 j and 8 b + 2 j + 1.  So (word >> 2 j) & 0x03030303 is four consecutive-k codes,
- * one per byte.  Returns 0 for invalid sizes (d_in % 64 != 0 or non-positive).
+ * two bits per weight, code c = t + 1 in {0,1,2}.  The matrix is cut into tiles of 16 output rows
+ * by 256 input columns; d_out is padded up to a multiple of 16 and d_in up to a multiple of 256
+ * with zero weights (code 1).  A tile is 1024 bytes: its 16 rows one after the other, 64 bytes per
+ * row.  Tiles are stored with the column-tile index running fastest: tile (R, C) starts at byte
+ * (R * (d_in_padded / 256) + C) * 1024, so the 16 rows of a row tile are one contiguous run.  The
+ * 64 bytes of a row are 16 little-endian 32-bit words; word i holds the weights whose column
+ * inside the tile is 16 i .. 16 i + 15, and with that column written 16 i + 4 j + b (j, b in 0..3)
+ * the code sits in bits 8 b + 2 j and 8 b + 2 j + 1.  So (word >> 2 j) & 0x03030303 is four
+ * consecutive-column codes, one per byte.
+ * Returns ceil(d_out / 16) * 16 * ceil(d_in / 256) * 256 / 4, or 0 for invalid sizes
+ * (d_in % 64 != 0 or non-positive).
  */
 size_t hgf_packed_bytes(int64_t d_out, int64_t d_in);
 
@@ -108,7 +114,9 @@ size_t hgf_workspace_bytes(int64_t M, int64_t d_in, int64_t d_out, int32_t r, ui
  * The per-token scale is floored at 1e-5 (an all-zero token yields zeros).
  * Requirements: M >= 1; d_in % 64 == 0; d_out >= 1; r in {0,16,32,48,64}; 16-byte aligned
  * pointers.  M <= HGF_DECODE_MAX_M runs the bandwidth-bound GEMV path, larger M the tcgen05
- * int8 GEMM path (which additionally needs d_in % 128 == 0 and d_out % 8 == 0).
+ * int8 GEMM path (which additionally needs d_out % 8 == 0).  The GEMV path keeps the layer's
+ * quantised activations in shared memory; a problem with (M + 1) * (d_in_padded + 64) above about
+ * 104 KiB (no shape of the paper's model classes at M <= 16) takes the GEMM path as well.
  * Calls on the same workspace must not overlap on the device.
  * Launch overlap: the decode kernels are launched with programmatic stream serialization and start
  * fetching `packed` before the preceding work on `stream` has finished (they wait for that work
@@ -132,7 +140,8 @@ hgf_status hgf_linear_forward(const void *x, int64_t M, const void *packed, floa
  * hgf_group_create records the problems (pointers are kept, not the data: x, y and the weights
  * stay owned by the caller and must stay valid) and allocates the group's descriptors and
  * workspace on the current device; it is a set-up call, not for the hot path.
- * hgf_group_forward only enqueues: one prologue launch and one GEMV launch for the whole group.
+ * hgf_group_forward only enqueues: one prologue launch and one GEMV launch for the whole group,
+ * which streams the packed weights of all its problems as one sequence split evenly over the SMs.
  * Forward calls of one group must not overlap on the device.  hgf_group_destroy frees the group
  * (the caller makes sure no forward is still running).
  */
@@ -154,6 +163,15 @@ typedef struct hgf_group hgf_group;
 hgf_status hgf_group_create(const hgf_problem *problems /* host array */, int32_t n, uint32_t flags,
                             hgf_group **out);
 hgf_status hgf_group_forward(hgf_group *group, void *stream);
+/*
+ * The two launches of hgf_group_forward separately, for measurement: HGF_PHASE_PROLOGUE runs
+ * Algorithm 1 steps 1-2 and 5-6 (activation quantisation, H = SiLU(x A)) into the group's
+ * workspace, HGF_PHASE_GEMV steps 3-4 and 7-8 from what the last prologue left there.  Both bits
+ * together are hgf_group_forward.
+ */
+#define HGF_PHASE_PROLOGUE 0x1u
+#define HGF_PHASE_GEMV 0x2u
+hgf_status hgf_group_forward_phases(hgf_group *group, uint32_t phases, void *stream);
 void hgf_group_destroy(hgf_group *group);
 
 /*

@@ -257,12 +257,14 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     return HGF_OK;
 }
 
-extern "C" hgf_status hgf_group_forward(hgf_group *g, void *stream_) {
-    if (!g) return HGF_ERR_INVALID_ARG;
+extern "C" hgf_status hgf_group_forward_phases(hgf_group *g, uint32_t phases, void *stream_) {
+    if (!g || !phases || (phases & ~(HGF_PHASE_PROLOGUE | HGF_PHASE_GEMV))) return HGF_ERR_INVALID_ARG;
     cudaStream_t stream = (cudaStream_t)stream_;
     const bool pdl = !(g->flags & HGF_FLAG_NO_PDL);
-    if (launch_decode_prologue_group(g->d_pps, g->d_blk_begin, g->n, g->total_blocks, pdl, stream) != cudaSuccess)
+    if ((phases & HGF_PHASE_PROLOGUE) &&
+        launch_decode_prologue_group(g->d_pps, g->d_blk_begin, g->n, g->total_blocks, pdl, stream) != cudaSuccess)
         return HGF_ERR_CUDA;
+    if (!(phases & HGF_PHASE_GEMV)) return HGF_OK;
     DecodeLaunch dl = {};
     dl.probs = g->d_probs;
     dl.n_probs = g->n;
@@ -271,6 +273,10 @@ extern "C" hgf_status hgf_group_forward(hgf_group *g, void *stream_) {
     dl.max_M = g->max_M;
     dl.xq_smem_bytes = g->xq_smem_bytes;
     return launch_decode_gemv(dl, nullptr, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
+}
+
+extern "C" hgf_status hgf_group_forward(hgf_group *g, void *stream) {
+    return hgf_group_forward_phases(g, HGF_PHASE_PROLOGUE | HGF_PHASE_GEMV, stream);
 }
 
 extern "C" void hgf_group_destroy(hgf_group *g) {

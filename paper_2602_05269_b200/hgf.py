@@ -19,12 +19,14 @@ FLAG_NO_SILU = 0x2
 FLAG_FORCE_GEMM = 0x4
 FLAG_NO_PDL = 0x8
 DECODE_MAX_M = 16
+PHASE_PROLOGUE = 0x1
+PHASE_GEMV = 0x2
 
 # every symbol include/hgf.h declares
 EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_workspace_bytes",
            "hgf_linear_forward", "hgf_act_quant", "hgf_check_status", "hgf_tmax_tokens_per_s",
            "hgf_launch_count", "hgf_status_string", "hgf_group_create", "hgf_group_forward",
-           "hgf_group_destroy"]
+           "hgf_group_destroy", "hgf_group_forward_phases"]
 
 
 class HgfError(RuntimeError):
@@ -81,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.hgf_group_create.argtypes = [c.POINTER(Problem), i32, u32, c.POINTER(vp)]
         L.hgf_group_forward.restype = c.c_int
         L.hgf_group_forward.argtypes = [vp, vp]
+        L.hgf_group_forward_phases.restype = c.c_int
+        L.hgf_group_forward_phases.argtypes = [vp, u32, vp]
         L.hgf_group_destroy.restype = None
         L.hgf_group_destroy.argtypes = [vp]
         L.hgf_status_string.restype = c.c_char_p
@@ -199,6 +203,9 @@ class Group:
 
     def forward(self, stream=None) -> None:
         _check("hgf_group_forward", lib().hgf_group_forward(self._handle, _stream(stream)))
+
+    def forward_phases(self, phases: int, stream=None) -> None:
+        _check("hgf_group_forward_phases", lib().hgf_group_forward_phases(self._handle, phases, _stream(stream)))
 
     def close(self) -> None:
         if self._handle:
