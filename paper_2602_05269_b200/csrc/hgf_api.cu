@@ -190,7 +190,9 @@ struct hgf_group {
     void *d_mem;              // one allocation: descriptors, block offsets, workspaces
     DecodeProblem *d_probs;
     PrologueParams *d_pps;
-    int *d_blk_begin;
+    int2 *d_blk_desc;         // per prologue block: (problem, block inside the problem)
+    int4 *d_cta_range;        // per GEMV CTA: (first tile, end tile, first problem, 0)
+    int grid;
 };
 
 extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, uint32_t flags, hgf_group **out) {
@@ -199,7 +201,7 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     *out = nullptr;
     std::vector<PrologueParams> pps((size_t)n);
     std::vector<DecodeProblem> dps((size_t)n);
-    std::vector<int> blk((size_t)n + 1);
+    std::vector<int2> blk;
     std::vector<WsLayout> lay((size_t)n);
     std::vector<int32_t> ranks((size_t)n);
     size_t ws_total = 0;
@@ -219,8 +221,11 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     }
     const size_t off_probs = 0;
     const size_t off_pps = align_up(off_probs + sizeof(DecodeProblem) * (size_t)n, 256);
+    size_t n_blocks = 0;
+    for (int i = 0; i < n; ++i) n_blocks += (size_t)problems[i].M + (size_t)ranks[i] / 16;
     const size_t off_blk = align_up(off_pps + sizeof(PrologueParams) * (size_t)n, 256);
-    const size_t off_ws = align_up(off_blk + sizeof(int) * ((size_t)n + 1), 256);
+    const size_t off_cta = align_up(off_blk + sizeof(int2) * n_blocks, 256);
+    const size_t off_ws = align_up(off_cta + sizeof(int4) * 1024, 256);
     void *mem = nullptr;
     if (cudaMalloc(&mem, off_ws + ws_total) != cudaSuccess) return HGF_ERR_CUDA;
     char *ws = (char *)mem + off_ws;
@@ -231,7 +236,7 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         ws += lay[i].total;
         dps[i].tile_begin = tiles;
         dps[i].cost_begin = cost;
-        blk[i] = blocks;
+        for (int b = 0; b < (int)q.M + ranks[i] / 16; ++b) blk.push_back(make_int2(i, b));
         tiles += (int)row_tiles(q.d_out);
         cost += (long long)row_tiles(q.d_out) * (long long)(padded_k(q.d_in) / 256);
         blocks += (int)q.M + ranks[i] / 16;
@@ -239,7 +244,6 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         const int xb = decode_xq_smem_bytes((int)q.M, (int)q.d_in);
         xq_smem = xb > xq_smem ? xb : xq_smem;
     }
-    blk[n] = blocks;
     hgf_group *g = new (std::nothrow) hgf_group();
     if (!g) { cudaFree(mem); return HGF_ERR_CUDA; }
     g->n = n; g->total_tiles = tiles; g->total_blocks = blocks; g->max_M = max_M; g->xq_smem_bytes = xq_smem;
@@ -247,11 +251,40 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     g->flags = flags; g->d_mem = mem;
     g->d_probs = (DecodeProblem *)((char *)mem + off_probs);
     g->d_pps = (PrologueParams *)((char *)mem + off_pps);
-    g->d_blk_begin = (int *)((char *)mem + off_blk);
+    g->d_blk_desc = (int2 *)((char *)mem + off_blk);
+    g->d_cta_range = (int4 *)((char *)mem + off_cta);
     cudaGetDevice(&g->device);
+    // the GEMV's split of the launch-wide tile sequence into equal contiguous shares, one per CTA
+    g->grid = decode_grid(tiles);
+    std::vector<int4> ranges;
+    if (g->grid > 0 && g->grid <= 1024) {
+        auto tile_of_cost = [&](long long c, int *prob) {
+            int lo = 0, hi = n - 1;
+            while (lo < hi) {  // last problem with cost_begin <= c
+                const int mid = (lo + hi + 1) >> 1;
+                if (dps[mid].cost_begin <= c) lo = mid; else hi = mid - 1;
+            }
+            const long long steps = padded_k(dps[lo].K) / 256, tl = row_tiles(dps[lo].N);
+            long long local = (c - dps[lo].cost_begin + steps - 1) / steps;
+            if (local > tl) local = tl;
+            *prob = lo;
+            return dps[lo].tile_begin + (int)local;
+        };
+        for (int c = 0; c < g->grid; ++c) {
+            int p0 = 0, p1 = 0;
+            const int t0 = tile_of_cost(cost * c / g->grid, &p0);
+            const int t1 = c + 1 == g->grid ? tiles : tile_of_cost(cost * (c + 1) / g->grid, &p1);
+            while (p0 + 1 < n && dps[p0 + 1].tile_begin <= t0) ++p0;  // the problem that holds tile t0
+            ranges.push_back(make_int4(t0, t1, p0, 0));
+        }
+    } else {
+        g->d_cta_range = nullptr;  // the kernel works its share out itself
+    }
     bool ok = cudaMemcpy(g->d_probs, dps.data(), sizeof(DecodeProblem) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
               cudaMemcpy(g->d_pps, pps.data(), sizeof(PrologueParams) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
-              cudaMemcpy(g->d_blk_begin, blk.data(), sizeof(int) * ((size_t)n + 1), cudaMemcpyHostToDevice) == cudaSuccess;
+              cudaMemcpy(g->d_blk_desc, blk.data(), sizeof(int2) * blk.size(), cudaMemcpyHostToDevice) == cudaSuccess &&
+              (ranges.empty() ||
+               cudaMemcpy(g->d_cta_range, ranges.data(), sizeof(int4) * ranges.size(), cudaMemcpyHostToDevice) == cudaSuccess);
     if (!ok) { cudaFree(mem); delete g; return HGF_ERR_CUDA; }
     *out = g;
     return HGF_OK;
@@ -262,7 +295,7 @@ extern "C" hgf_status hgf_group_forward_phases(hgf_group *g, uint32_t phases, vo
     cudaStream_t stream = (cudaStream_t)stream_;
     const bool pdl = !(g->flags & HGF_FLAG_NO_PDL);
     if ((phases & HGF_PHASE_PROLOGUE) &&
-        launch_decode_prologue_group(g->d_pps, g->d_blk_begin, g->n, g->total_blocks, pdl, stream) != cudaSuccess)
+        launch_decode_prologue_group(g->d_pps, g->d_blk_desc, g->total_blocks, pdl, stream) != cudaSuccess)
         return HGF_ERR_CUDA;
     if (!(phases & HGF_PHASE_GEMV)) return HGF_OK;
     DecodeLaunch dl = {};
@@ -272,6 +305,7 @@ extern "C" hgf_status hgf_group_forward_phases(hgf_group *g, uint32_t phases, vo
     dl.total_cost = g->total_cost;
     dl.max_M = g->max_M;
     dl.xq_smem_bytes = g->xq_smem_bytes;
+    dl.cta_range = g->grid == decode_grid(g->total_tiles) ? g->d_cta_range : nullptr;
     return launch_decode_gemv(dl, nullptr, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
 }
 

@@ -101,18 +101,21 @@ struct DecodeLaunch {
     int max_M;                   // largest token count of any problem
     int xq_smem_bytes;           // shared memory for the largest problem's activations
     int ring_slots;              // weight-ring slots per warp (set by the launcher)
+    const int4 *cta_range;       // per CTA: first tile, end tile, first problem (device array), or null
 };
 
 // host-side launchers (each enqueues on `stream` and returns the CUDA error of the launch)
 cudaError_t launch_quant(const PrologueParams &p, cudaStream_t stream);
 cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream_t stream);
-cudaError_t launch_decode_prologue_group(const PrologueParams *d_pps, const int *d_blk_begin, int n, int total_blocks,
+cudaError_t launch_decode_prologue_group(const PrologueParams *d_pps, const int2 *d_blk_desc, int total_blocks,
                                          bool pdl, cudaStream_t stream);
 cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream);
 cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream);
 // Shared memory the decode kernel needs for one problem's activations, and the largest it accepts.
 int decode_xq_smem_bytes(int M, int K);
 int decode_xq_smem_limit();
+// Grid of the decode GEMV for a launch with that many row tiles (0 if the device cannot be queried).
+int decode_grid(int total_tiles);
 
 struct GemmParams {
     const int8_t *xq;        // [M][K]

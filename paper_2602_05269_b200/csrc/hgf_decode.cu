@@ -157,10 +157,14 @@ __device__ int tile_of_cost(const DecodeLaunch &L, const DecodeProblem &single, 
 }
 
 // First segment (first = true) or the one after `s`, inside the CTA's tile range [t0, t1).
-__device__ bool next_segment(const DecodeLaunch &L, const DecodeProblem &single, int t0, int t1, bool first, Seg &s) {
+// p_first >= 0 names the problem that holds tile t0 (saves the search).
+__device__ bool next_segment(const DecodeLaunch &L, const DecodeProblem &single, int t0, int t1, bool first, Seg &s,
+                             int p_first = -1) {
     if (t0 >= t1) return false;
     int p;
-    if (first) {
+    if (first && p_first >= 0) {
+        p = p_first;
+    } else if (first) {
         int lo = 0, hi = L.n_probs - 1;
         while (lo < hi) {  // last problem with tile_begin <= t0
             const int mid = (lo + hi + 1) >> 1;
@@ -238,17 +242,23 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
     __syncthreads();
 
     // this CTA's share of the launch-wide tile sequence
-    const long long c0 = L.total_cost * (long long)blockIdx.x / (long long)gridDim.x;
-    const long long c1 = L.total_cost * (long long)(blockIdx.x + 1) / (long long)gridDim.x;
-    const int t0 = tile_of_cost(L, single, c0);
-    const int t1 = (blockIdx.x + 1 == gridDim.x) ? L.total_tiles : tile_of_cost(L, single, c1);
+    int t0, t1, p_first = -1;
+    if (L.cta_range) {  // precomputed on the host for a group
+        const int4 cr = L.cta_range[blockIdx.x];
+        t0 = cr.x; t1 = cr.y; p_first = cr.z;
+    } else {
+        const long long c0 = L.total_cost * (long long)blockIdx.x / (long long)gridDim.x;
+        const long long c1 = L.total_cost * (long long)(blockIdx.x + 1) / (long long)gridDim.x;
+        t0 = tile_of_cost(L, single, c0);
+        t1 = (blockIdx.x + 1 == gridDim.x) ? L.total_tiles : tile_of_cost(L, single, c1);
+    }
 
     // ---- producer ------------------------------------------------------------------------------
     // A slot receives up to kSlotTiles consecutive tiles of one item; items are cut into slots from
     // their first tile on, so the consumer knows each slot's size from its own position.
     Producer pr;
     pr.left = 0; pr.round = -1; pr.rounds = 0; pr.src = nullptr; pr.bt_src = nullptr; pr.bt_bytes = 0;
-    pr.done = !next_segment(L, single, t0, t1, true, pr.seg);
+    pr.done = !next_segment(L, single, t0, t1, true, pr.seg, p_first);
     if (!pr.done) pr.rounds = seg_rounds(pr.seg);
 
     auto next_item = [&]() {  // slow path of the producer: find this warp's next item with work
@@ -301,7 +311,7 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
     bool ok = true;         // false once a wait gave up (this warp stops computing but keeps the barriers)
     Seg seg;
     int seg_idx = 0;
-    for (bool more = next_segment(L, single, t0, t1, true, seg); more;
+    for (bool more = next_segment(L, single, t0, t1, true, seg, p_first); more;
          more = next_segment(L, single, t0, t1, false, seg), ++seg_idx) {
         const DecodeProblem &Pg = problem_of(L, single, seg.p);
         const int K = Pg.K, M = Pg.M, N = Pg.N, r = Pg.r;
@@ -551,16 +561,21 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
     }
 }
 
-cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *single, bool pdl, cudaStream_t stream) {
-    static int sm_count = 0;
-    static bool attr_set = false;
-    if (!sm_count) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
+static int g_sm_count = 0;
+int decode_grid(int total_tiles) {
+    if (!g_sm_count) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        g_sm_count = n;
     }
+    return total_tiles < g_sm_count ? total_tiles : g_sm_count;
+}
+
+cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *single, bool pdl, cudaStream_t stream) {
+    static bool attr_set = false;
+    const int grid = decode_grid(L_in.total_tiles);
+    if (grid <= 0) return cudaErrorInvalidDevice;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(decode_gemv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
         if (e != cudaSuccess) return e;
@@ -577,7 +592,6 @@ cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *si
     int slots = (kSmemLimit - kOffXq - xq_bytes) / (kDecWarps * kSlotBytes);
     slots = slots > kMaxSlots ? kMaxSlots : slots;
     L.ring_slots = slots;
-    const int grid = L.total_tiles < sm_count ? L.total_tiles : sm_count;
     DecodeProblem dummy = {};
     const DecodeProblem &sp = single ? *single : dummy;
 

@@ -214,22 +214,16 @@ __global__ void __launch_bounds__(kThreads) decode_prologue_kernel(const Prologu
         lora_down_block(p, blockIdx.x - p.M);
 }
 
-// The same for a group of problems: blk_begin[i] = first block of problem i (n + 1 entries).
-__global__ void __launch_bounds__(kThreads) decode_prologue_group_kernel(const PrologueParams *pps, const int *blk_begin,
-                                                                         int n) {
+// The same for a group of problems: blk_desc[b] = (problem, block index inside the problem).
+__global__ void __launch_bounds__(kThreads) decode_prologue_group_kernel(const PrologueParams *pps, const int2 *blk_desc) {
     pdl_launch_dependents();
+    const int2 d = blk_desc[blockIdx.x];  // written at set-up, not by the preceding work
     pdl_wait();
-    int lo = 0, hi = n - 1;
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (blk_begin[mid] <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
-    }
-    const PrologueParams p = pps[lo];
-    const int b = blockIdx.x - blk_begin[lo];
-    if (b < p.M)
-        quant_row(p, b);
+    const PrologueParams p = pps[d.x];
+    if (d.y < p.M)
+        quant_row(p, d.y);
     else
-        lora_down_block(p, b - p.M);
+        lora_down_block(p, d.y - p.M);
 }
 
 // ---- GEMM-path LoRA down-projection on tensor cores (legacy warp MMA, tf32 inputs) -----------
@@ -349,11 +343,11 @@ cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t launch_decode_prologue_group(const PrologueParams *d_pps, const int *d_blk_begin, int n, int total_blocks,
+cudaError_t launch_decode_prologue_group(const PrologueParams *d_pps, const int2 *d_blk_desc, int total_blocks,
                                          bool pdl, cudaStream_t stream) {
     cudaLaunchAttribute attr[1];
     cudaLaunchConfig_t cfg = prologue_cfg(total_blocks, pdl, stream, attr);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_prologue_group_kernel, d_pps, d_blk_begin, n);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_prologue_group_kernel, d_pps, d_blk_desc);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }
