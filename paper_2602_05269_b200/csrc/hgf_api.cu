@@ -190,7 +190,9 @@ struct hgf_group {
     void *d_mem;              // one allocation: descriptors, block offsets, workspaces
     DecodeProblem *d_probs;
     PrologueParams *d_pps;
-    int2 *d_blk_desc;         // per prologue block: (problem, block inside the problem)
+    QuantItem *d_quant_items; // prologue: one per (problem, token)
+    LoraItem *d_lora_items;   // prologue: one per (problem, 16 columns of H, K slice)
+    int n_quant, n_lora;
     int4 *d_cta_range;        // per GEMV CTA: (first tile, end tile, first problem, 0)
     int grid;
 };
@@ -201,7 +203,8 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     *out = nullptr;
     std::vector<PrologueParams> pps((size_t)n);
     std::vector<DecodeProblem> dps((size_t)n);
-    std::vector<int2> blk;
+    std::vector<QuantItem> qitems;
+    std::vector<LoraItem> litems;
     std::vector<WsLayout> lay((size_t)n);
     std::vector<int32_t> ranks((size_t)n);
     size_t ws_total = 0;
@@ -221,14 +224,24 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     }
     const size_t off_probs = 0;
     const size_t off_pps = align_up(off_probs + sizeof(DecodeProblem) * (size_t)n, 256);
-    size_t n_blocks = 0;
-    for (int i = 0; i < n; ++i) n_blocks += (size_t)problems[i].M + (size_t)ranks[i] / 16;
-    const size_t off_blk = align_up(off_pps + sizeof(PrologueParams) * (size_t)n, 256);
-    const size_t off_cta = align_up(off_blk + sizeof(int2) * n_blocks, 256);
-    const size_t off_ws = align_up(off_cta + sizeof(int4) * 1024, 256);
+    // prologue items, and the scratch of the LoRA items: per problem (r / 16) x slices x 8 x 32 floats
+    int all_M = 0;
+    for (int i = 0; i < n; ++i) all_M = problems[i].M > all_M ? (int)problems[i].M : all_M;
+    const int slice_k = prologue_slice_k(all_M);
+    size_t n_quant = 0, n_lora = 0;
+    for (int i = 0; i < n; ++i) {
+        n_quant += (size_t)problems[i].M;
+        n_lora += ((size_t)ranks[i] / 16) * (size_t)((problems[i].d_in + slice_k - 1) / slice_k);
+    }
+    const size_t off_qit = align_up(off_pps + sizeof(PrologueParams) * (size_t)n, 256);
+    const size_t off_lit = align_up(off_qit + sizeof(QuantItem) * n_quant, 256);
+    const size_t off_cta = align_up(off_lit + sizeof(LoraItem) * n_lora, 256);
+    const size_t off_hpart = align_up(off_cta + sizeof(int4) * 1024, 256);
+    const size_t off_ws = align_up(off_hpart + n_lora * 8 * 32 * sizeof(float), 256);
     void *mem = nullptr;
     if (cudaMalloc(&mem, off_ws + ws_total) != cudaSuccess) return HGF_ERR_CUDA;
     char *ws = (char *)mem + off_ws;
+    float *hpart = (float *)((char *)mem + off_hpart);
     for (int i = 0; i < n; ++i) {
         const hgf_problem &q = problems[i];
         fill_params(q.x, q.M, q.packed, q.gamma, q.d_in, q.d_out, q.At, q.Bt, ranks[i], q.gate, q.y, ws, lay[i], false,
@@ -236,7 +249,28 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         ws += lay[i].total;
         dps[i].tile_begin = tiles;
         dps[i].cost_begin = cost;
-        for (int b = 0; b < (int)q.M + ranks[i] / 16; ++b) blk.push_back(make_int2(i, b));
+        {
+            const int slices = (int)((q.d_in + slice_k - 1) / slice_k), jts = ranks[i] / 16;
+            dps[i].hpart = jts ? hpart : nullptr;
+            dps[i].nslices = jts ? slices : 0;
+            for (int m = 0; m < (int)q.M; ++m) {
+                QuantItem qi = {pps[i].x + (size_t)m * q.d_in, pps[i].xq + (size_t)m * q.d_in, pps[i].gamma_x + m,
+                                pps[i].row_sum + m, (int)q.d_in, 0};
+                qitems.push_back(qi);
+            }
+            for (int sl = 0; sl < slices; ++sl)      // slice-major: neighbouring warps share x
+                for (int jt = 0; jt < jts; ++jt) {
+                    const int64_t k0 = (int64_t)sl * slice_k, kvalid = q.d_in - k0 < slice_k ? q.d_in - k0 : slice_k;
+                    LoraItem it;
+                    it.At = (const __half *)q.At + (size_t)16 * jt * q.d_in + k0;
+                    it.x = (const __nv_bfloat16 *)q.x + k0;
+                    it.hpart = hpart + ((size_t)jt * slices + sl) * 8 * 32;
+                    it.K = (int)q.d_in;
+                    it.kvalid_M = (int)(kvalid << 8) | (int)q.M;
+                    litems.push_back(it);
+                }
+            hpart += (size_t)jts * slices * 8 * 32;
+        }
         tiles += (int)row_tiles(q.d_out);
         cost += (long long)row_tiles(q.d_out) * (long long)(padded_k(q.d_in) / 256);
         blocks += (int)q.M + ranks[i] / 16;
@@ -251,7 +285,10 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     g->flags = flags; g->d_mem = mem;
     g->d_probs = (DecodeProblem *)((char *)mem + off_probs);
     g->d_pps = (PrologueParams *)((char *)mem + off_pps);
-    g->d_blk_desc = (int2 *)((char *)mem + off_blk);
+    g->d_quant_items = (QuantItem *)((char *)mem + off_qit);
+    g->d_lora_items = (LoraItem *)((char *)mem + off_lit);
+    g->n_quant = (int)qitems.size();
+    g->n_lora = (int)litems.size();
     g->d_cta_range = (int4 *)((char *)mem + off_cta);
     cudaGetDevice(&g->device);
     // the GEMV's split of the launch-wide tile sequence into equal contiguous shares, one per CTA
@@ -282,7 +319,9 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     }
     bool ok = cudaMemcpy(g->d_probs, dps.data(), sizeof(DecodeProblem) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
               cudaMemcpy(g->d_pps, pps.data(), sizeof(PrologueParams) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
-              cudaMemcpy(g->d_blk_desc, blk.data(), sizeof(int2) * blk.size(), cudaMemcpyHostToDevice) == cudaSuccess &&
+              cudaMemcpy(g->d_quant_items, qitems.data(), sizeof(QuantItem) * qitems.size(), cudaMemcpyHostToDevice) == cudaSuccess &&
+              (litems.empty() || cudaMemcpy(g->d_lora_items, litems.data(), sizeof(LoraItem) * litems.size(),
+                                            cudaMemcpyHostToDevice) == cudaSuccess) &&
               (ranges.empty() ||
                cudaMemcpy(g->d_cta_range, ranges.data(), sizeof(int4) * ranges.size(), cudaMemcpyHostToDevice) == cudaSuccess);
     if (!ok) { cudaFree(mem); delete g; return HGF_ERR_CUDA; }
@@ -295,7 +334,8 @@ extern "C" hgf_status hgf_group_forward_phases(hgf_group *g, uint32_t phases, vo
     cudaStream_t stream = (cudaStream_t)stream_;
     const bool pdl = !(g->flags & HGF_FLAG_NO_PDL);
     if ((phases & HGF_PHASE_PROLOGUE) &&
-        launch_decode_prologue_group(g->d_pps, g->d_blk_desc, g->total_blocks, pdl, stream) != cudaSuccess)
+        launch_decode_prologue_group(g->d_quant_items, g->n_quant, g->d_lora_items, g->n_lora, g->max_M, pdl,
+                                     stream) != cudaSuccess)
         return HGF_ERR_CUDA;
     if (!(phases & HGF_PHASE_GEMV)) return HGF_OK;
     DecodeLaunch dl = {};

@@ -82,6 +82,8 @@ struct DecodeProblem {
     const int32_t *row_sum;  // [M]
     const __half *h_hi;      // [M][r]
     const __half *h_lo;      // [M][r]
+    const float *hpart;      // group launches: partial sums of x A per (16-column tile, K slice), else null
+    int nslices;             // K slices per tile in hpart
     const __half *Bt;        // [N][r]
     const float *gate;       // [N]
     void *y;                 // [M][N] fp32 or bf16
@@ -107,8 +109,28 @@ struct DecodeLaunch {
 // host-side launchers (each enqueues on `stream` and returns the CUDA error of the launch)
 cudaError_t launch_quant(const PrologueParams &p, cudaStream_t stream);
 cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream_t stream);
-cudaError_t launch_decode_prologue_group(const PrologueParams *d_pps, const int2 *d_blk_desc, int total_blocks,
-                                         bool pdl, cudaStream_t stream);
+// Group prologue.  A quantisation item is one token row.  A LoRA item is 16 columns of H (rows
+// 16 jt .. 16 jt + 15 of A^T) over one K slice of a problem; its 16 x 16 partial sums of x A go to
+// `hpart` as [8 accumulator registers][32 lanes] floats, and the GEMV adds the slices of a tile in
+// slice order.  Slices are 512 columns when every problem of the group has M <= 8, else 256.
+struct LoraItem {
+    const __half *At;          // row 16 jt of A^T, first column of the slice
+    const __nv_bfloat16 *x;    // token 0, first column of the slice
+    float *hpart;              // this item's 8 x 32 floats
+    int K;                     // row pitch of A^T and x
+    int kvalid_M;              // (columns of the slice inside K) << 8 | M
+};
+struct QuantItem {
+    const __nv_bfloat16 *x;    // the token's row
+    int8_t *xq;                // its quantised row
+    float *gamma_x;            // its scale
+    int32_t *row_sum;          // its sum of quantised values
+    int K, pad;
+};
+static inline int prologue_slice_k(int max_M) { return max_M <= 8 ? 512 : 256; }
+cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_quant,
+                                         const LoraItem *d_lora_items, int n_lora, int max_M, bool pdl,
+                                         cudaStream_t stream);
 cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream);
 cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream);
 // Shared memory the decode kernel needs for one problem's activations, and the largest it accepts.

@@ -349,12 +349,32 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
                 sm.row_sum[tid] = tid < M ? Pg.row_sum[tid] : 0;
             }
             if (tid == 32) { sm.y = Pg.y; sm.dbg_y_int = Pg.dbg_y_int; sm.gate = Pg.gate; sm.flags = Pg.flags; }
-            const int words = r >> 1;  // 32-bit words per row of H
-            const uint32_t *hi_g = reinterpret_cast<const uint32_t *>(Pg.h_hi), *lo_g = reinterpret_cast<const uint32_t *>(Pg.h_lo);
-            for (int u = tid; u < M * words; u += kDecThreads) {
-                const int m = u / words, w = u - m * words;
-                reinterpret_cast<uint32_t *>(&sm.h_hi[m][0])[w] = hi_g[u];
-                reinterpret_cast<uint32_t *>(&sm.h_lo[m][0])[w] = lo_g[u];
+            if (Pg.nslices > 0) {
+                // group launch: H = act(sum over K slices of the parked partial sums of x A), slices in
+                // order.  The partial sums sit in the tf32 MMA's accumulator layout: column j = 16 jt + jl
+                // and token m are register 4 (m / 8) + 2 (jl / 8) + (m % 2) of lane 4 (jl % 8) + (m % 8) / 2.
+                const float *hp = Pg.hpart;
+                const int ns = Pg.nslices;
+                const bool no_silu = (Pg.flags & HGF_FLAG_NO_SILU) != 0;
+                for (int u = tid; u < M * r; u += kDecThreads) {
+                    const int m = u / r, j = u - m * r, jt = j >> 4, jl = j & 15;
+                    const int idx = 4 * (m >> 3) + 2 * (jl >> 3) + (m & 1), ln = 4 * (jl & 7) + ((m & 7) >> 1);
+                    const float *src = hp + ((size_t)jt * ns * 8 + idx) * 32 + ln;
+                    float z = 0.0f;
+                    for (int sl = 0; sl < ns; ++sl) z += __ldcg(src + (size_t)sl * 256);
+                    const float h = no_silu ? z : silu_f(z);
+                    const __half hi = __float2half_rn(h);
+                    sm.h_hi[m][j] = hi;
+                    sm.h_lo[m][j] = __float2half_rn(h - __half2float(hi));
+                }
+            } else {
+                const int words = r >> 1;  // 32-bit words per row of H
+                const uint32_t *hi_g = reinterpret_cast<const uint32_t *>(Pg.h_hi), *lo_g = reinterpret_cast<const uint32_t *>(Pg.h_lo);
+                for (int u = tid; u < M * words; u += kDecThreads) {
+                    const int m = u / words, w = u - m * words;
+                    reinterpret_cast<uint32_t *>(&sm.h_hi[m][0])[w] = hi_g[u];
+                    reinterpret_cast<uint32_t *>(&sm.h_lo[m][0])[w] = lo_g[u];
+                }
             }
         }
         __syncthreads();

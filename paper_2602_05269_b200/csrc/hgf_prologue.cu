@@ -23,13 +23,42 @@ __device__ __forceinline__ float warp_sum_f(float v) {
     return v;
 }
 
-// Round-to-nearest-even of the exact quotient 127 x / gamma: 127 x is exact in fp32 for a bf16 x,
-// the IEEE division is correctly rounded and k + 1/2 is representable, so rintf of the rounded
-// quotient equals the rounding of the exact one.
-__device__ __forceinline__ int quant1(float x, float gamma) {
+// Round-to-nearest-even of the exact quotient 127 x / gamma for a bf16 x.
+//
+// Reference form: 127 x is exact in fp32, the IEEE division is correctly rounded and k + 1/2 is
+// representable, so rintf of the rounded quotient equals the rounding of the exact one.
+__device__ __forceinline__ int quant1_div(float x, float gamma) {
     float q = rintf(__fdiv_rn(127.0f * x, gamma));
     q = fminf(fmaxf(q, -127.0f), 127.0f);
     return __float2int_rn(q);
+}
+// Division-free form, for gamma = max |x| over bf16 values (so gamma is a bf16 value itself, i.e. not
+// the 1e-5 floor).  A candidate q = rint(x * (127 / gamma)) is within one of the answer.  The
+// residual 127 x - q gamma is exact in one fma (127 x and q gamma each have at most 15 significant
+// bits), and the exact quotient is q + residual / gamma: the candidate stands iff
+// 2 |residual| < gamma, or = gamma with q even (a tie goes to the even neighbour); otherwise it
+// moves one step towards the residual's sign.
+struct QuantScale {
+    float gamma, inv127;  // inv127 = 127 / gamma
+    bool fast;            // gamma is a bf16 value
+};
+__device__ __forceinline__ QuantScale make_quant_scale(float gamma) {
+    QuantScale s;
+    s.gamma = gamma;
+    s.inv127 = __fdiv_rn(127.0f, gamma);
+    s.fast = (__float_as_uint(gamma) & 0xffffu) == 0u;
+    return s;
+}
+__device__ __forceinline__ int quant1_fast(float x, const QuantScale &s) {
+    float q = rintf(x * s.inv127);
+    const float res = fmaf(-q, s.gamma, 127.0f * x);
+    const float two = 2.0f * fabsf(res);
+    const bool odd = (__float2int_rn(q) & 1) != 0;
+    if (two > s.gamma || (two == s.gamma && odd)) q += copysignf(1.0f, res);
+    return __float2int_rn(q);
+}
+__device__ __forceinline__ int quant1(float x, const QuantScale &s) {
+    return s.fast ? quant1_fast(x, s) : quant1_div(x, s.gamma);
 }
 
 // One block quantises one token row.
@@ -57,6 +86,7 @@ __device__ void quant_row(const PrologueParams &p, int m) {
 #pragma unroll
     for (int w = 1; w < kWarps; ++w) g = fmaxf(g, s_red_f[w]);
     g = fmaxf(g, 1e-5f);
+    const QuantScale qs = make_quant_scale(g);
 
     int sum = 0;
     uint2 *qv = reinterpret_cast<uint2 *>(p.xq + (size_t)m * K);
@@ -67,8 +97,8 @@ __device__ void quant_row(const PrologueParams &p, int m) {
         uint32_t o[2] = {0u, 0u};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            int q0 = quant1(bf16lo_to_float(w[j]), g);
-            int q1 = quant1(bf16hi_to_float(w[j]), g);
+            int q0 = quant1(bf16lo_to_float(w[j]), qs);
+            int q1 = quant1(bf16hi_to_float(w[j]), qs);
             sum += q0 + q1;
             o[j >> 1] |= (uint32_t)(q0 & 0xff) << (16 * (j & 1));
             o[j >> 1] |= (uint32_t)(q1 & 0xff) << (16 * (j & 1) + 8);
@@ -214,16 +244,172 @@ __global__ void __launch_bounds__(kThreads) decode_prologue_kernel(const Prologu
         lora_down_block(p, blockIdx.x - p.M);
 }
 
-// The same for a group of problems: blk_desc[b] = (problem, block index inside the problem).
-__global__ void __launch_bounds__(kThreads) decode_prologue_group_kernel(const PrologueParams *pps, const int2 *blk_desc) {
+// ---- group prologue: persistent CTAs, one warp per work item ------------------------------------
+// The rows of A^T are the bulk of what a decode prologue reads, and a group has thousands of small
+// pieces of them, each behind a chain of dependent memory latencies.  Here the grid stays resident
+// (one CTA of 8 warps per SM) and every warp walks the item tables with a grid-wide stride.  For a
+// LoRA item the warp requests everything the item reads at once - per lane up to 32 + 16 asynchronous
+// 16-byte copies into its own part of shared memory, which serves as a register extension: a lane
+// reads back only what it requested itself - while the next item's descriptor is already on its
+// way, then runs the tf32 MMAs (rows of A^T are the 16-row operand, tokens the 8-column operand) and
+// parks the 16 x 16 partial sums; the GEMV adds a tile's K slices in slice order.
+constexpr int kPgWarps = 8;
+constexpr int kPgThreads = kPgWarps * 32;
+
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros and reads nothing.
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ uint4 pg_lds_u4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
+// One warp quantises one token row (Algorithm 1, steps 1-2).  The row is brought into the warp's
+// shared-memory buffer with asynchronous copies, all requested at once, so both passes (maximum,
+// then rounding) read it from there; a row longer than the buffer goes through in pieces and is
+// fetched a second time for the second pass.
+__device__ void warp_quant_row(const QuantItem &q, uint32_t buf_u32, const uint8_t *buf, int buf_bytes, int lane) {
+    const int K = q.K, piece = buf_bytes / 2;  // elements per piece (a multiple of 256)
+    const int npieces = (K + piece - 1) / piece;
+    auto fetch = [&](int pc) {  // units of 8 elements; lane-strided, so a lane reads back its own units
+        const int n = (K - pc * piece < piece ? K - pc * piece : piece) / 8;
+        for (int i = lane; i < n; i += 32) cp_async_16(buf_u32 + 16 * i, q.x + (size_t)pc * piece + 8 * i, 16u);
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+        asm volatile("cp.async.wait_all;\n" ::: "memory");
+        return n;
+    };
+    float amax = 0.0f;
+    int n = 0;
+    for (int pc = 0; pc < npieces; ++pc) {
+        n = fetch(pc);
+        for (int i = lane; i < n; i += 32) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(buf + 16 * i);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                amax = fmaxf(amax, fabsf(bf16lo_to_float(w[j])));
+                amax = fmaxf(amax, fabsf(bf16hi_to_float(w[j])));
+            }
+        }
+    }
+    const float g = fmaxf(warp_max(amax), 1e-5f);
+    const QuantScale qs = make_quant_scale(g);
+    int sum = 0;
+    for (int pc = 0; pc < npieces; ++pc) {
+        if (npieces > 1) n = fetch(pc);
+        uint2 *qv = reinterpret_cast<uint2 *>(q.xq + (size_t)pc * piece);
+        for (int i = lane; i < n; i += 32) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(buf + 16 * i);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            uint32_t o[2] = {0u, 0u};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int q0 = quant1(bf16lo_to_float(w[j]), qs), q1 = quant1(bf16hi_to_float(w[j]), qs);
+                sum += q0 + q1;
+                o[j >> 1] |= (uint32_t)(q0 & 0xff) << (16 * (j & 1));
+                o[j >> 1] |= (uint32_t)(q1 & 0xff) << (16 * (j & 1) + 8);
+            }
+            qv[i] = make_uint2(o[0], o[1]);
+        }
+    }
+    sum = warp_sum_i(sum);
+    if (lane == 0) {
+        *q.row_sum = sum;
+        *q.gamma_x = g;
+    }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(kPgThreads, 1)
+decode_prologue_group_kernel(const QuantItem *quant_items, int n_quant, const LoraItem *lora, int n_lora) {
+    constexpr int CH = 16 / NT;                       // 32-column chunks per item
+    constexpr int kWarpBytes = CH * (1024 + 512 * NT);  // per chunk: two rows of A^T and NT rows of x, 16 bytes per lane
+    extern __shared__ __align__(128) uint8_t pg_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
+    const int gw = blockIdx.x * kPgWarps + warp, nw = gridDim.x * kPgWarps;
+    const uint32_t buf = (uint32_t)__cvta_generic_to_shared(pg_smem) + warp * kWarpBytes + 16 * lane;
+
     pdl_launch_dependents();
-    const int2 d = blk_desc[blockIdx.x];  // written at set-up, not by the preceding work
-    pdl_wait();
-    const PrologueParams p = pps[d.x];
-    if (d.y < p.M)
-        quant_row(p, d.y);
-    else
-        lora_down_block(p, d.y - p.M);
+    // the item tables are written at set-up, not by the preceding work
+    uint4 d0 = make_uint4(0u, 0u, 0u, 0u), d1 = d0;
+    if (gw < n_lora) {
+        d0 = reinterpret_cast<const uint4 *>(lora + gw)[0];
+        d1 = reinterpret_cast<const uint4 *>(lora + gw)[1];
+    }
+    pdl_wait();  // x, and the scratch this kernel overwrites, belong to earlier work
+
+    // LoRA items are dealt from the first warp up, quantisation items from the last warp down, so the
+    // warps with one LoRA item fewer take the rows
+    for (int i = nw - 1 - gw; i < n_quant; i += nw) {
+        const QuantItem q = quant_items[i];
+        warp_quant_row(q, buf - 16 * lane, pg_smem + warp * kWarpBytes, kWarpBytes, lane);
+    }
+
+    for (int i = gw; i < n_lora; i += nw) {
+        const LoraItem it = {reinterpret_cast<const __half *>(((uint64_t)d0.y << 32) | d0.x),
+                             reinterpret_cast<const __nv_bfloat16 *>(((uint64_t)d0.w << 32) | d0.z),
+                             reinterpret_cast<float *>(((uint64_t)d1.y << 32) | d1.x), (int)d1.z, (int)d1.w};
+        const int K = it.K, M = it.kvalid_M & 0xff, nchunks = (it.kvalid_M >> 8) / 32;
+        // everything this item reads, requested at once
+        const __half *rowA = it.At + (size_t)g * K + 8 * t;
+        const __half *rowB = rowA + (size_t)8 * K;
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const bool in = c < nchunks;
+            cp_async_16(buf + c * 1024, in ? rowA + 32 * c : it.At, in ? 16u : 0u);
+            cp_async_16(buf + c * 1024 + 512, in ? rowB + 32 * c : it.At, in ? 16u : 0u);
+        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const bool tok = g + 8 * nt < M;
+            const __nv_bfloat16 *xr = it.x + (size_t)(tok ? g + 8 * nt : 0) * K + 8 * t;
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const bool in = tok && c < nchunks;
+                cp_async_16(buf + CH * 1024 + (c * NT + nt) * 512, in ? xr + 32 * c : it.x, in ? 16u : 0u);
+            }
+        }
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+        if (i + nw < n_lora) {  // the next item's descriptor travels meanwhile
+            d0 = reinterpret_cast<const uint4 *>(lora + i + nw)[0];
+            d1 = reinterpret_cast<const uint4 *>(lora + i + nw)[1];
+        }
+        asm volatile("cp.async.wait_all;\n" ::: "memory");
+
+        float acc[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[nt][c] = 0.0f;
+#pragma unroll 4
+        for (int c = 0; c < CH; ++c) {
+            const uint4 av = pg_lds_u4(buf + c * 1024), bv = pg_lds_u4(buf + c * 1024 + 512);
+            uint4 xv[NT];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) xv[nt] = pg_lds_u4(buf + CH * 1024 + (c * NT + nt) * 512);
+            const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
+            const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                // elements 2 e and 2 e + 1 of this lane's eight take the k slots t and t + 4 of the MMA
+                const float2 fa = __half22float2(*reinterpret_cast<const __half2 *>(&aw[e]));
+                const float2 fb = __half22float2(*reinterpret_cast<const __half2 *>(&bw[e]));
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint32_t xw = (&xv[nt].x)[e];
+                    mma_tf32(acc[nt], __float_as_uint(fa.x), __float_as_uint(fb.x), __float_as_uint(fa.y),
+                             __float_as_uint(fb.y), xw << 16, xw & 0xffff0000u);
+                }
+            }
+        }
+        // park the partial sums: [register 0..7][lane]
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) __stcg(it.hpart + (nt * 4 + c) * 32 + lane, acc[nt][c]);
+    }
 }
 
 // ---- GEMM-path LoRA down-projection on tensor cores (legacy warp MMA, tf32 inputs) -----------
@@ -343,11 +529,40 @@ cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t launch_decode_prologue_group(const PrologueParams *d_pps, const int2 *d_blk_desc, int total_blocks,
-                                         bool pdl, cudaStream_t stream) {
+cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_quant, const LoraItem *d_lora_items, int n_lora, int max_M, bool pdl,
+                                         cudaStream_t stream) {
+    static int sm_count = 0;
+    static bool attr_set = false;
+    if (!sm_count) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+    }
+    const int smem1 = kPgWarps * 16 * (1024 + 512), smem2 = kPgWarps * 8 * (1024 + 1024);
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(decode_prologue_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(decode_prologue_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int most = n_lora > n_quant ? n_lora : n_quant;
+    int blocks = (most + kPgWarps - 1) / kPgWarps;
+    blocks = blocks < sm_count ? blocks : sm_count;
+    if (blocks < 1) blocks = 1;
     cudaLaunchAttribute attr[1];
-    cudaLaunchConfig_t cfg = prologue_cfg(total_blocks, pdl, stream, attr);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_prologue_group_kernel, d_pps, d_blk_desc);
+    cudaLaunchConfig_t cfg = prologue_cfg(blocks, pdl, stream, attr);
+    cfg.blockDim = dim3(kPgThreads);
+    cudaError_t e;
+    if (max_M <= 8) {
+        cfg.dynamicSmemBytes = smem1;
+        e = cudaLaunchKernelEx(&cfg, decode_prologue_group_kernel<1>, d_quant_items, n_quant, d_lora_items, n_lora);
+    } else {
+        cfg.dynamicSmemBytes = smem2;
+        e = cudaLaunchKernelEx(&cfg, decode_prologue_group_kernel<2>, d_quant_items, n_quant, d_lora_items, n_lora);
+    }
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }

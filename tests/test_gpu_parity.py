@@ -260,7 +260,8 @@ def test_group_of_independent_layers_matches_oracle_and_single_calls(hgf, M):
         assert err <= TOL_DECODE, (s, err)
         y_single = hgf.linear_forward(q["x"], q["packed"], q["gamma"], s.d_in, s.d_out, q.get("At"), q.get("Bt"),
                                       q.get("gate"))
-        assert torch.equal(y_single, q["y"]), s     # same kernels, same arithmetic order
+        # same GEMV kernel; the two prologues add the K slices of x A in different orders (fp32)
+        assert (y_single - q["y"]).abs().max().item() <= 2e-6 * np.abs(ref["y"]).max(), s
     group.close()
 
 
