@@ -63,7 +63,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
         except OSError:
@@ -310,7 +310,9 @@ def run_ours(args):
 # DRAM traffic of the decode GEMV launch from the committed ncu capture (profiles/): bytes moved
 # per algorithmic byte on the captured case.  It is only reported while the kernel source is the one
 # that was profiled.
-DECODE_TRAFFIC = {"source_sha1": None, "dram_bytes_per_algorithmic_byte": None, "profile": None}
+DECODE_TRAFFIC = {"source_sha1": "e0452d22d4e638f2fbf061fdc86f1c676d99c7e6",
+                  "dram_bytes_per_algorithmic_byte": (517.408768e6 + 6.296832e6) / 518805504.0,
+                  "profile": "profiles/decode_gemv_config1_m1.md"}
 
 
 def decode_traffic(gemv_bytes):
@@ -466,20 +468,47 @@ def run_profile_case(spec: str, reps: int):
     print(json.dumps({"profile_case": spec, "reps": reps, "launches": hgf.launch_count()}))
 
 
+def run_profile_group(spec: str, reps: int):
+    """A few grouped decode steps of one configuration, for use under a profiler (never a benchmark value)."""
+    import torch
+
+    from paper_2602_05269_b200 import hgf, inputs as syn
+
+    cfg, M = (int(v) for v in spec.split(","))
+    torch.cuda.set_device(0)
+    stream = torch.cuda.Stream()
+    shapes = syn.CONFIGS[cfg]["layers"]
+    block = sum(layer_bytes(s.d_in, s.d_out, s.r, M) for s in shapes)
+    copies = max(32 if cfg == 4 else 1, int(np.ceil(4.4 * L2_BYTES / block)))
+    w = Workload(hgf, torch, shapes, M, copies)
+    w.make_group()
+    with torch.cuda.stream(stream):
+        for _ in range(reps + 5):
+            w.group.forward(stream)
+        stream.synchronize()
+    hgf.check_status(stream)
+    print(json.dumps({"profile_group": spec, "layers": len(w.layers), "steps": reps + 5, "launches": hgf.launch_count()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline measurement only")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
     ap.add_argument("--profile", default=None,
                     help="run plain launches of one case for a profiler, e.g. prefill:2048x5632x8192x32:bf16")
+    ap.add_argument("--profile-group", default=None,
+                    help="run a few hgf_group_forward steps of one decode workload for a profiler: CONFIG,M (e.g. 1,1)")
     ap.add_argument("--reps", type=int, default=3)
     args = ap.parse_args()
     if args.profile:
         run_profile_case(args.profile, args.reps)
+        return
+    if args.profile_group:
+        run_profile_group(args.profile_group, args.reps)
         return
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
