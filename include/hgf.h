@@ -38,7 +38,8 @@ typedef enum {
     HGF_ERR_MISALIGNED = 3,        /* a device pointer is not 16-byte aligned */
     HGF_ERR_WORKSPACE = 4,         /* workspace missing or smaller than hgf_workspace_bytes() */
     HGF_ERR_CUDA = 5,              /* a CUDA runtime/driver call failed (launch error, no device) */
-    HGF_ERR_TIMEOUT = 6            /* a bounded device-side wait gave up (reported by hgf_check_status) */
+    HGF_ERR_TIMEOUT = 6,           /* a bounded device-side wait gave up (reported by hgf_check_status) */
+    HGF_ERR_TOO_LARGE = 7          /* the problem needs more scratch than HGF_STATIC_SCRATCH_BYTES */
 } hgf_status;
 
 /* flags of hgf_linear_forward / hgf_workspace_bytes */
@@ -128,6 +129,43 @@ hgf_status hgf_linear_forward(const void *x, int64_t M, const void *packed, floa
                               int32_t r, const float *gate, void *y, void *workspace,
                               size_t workspace_bytes, const hgf_debug_out *dbg, uint32_t flags,
                               void *stream);
+
+/*
+ * hgf_linear_forward for callers that cannot hand over a workspace.  (The paper has no counterpart:
+ * this is a convenience of the library, not a step of the method.)
+ *
+ * Who needs it: code that runs where device memory may not be allocated - a serving loop whose
+ * memory plan was fixed at start-up and is fully spent, a plug-in inside a host framework that owns
+ * every byte of device memory through its own pool and forbids cudaMalloc behind its back, or a
+ * latency-critical decode thread for which cudaMalloc's implicit device-wide synchronisation is a
+ * stall it cannot afford.  Such a caller still owns x, the weights and y, but has nowhere to get
+ * the few hundred KiB of scratch that the layer's kernels exchange intermediate results through.
+ *
+ * This entry point takes that scratch from an array that is part of the library image itself
+ * (HGF_STATIC_SCRATCH_BYTES of device memory, held by every GPU that loads the library until the
+ * process exits).  It calls no allocator of any kind.  Arguments are those of hgf_linear_forward
+ * without workspace and debug outputs; results are the same.
+ *
+ * Limits: only decode-sized problems (those hgf_linear_forward serves with its GEMV path, M <=
+ * HGF_DECODE_MAX_M) whose hgf_workspace_bytes(M, d_in, d_out, r, flags) is at most
+ * HGF_STATIC_SCRATCH_BYTES; e.g. M = 16 with d_in <= 6656, or M = 1 with any supported d_in.
+ * A problem that needs more scratch returns HGF_ERR_TOO_LARGE, one that would take the GEMM path
+ * HGF_ERR_UNSUPPORTED_SHAPE; nothing is launched in either case.
+ *
+ * Sharing: all calls on a device use the same array, and it keeps what the last call left in it.
+ * Nothing in it has to be cleared (each call writes every value before reading it), but two calls
+ * whose kernels may run at the same time - different streams, or different host threads without
+ * ordering between their streams - would overwrite each other's intermediates: order them.
+ *
+ * Set-up: the first call on each device looks up the array's device address (the current device
+ * must be the one the pointers belong to).  Make that first call before starting any stream
+ * capture.
+ */
+#define HGF_STATIC_SCRATCH_BYTES (288u * 1024u)
+hgf_status hgf_linear_forward_static(const void *x, int64_t M, const void *packed, float gamma,
+                                     int64_t d_in, int64_t d_out, const void *At, const void *Bt,
+                                     int32_t r, const float *gate, void *y, uint32_t flags,
+                                     void *stream);
 
 /*
  * A group of independent decode-sized layer problems served by one pair of launches.  The paper's

@@ -182,6 +182,42 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
     return launch_prefill_gemm(gp, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
 }
 
+// ---- a forward call that allocates nothing ------------------------------------------------------
+// Scratch for callers that cannot provide a workspace: part of the library image, one copy per
+// device that loads it.  In host code the name below is only a handle for the symbol, never a
+// device address; the address a kernel can use comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[HGF_STATIC_SCRATCH_BYTES];
+
+namespace hgf {
+static void *static_scratch_address() {
+    constexpr int kMaxDevices = 64;
+    static std::atomic<void *> cache[kMaxDevices];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    void *ptr = cache[dev].load(std::memory_order_acquire);
+    if (!ptr) {
+        if (cudaGetSymbolAddress((void **)&ptr, g_static_scratch) != cudaSuccess || !ptr) return nullptr;
+        cache[dev].store(ptr, std::memory_order_release);
+    }
+    return ptr;
+}
+}  // namespace hgf
+
+extern "C" hgf_status hgf_linear_forward_static(const void *x, int64_t M, const void *packed, float gamma, int64_t d_in,
+                                                int64_t d_out, const void *At, const void *Bt, int32_t r,
+                                                const float *gate, void *y, uint32_t flags, void *stream) {
+    if (M <= 0 || d_in <= 0 || d_out <= 0 || r < 0) return HGF_ERR_INVALID_ARG;
+    if (flags & HGF_FLAG_FORCE_GEMM) return HGF_ERR_INVALID_ARG;
+    if (d_in % 64 != 0 || d_in > 65536 || M > HGF_DECODE_MAX_M) return HGF_ERR_UNSUPPORTED_SHAPE;
+    const int32_t r_eff = (At && Bt && gate) ? r : 0;
+    if (ws_layout(M, d_in, r_eff, false).total > (size_t)HGF_STATIC_SCRATCH_BYTES) return HGF_ERR_TOO_LARGE;
+    if (takes_gemm_path(M, d_in, flags)) return HGF_ERR_UNSUPPORTED_SHAPE;
+    void *scratch = static_scratch_address();
+    if (!scratch) return HGF_ERR_CUDA;
+    return hgf_linear_forward(x, M, packed, gamma, d_in, d_out, At, Bt, r, gate, y, scratch, HGF_STATIC_SCRATCH_BYTES,
+                              nullptr, flags, stream);
+}
+
 // ---- groups of independent decode problems --------------------------------------------------------
 struct hgf_group {
     int n, total_tiles, total_blocks, max_M, xq_smem_bytes, device;
@@ -388,6 +424,7 @@ extern "C" const char *hgf_status_string(hgf_status s) {
         case HGF_ERR_WORKSPACE: return "workspace missing or too small";
         case HGF_ERR_CUDA: return "CUDA error";
         case HGF_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case HGF_ERR_TOO_LARGE: return "the problem needs more scratch than the library's built-in array holds";
     }
     return "unknown status";
 }

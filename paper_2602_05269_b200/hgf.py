@@ -26,7 +26,7 @@ PHASE_GEMV = 0x2
 EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_workspace_bytes",
            "hgf_linear_forward", "hgf_act_quant", "hgf_check_status", "hgf_tmax_tokens_per_s",
            "hgf_launch_count", "hgf_status_string", "hgf_group_create", "hgf_group_forward",
-           "hgf_group_destroy", "hgf_group_forward_phases"]
+           "hgf_group_destroy", "hgf_group_forward_phases", "hgf_linear_forward_static"]
 
 
 class HgfError(RuntimeError):
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.hgf_linear_forward.restype = c.c_int
         L.hgf_linear_forward.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, vp, sz,
                                          c.POINTER(DebugOut), u32, vp]
+        L.hgf_linear_forward_static.restype = c.c_int
+        L.hgf_linear_forward_static.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, u32, vp]
         L.hgf_act_quant.restype = c.c_int
         L.hgf_act_quant.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.hgf_check_status.restype = c.c_int
@@ -181,6 +183,25 @@ def linear_forward(x, packed, gamma, d_in, d_out, At=None, Bt=None, gate=None, *
     if debug:
         dbg["h"] = dbg["h"][:, :r]
         return y, dbg
+    return y
+
+
+STATIC_SCRATCH_BYTES = 288 * 1024
+
+
+def linear_forward_static(x, packed, gamma, d_in, d_out, y, At=None, Bt=None, gate=None, *, flags=0, stream=None):
+    """hgf_linear_forward_static: the layer forward for callers that may not allocate device memory.
+
+    Everything, y included, is passed in; the call itself allocates nothing (no workspace tensor, no
+    debug outputs): the library uses a scratch array built into its image.  Decode-sized problems
+    only; HgfError status 7 if the problem needs more scratch than STATIC_SCRATCH_BYTES.  Calls on
+    one device share that array, so they must not overlap on the GPU.
+    """
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and y.is_cuda and y.is_contiguous()
+    r = 0 if At is None else At.shape[0]
+    st = lib().hgf_linear_forward_static(_ptr(x), x.shape[0], _ptr(packed), ctypes.c_float(gamma), d_in, d_out,
+                                         _ptr(At), _ptr(Bt), r, _ptr(gate), _ptr(y), flags, _stream(stream))
+    _check("hgf_linear_forward_static", st)
     return y
 
 
