@@ -1,15 +1,17 @@
 // GEMM path (M > 16 tokens): Y_int = X~ x T^T on the 5th-generation tensor cores
 // (tcgen05.mma kind::i8, int32 accumulators in tensor memory), with the dequantisation, the
-// LoRA up-projection (a second, small tcgen05.mma kind::f16 into an fp32 accumulator) and the
-// gated fusion in the epilogue.  Algorithm 1, steps 3, 4, 7, 8.
+// LoRA up-projection (a second, small tcgen05.mma kind::f16 on top of the dequantised accumulator,
+// with the gate folded into B) and the gated fusion in the epilogue.  Two accumulators alternate,
+// so the epilogue of a tile runs under the main loop of the next.  Algorithm 1, steps 3, 4, 7, 8.
 //
 // One persistent CTA per SM, 10 warps with fixed roles:
 //   warp 0      TMA producer: per 128-wide k block, the int8 activation tile (128 tokens x 128 B,
 //               128-byte swizzle) and the packed weight tile (256 rows x 32 B, gathered
 //               from 16 consecutive row tiles of the tiled weight layout)
 //   warp 1      allocates tensor memory; one lane issues the MMAs and commits to mbarriers
-//   warps 2-5   epilogue: stage the LoRA operands of the tile, then read both accumulators with
-//               tcgen05.ld, combine, and write through shared memory with TMA stores
+//   warps 2-5   epilogue: stage the LoRA operands of the tile, dequantise the accumulator in place
+//               (tcgen05.ld / tcgen05.st), wait for the correction MMA, read the result and write it
+//               through shared memory with TMA stores
 //   warps 6-9   expand the 2-bit codes of a packed tile into the int8, K-major, 128-byte-swizzled
 //               operand layout the tensor core reads from shared memory
 // The tile is 128 tokens (MMA M) x 256 output channels (MMA N).  Codes are c = t + 1 (both operands
@@ -33,7 +35,7 @@ constexpr int LORA_A_BYTES = TILE_M * 128;       // 128 tokens x 64 fp16
 constexpr int LORA_B_BYTES = TILE_N * 128;       // 256 channels x 64 fp16
 constexpr int STORE_BUF_BYTES = 32 * 128;        // 32 rows x 128 B per epilogue warp and buffer
 constexpr int GEMM_THREADS = 320;
-constexpr int TMEM_COLS = 512, TMEM_COL_INT = 0, TMEM_COL_FP = 256;
+constexpr int TMEM_COLS = 512, ACC_COLS = 256;  // two accumulators of 128 lanes x 256 columns
 
 constexpr int OFF_X = 0;
 constexpr int OFF_B = OFF_X + XSTAGES * X_TILE_BYTES;
@@ -41,15 +43,14 @@ constexpr int OFF_LA = OFF_B + BSTAGES * B_TILE_BYTES;
 constexpr int OFF_LB = OFF_LA + LORA_A_BYTES;
 constexpr int OFF_ST = OFF_LB + LORA_B_BYTES;
 constexpr int OFF_P = OFF_ST + 4 * 2 * STORE_BUF_BYTES;
-constexpr int OFF_GATE = OFF_P + XSTAGES * P_TILE_BYTES;
-constexpr int OFF_BAR = OFF_GATE + 4 * TILE_N * 4;  // one gate copy per epilogue warp
+constexpr int OFF_BAR = OFF_P + XSTAGES * P_TILE_BYTES;
 constexpr int SMEM_USED = OFF_BAR + 256;
 constexpr int SMEM_BYTES = SMEM_USED + 1024;  // slack for the 1024-byte alignment of the base
 
 // barrier slots (8 bytes each) inside the OFF_BAR block
 enum { BAR_FULL = 0, BAR_EMPTY = BAR_FULL + XSTAGES, BAR_BFULL = BAR_EMPTY + XSTAGES,
-       BAR_BEMPTY = BAR_BFULL + BSTAGES, BAR_ACCFULL = BAR_BEMPTY + BSTAGES, BAR_ACCEMPTY,
-       BAR_LORAFULL, BAR_COUNT };
+       BAR_BEMPTY = BAR_BFULL + BSTAGES, BAR_ACCFULL = BAR_BEMPTY + BSTAGES, BAR_ACCEMPTY = BAR_ACCFULL + 2,
+       BAR_LORAREADY = BAR_ACCEMPTY + 2, BAR_LORADONE = BAR_LORAREADY + 2, BAR_COUNT = BAR_LORADONE + 2 };
 static_assert(BAR_COUNT * 8 + 16 <= 256, "barrier block too small");
 
 constexpr uint32_t kSpinLimit = 1u << 22;            // polls of a drain loop
@@ -158,6 +159,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
 
 // Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, groups of 8 rows
@@ -202,9 +215,12 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             mbar_init(bar(BAR_BFULL + u), 4);
             mbar_init(bar(BAR_BEMPTY + u), 1);
         }
-        mbar_init(bar(BAR_ACCFULL), 1);
-        mbar_init(bar(BAR_ACCEMPTY), 4);
-        mbar_init(bar(BAR_LORAFULL), 4);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(BAR_ACCFULL + b), 1);
+            mbar_init(bar(BAR_ACCEMPTY + b), 4);
+            mbar_init(bar(BAR_LORAREADY + b), 4);
+            mbar_init(bar(BAR_LORADONE + b), 1);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         fence_proxy_async();
@@ -250,16 +266,35 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
+        // Tile `it` accumulates into accumulator it % 2, so the epilogue of one tile runs under the
+        // main loop of the next.  With a correction, the epilogue first rewrites the accumulator as
+        // fp32 (dequantised), then this thread adds (H) (g B)^T into it with one more MMA, slipped in
+        // between the k blocks of the tile in progress as soon as the epilogue is ready for it.
         if (lane == 0) {
             int s = 0, u = 0;
             uint32_t ph = 0, bph = 0;
             bool ok = true;
-            int it = 0;
+            int it = 0, pend = -1;  // pend: tile whose correction MMA is still to be issued
+            auto issue_lora = [&](int t) {
+                const int b = t & 1;
+                tc_fence_after();
+                const uint64_t adesc = make_sw128_desc(sbase + OFF_LA);
+                const uint64_t bdesc = make_sw128_desc(sbase + OFF_LB);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)  // 64 fp16 = 4 x (K = 16), on top of the fp32 values
+                    mma_f16(tmem_base + b * ACC_COLS, adesc + 2u * kk, bdesc + 2u * kk, IDESC_F16, 1u);
+                tc_commit(bar(BAR_LORADONE + b));
+            };
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-                if (it > 0 && !(ok = mbar_wait(bar(BAR_ACCEMPTY), (uint32_t)(it - 1) & 1u, abort_flag, status, 0x200u)))
+                const int b = it & 1;
+                if (it >= 2 && !(ok = mbar_wait(bar(BAR_ACCEMPTY + b), (uint32_t)((it >> 1) - 1) & 1u, abort_flag, status, 0x200u)))
                     break;
                 tc_fence_after();
                 for (int kb = 0; kb < kblocks; ++kb) {
+                    if (pend >= 0 && mbar_try_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u)) {
+                        issue_lora(pend);
+                        pend = -1;
+                    }
                     if (!(ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag, status, 0x210u + s))) break;
                     if (!(ok = mbar_wait(bar(BAR_BFULL + u), bph, abort_flag, status, 0x220u + u))) break;
                     tc_fence_after();
@@ -267,32 +302,31 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint64_t bdesc = make_sw128_desc(sbase + OFF_B + u * B_TILE_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < KBLK / 32; ++kk)
-                        mma_i8(tmem_base + TMEM_COL_INT, adesc + 2u * kk, bdesc + 2u * kk, IDESC_I8,
-                               (kb | kk) ? 1u : 0u);
+                        mma_i8(tmem_base + b * ACC_COLS, adesc + 2u * kk, bdesc + 2u * kk, IDESC_I8, (kb | kk) ? 1u : 0u);
                     tc_commit(bar(BAR_EMPTY + s));
                     tc_commit(bar(BAR_BEMPTY + u));
                     if (++s == XSTAGES) { s = 0; ph ^= 1u; }
                     if (++u == BSTAGES) { u = 0; bph ^= 1u; }
                 }
                 if (!ok) break;
-                if (has_lora) {
-                    if (!(ok = mbar_wait(bar(BAR_LORAFULL), (uint32_t)it & 1u, abort_flag, status, 0x230u))) break;
-                    tc_fence_after();
-                    const uint64_t adesc = make_sw128_desc(sbase + OFF_LA);
-                    const uint64_t bdesc = make_sw128_desc(sbase + OFF_LB);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)  // 64 fp16 = 4 x (K = 16)
-                        mma_f16(tmem_base + TMEM_COL_FP, adesc + 2u * kk, bdesc + 2u * kk, IDESC_F16, kk ? 1u : 0u);
+                tc_commit(bar(BAR_ACCFULL + b));
+                if (pend >= 0) {  // the previous tile's correction has to be out before its accumulator's next turn
+                    if (!(ok = mbar_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x230u)))
+                        break;
+                    issue_lora(pend);
+                    pend = -1;
                 }
-                tc_commit(bar(BAR_ACCFULL));
+                if (has_lora) pend = it;
             }
+            if (ok && pend >= 0 &&
+                mbar_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x231u))
+                issue_lora(pend);
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------------ epilogue warps
         const int e = warp - 2;          // staging role index
         const int q = warp & 3;          // TMEM lane quarter this warp may read
         uint8_t *stbuf = smem + OFF_ST + e * 2 * STORE_BUF_BYTES;
-        float *gate_s = reinterpret_cast<float *>(smem + OFF_GATE) + e * TILE_N;
         const float gw = p.gw_over_127;
         constexpr int ES = OUT_BF16 ? 2 : 4;
         constexpr int COLS_PER_STORE = 128 / ES;  // 32 fp32 or 64 bf16 columns per 128-byte row
@@ -300,7 +334,11 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         int it = 0, sbuf = 0;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
             const int m0 = (tile % tiles_m) * TILE_M, n0 = (tile / tiles_m) * TILE_N;
+            const int b = it & 1;
+            const uint32_t par = (uint32_t)(it >> 1) & 1u;
             if (has_lora) {
+                // (the correction MMA of the previous tile has finished reading these buffers: this warp
+                // waited for it before the previous tile's second pass)
                 // H tile: rows 32 e .. 32 e + 31, 8 chunks of 16 bytes each
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
@@ -309,32 +347,58 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     if (m < p.M) v = *reinterpret_cast<const uint4 *>(p.h16 + (size_t)m * 64 + c * 8);
                     *reinterpret_cast<uint4 *>(smem + OFF_LA + row * 128 + ((c ^ (row & 7)) << 4)) = v;
                 }
-                // B^T tile: rows 64 e .. 64 e + 63
+                // (g B)^T tile: rows 64 e .. 64 e + 63, each row of B^T scaled by its channel's gate
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const int idx = i * 32 + lane, row = 64 * e + idx / 8, c = idx % 8, n = n0 + row;
                     uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (n < p.N && c * 8 < p.r) v = *reinterpret_cast<const uint4 *>(p.Bt + (size_t)n * p.r + c * 8);
+                    if (n < p.N && c * 8 < p.r) {
+                        v = *reinterpret_cast<const uint4 *>(p.Bt + (size_t)n * p.r + c * 8);
+                        const float g = p.gate[n];
+                        __half2 *h2 = reinterpret_cast<__half2 *>(&v);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const float2 f = __half22float2(h2[k]);
+                            h2[k] = __floats2half2_rn(g * f.x, g * f.y);
+                        }
+                    }
                     *reinterpret_cast<uint4 *>(smem + OFF_LB + row * 128 + ((c ^ (row & 7)) << 4)) = v;
                 }
-#pragma unroll
-                for (int i = 0; i < TILE_N / 32; ++i) {  // this warp's own copy of the tile's gate values
-                    const int col = 32 * i + lane, n = n0 + col;
-                    gate_s[col] = n < p.N ? p.gate[n] : 0.0f;
-                }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_LORAFULL));
             }
 
             const int m = m0 + 32 * q + lane;  // this thread's token = its TMEM lane
             const float scale = m < p.M ? p.gamma_x[m] * gw : 0.0f;
             const int rs = m < p.M ? p.row_sum[m] : 0;
 
-            ok = mbar_wait(bar(BAR_ACCFULL), (uint32_t)it & 1u, abort_flag, status, 0x300u);
+            ok = mbar_wait(bar(BAR_ACCFULL + b), par, abort_flag, status, 0x300u);
             if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
             tc_fence_after();
-            const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16);
+            const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16) + b * ACC_COLS;
+
+            if (has_lora) {
+                // first pass: dequantise in place (int32 -> fp32), then let the MMA warp add the correction
+                for (int cc = 0; cc < TILE_N; cc += 32) {
+                    uint32_t ai[32];
+                    tmem_ld32(lane_base + cc, ai);
+                    tmem_ld_wait();
+                    if (p.dbg_y_int && m < p.M) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + cc + j < p.N) p.dbg_y_int[(size_t)m * p.N + n0 + cc + j] = (int)ai[j] - rs;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) ai[j] = __float_as_uint((float)((int)ai[j] - rs) * scale);
+                    tmem_st32(lane_base + cc, ai);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                fence_proxy_async();  // the staged H and (g B)^T tiles
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_LORAREADY + b));
+                ok = mbar_wait(bar(BAR_LORADONE + b), par, abort_flag, status, 0x310u);
+                if (!(ok = __all_sync(0xffffffffu, ok))) break;
+                tc_fence_after();
+            }
 
             for (int c0 = 0; c0 < TILE_N; c0 += COLS_PER_STORE) {
                 uint8_t *buf = stbuf + sbuf * STORE_BUF_BYTES;
@@ -344,23 +408,24 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 #pragma unroll
                 for (int sub = 0; sub < COLS_PER_STORE / 32; ++sub) {
                     const int cc = c0 + 32 * sub;
-                    uint32_t ai[32], af[32];
-                    tmem_ld32(lane_base + TMEM_COL_INT + cc, ai);
-                    if (has_lora) tmem_ld32(lane_base + TMEM_COL_FP + cc, af);
+                    uint32_t ai[32];
+                    tmem_ld32(lane_base + cc, ai);
                     tmem_ld_wait();
                     float yv[32];
+                    if (has_lora) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int yi = (int)ai[j] - rs;
-                        float y = (float)yi * scale;
-                        if (has_lora) y = fmaf(gate_s[cc + j], __uint_as_float(af[j]), y);
-                        yv[j] = y;
-                        ai[j] = (uint32_t)yi;
-                    }
-                    if (p.dbg_y_int && m < p.M) {
+                        for (int j = 0; j < 32; ++j) yv[j] = __uint_as_float(ai[j]);
+                    } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (n0 + cc + j < p.N) p.dbg_y_int[(size_t)m * p.N + n0 + cc + j] = (int)ai[j];
+                        for (int j = 0; j < 32; ++j) {
+                            ai[j] = (uint32_t)((int)ai[j] - rs);
+                            yv[j] = (float)(int)ai[j] * scale;
+                        }
+                        if (p.dbg_y_int && m < p.M) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (n0 + cc + j < p.N) p.dbg_y_int[(size_t)m * p.N + n0 + cc + j] = (int)ai[j];
+                        }
                     }
                     if (OUT_BF16) {
 #pragma unroll
@@ -391,10 +456,10 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
                 sbuf ^= 1;
             }
-            // all TMEM reads of this tile are done: hand the accumulators back to the MMA warp
+            // all TMEM reads of this tile are done: hand the accumulator back to the MMA warp
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_ACCEMPTY));
+            if (lane == 0) mbar_arrive(bar(BAR_ACCEMPTY + b));
         }
         if (lane == 0) bulk_wait_read<0>();
         __syncwarp();
