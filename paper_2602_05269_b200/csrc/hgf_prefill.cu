@@ -1,21 +1,28 @@
 // GEMM path (M > 16 tokens): Y_int = X~ x T^T on the 5th-generation tensor cores
-// (tcgen05.mma kind::i8, int32 accumulators in tensor memory), with the dequantisation, the
-// LoRA up-projection (a second, small tcgen05.mma kind::f16 on top of the dequantised accumulator,
-// with the gate folded into B) and the gated fusion in the epilogue.  Two accumulators alternate,
-// so the epilogue of a tile runs under the main loop of the next.  Algorithm 1, steps 3, 4, 7, 8.
+// (tcgen05.mma kind::i8, int32 accumulator in tensor memory), with the dequantisation, the LoRA
+// up-projection (a small tcgen05.mma kind::f16 on top of the dequantised accumulator, with the gate
+// folded into B) and the gated fusion in the epilogue.  Algorithm 1, steps 3, 4, 7, 8.
+//
+// The ternary weights are the MMA's first operand and are read from TENSOR MEMORY: the tensor core
+// cannot read 2-bit codes, and expanding them to int8 in shared memory costs four times their bytes
+// in shared-memory writes plus the same again when the MMA reads them - more than the port has.
+// Here four warps expand a packed 128 x 128 tile straight from its 4 KiB in shared memory into
+// registers (one 128-channel row per thread: a shift and a mask per register) and store it with one
+// tcgen05.st into the operand's place in tensor memory, so shared memory carries only the int8
+// activation tile (TMA in, MMA out) and the packed codes.  The output tile is therefore
+// 128 output channels (tensor-memory lanes, MMA M) x 256 tokens (columns, MMA N).
 //
 // One persistent CTA per SM, 10 warps with fixed roles:
-//   warp 0      TMA producer: per 128-wide k block, the int8 activation tile (128 tokens x 128 B,
-//               128-byte swizzle) and the packed weight tile (256 rows x 32 B, gathered
-//               from 16 consecutive row tiles of the tiled weight layout)
+//   warp 0      TMA producer: per 128-wide k block the int8 activation tile (256 tokens x 128 B,
+//               128-byte swizzle) and the packed weight tile (128 rows x 32 B, gathered from 8
+//               consecutive row tiles of the tiled weight layout)
 //   warp 1      allocates tensor memory; one lane issues the MMAs and commits to mbarriers
-//   warps 2-5   epilogue: stage the LoRA operands of the tile, dequantise the accumulator in place
-//               (tcgen05.ld / tcgen05.st), wait for the correction MMA, read the result and write it
-//               through shared memory with TMA stores
-//   warps 6-9   expand the 2-bit codes of a packed tile into the int8, K-major, 128-byte-swizzled
-//               operand layout the tensor core reads from shared memory
-// The tile is 128 tokens (MMA M) x 256 output channels (MMA N).  Codes are c = t + 1 (both operands
-// are declared signed 8-bit; 0, 1, 2 read the same either way); sum_k t x~ = sum_k c x~ - sum_k x~ is restored in the epilogue from the row sums.
+//   warps 2-5   epilogue: stage the correction's operands, dequantise the accumulator in place
+//               (tcgen05.ld / tcgen05.st), wait for the correction MMA, read the result, transpose it
+//               through shared memory and store y with TMA
+//   warps 6-9   expand the packed tile into tensor memory
+// Codes are c = t + 1 (both operands are declared signed 8-bit; 0, 1, 2 read the same either way);
+// sum_k t x~ = sum_k c x~ - sum_k x~ is restored in the epilogue from the row sums.
 //
 // Every wait is bounded: when one gives up, the CTA records it in the device status word, all
 // roles leave their loops, in-flight bulk copies are drained, tensor memory is freed and the
@@ -26,31 +33,33 @@
 
 namespace hgf {
 
-constexpr int TILE_M = 128, TILE_N = 256, KBLK = 128;
-constexpr int XSTAGES = 3, BSTAGES = 2;
-constexpr int X_TILE_BYTES = TILE_M * KBLK;      // 16 KiB
-constexpr int P_TILE_BYTES = TILE_N * KBLK / 4;  // 8 KiB
-constexpr int B_TILE_BYTES = TILE_N * KBLK;      // 32 KiB
-constexpr int LORA_A_BYTES = TILE_M * 128;       // 128 tokens x 64 fp16
-constexpr int LORA_B_BYTES = TILE_N * 128;       // 256 channels x 64 fp16
-constexpr int STORE_BUF_BYTES = 32 * 128;        // 32 rows x 128 B per epilogue warp and buffer
+constexpr int TILE_C = 128;   // output channels per tile (MMA M, tensor-memory lanes)
+constexpr int TILE_T = 256;   // tokens per tile (MMA N, accumulator columns)
+constexpr int KBLK = 128;
+constexpr int STAGES = 4;
+constexpr int X_TILE_BYTES = TILE_T * KBLK;      // 32 KiB
+constexpr int P_TILE_BYTES = TILE_C * KBLK / 4;  // 4 KiB
+constexpr int LORA_H_BYTES = TILE_T * 128;       // 256 tokens x 64 fp16
+constexpr int LORA_B_BYTES = TILE_C * 128;       // 128 channels x 64 fp16
+constexpr int TOKV_BYTES = TILE_T * 8;           // per epilogue warp: row sum and scale of the tile's tokens
+constexpr int STORE_BUF_BYTES = 32 * 32 * 4;     // per epilogue warp: 32 tokens x 32 channels
 constexpr int GEMM_THREADS = 320;
-constexpr int TMEM_COLS = 512, ACC_COLS = 256;  // two accumulators of 128 lanes x 256 columns
+constexpr int TMEM_COLS = 512, ACC_COL = 0, A_COL = 256, A_STAGE_COLS = KBLK / 4;  // 32 columns = 128 int8 per lane
 
 constexpr int OFF_X = 0;
-constexpr int OFF_B = OFF_X + XSTAGES * X_TILE_BYTES;
-constexpr int OFF_LA = OFF_B + BSTAGES * B_TILE_BYTES;
-constexpr int OFF_LB = OFF_LA + LORA_A_BYTES;
-constexpr int OFF_ST = OFF_LB + LORA_B_BYTES;
-constexpr int OFF_P = OFF_ST + 4 * 2 * STORE_BUF_BYTES;
-constexpr int OFF_BAR = OFF_P + XSTAGES * P_TILE_BYTES;
+constexpr int OFF_LH = OFF_X + STAGES * X_TILE_BYTES;
+constexpr int OFF_LB = OFF_LH + LORA_H_BYTES;
+constexpr int OFF_P = OFF_LB + LORA_B_BYTES;
+constexpr int OFF_TOKV = OFF_P + STAGES * P_TILE_BYTES;
+constexpr int OFF_ST = OFF_TOKV + 4 * TOKV_BYTES;
+constexpr int OFF_BAR = OFF_ST + 4 * STORE_BUF_BYTES;
+static_assert(OFF_BAR + 256 + 1024 <= 227 * 1024, "shared memory budget");
 constexpr int SMEM_USED = OFF_BAR + 256;
 constexpr int SMEM_BYTES = SMEM_USED + 1024;  // slack for the 1024-byte alignment of the base
 
 // barrier slots (8 bytes each) inside the OFF_BAR block
-enum { BAR_FULL = 0, BAR_EMPTY = BAR_FULL + XSTAGES, BAR_BFULL = BAR_EMPTY + XSTAGES,
-       BAR_BEMPTY = BAR_BFULL + BSTAGES, BAR_ACCFULL = BAR_BEMPTY + BSTAGES, BAR_ACCEMPTY = BAR_ACCFULL + 2,
-       BAR_LORAREADY = BAR_ACCEMPTY + 2, BAR_LORADONE = BAR_LORAREADY + 2, BAR_COUNT = BAR_LORADONE + 2 };
+enum { BAR_FULL = 0, BAR_EMPTY = BAR_FULL + STAGES, BAR_AFULL = BAR_EMPTY + STAGES, BAR_ACCFULL = BAR_AFULL + STAGES,
+       BAR_ACCEMPTY, BAR_LORAREADY, BAR_LORADONE, BAR_COUNT };
 static_assert(BAR_COUNT * 8 + 16 <= 256, "barrier block too small");
 
 constexpr uint32_t kSpinLimit = 1u << 22;            // polls of a drain loop
@@ -84,14 +93,20 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after kWaitLimitNs of wall time (and at the latest after kSpinLimit polls
-// past the first clock reading).  Returns false if it gave up or another role already aborted.
+// Bounded wait: gives up after kWaitLimitNs of wall time.  Returns false if it gave up or another
+// role already aborted.  A waiting warp sleeps between polls (20 ns, growing to 320 ns): the roles of
+// this kernel share the SM's schedulers and its shared-memory pipe, and warps that poll without a
+// pause slow the ones that have work.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           unsigned int *status, unsigned int code) {
+    if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;
+    unsigned int ns = 20;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        __nanosleep(ns);
+        if (ns < 320) ns *= 2;
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 127u) == 127u) {
+        if ((i & 63u) == 63u) {
             if (*abort_flag) return false;
             const unsigned long long now = global_timer_ns();
             if (t0 == 0) t0 = now;
@@ -181,12 +196,20 @@ __device__ __forceinline__ uint64_t make_sw128_desc(uint32_t saddr) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
            (2ull << 61);
 }
+__device__ __forceinline__ void mma_i8_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n}\n"
+        ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // Instruction descriptor: D format (bits 4-5), A format (7-9), B format (10-12), K-major A and B,
 // N >> 3 (17-22), M >> 4 (24-28).
-constexpr uint32_t IDESC_I8 = (2u << 4) /*s32*/ | (1u << 7) /*A s8*/ | (1u << 10) /*B s8: the codes 0..2 read the same*/ |
-                              ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+constexpr uint32_t IDESC_I8 = (2u << 4) /*s32*/ | (1u << 7) /*A s8*/ | (1u << 10) /*B s8*/ |
+                              ((uint32_t)(TILE_T >> 3) << 17) | ((uint32_t)(TILE_C >> 4) << 24);
 constexpr uint32_t IDESC_F16 = (1u << 4) /*f32*/ | (0u << 7) /*A f16*/ | (0u << 10) /*B f16*/ |
-                               ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+                               ((uint32_t)(TILE_T >> 3) << 17) | ((uint32_t)(TILE_C >> 4) << 24);
 
 template <bool OUT_BF16>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -201,26 +224,21 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_BAR + BAR_COUNT * 8 + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int tiles_m = (p.M + TILE_M - 1) / TILE_M, tiles_n = (p.N + TILE_N - 1) / TILE_N;
-    const int num_tiles = tiles_m * tiles_n;
+    const int tiles_t = (p.M + TILE_T - 1) / TILE_T, tiles_c = (p.N + TILE_C - 1) / TILE_C;
+    const int num_tiles = tiles_t * tiles_c;
     const int kblocks = (p.K + KBLK - 1) / KBLK;
     const bool has_lora = p.r > 0;
 
     if (tid == 0) {
-        for (int s = 0; s < XSTAGES; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar(BAR_FULL + s), 1);
-            mbar_init(bar(BAR_EMPTY + s), 1 + 4);  // MMA commit + four unpack warps
+            mbar_init(bar(BAR_EMPTY + s), 1 + 4);  // MMA commit (activations read) + four unpack warps (codes read)
+            mbar_init(bar(BAR_AFULL + s), 4);
         }
-        for (int u = 0; u < BSTAGES; ++u) {
-            mbar_init(bar(BAR_BFULL + u), 4);
-            mbar_init(bar(BAR_BEMPTY + u), 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar(BAR_ACCFULL + b), 1);
-            mbar_init(bar(BAR_ACCEMPTY + b), 4);
-            mbar_init(bar(BAR_LORAREADY + b), 4);
-            mbar_init(bar(BAR_LORADONE + b), 1);
-        }
+        mbar_init(bar(BAR_ACCFULL), 1);
+        mbar_init(bar(BAR_ACCEMPTY), 4);
+        mbar_init(bar(BAR_LORAREADY), 4);
+        mbar_init(bar(BAR_LORADONE), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         fence_proxy_async();
@@ -241,24 +259,24 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         if (lane == 0) {
             int s = 0;
             uint32_t ph = 0;
-            uint32_t issued[XSTAGES] = {0, 0, 0};
+            uint32_t issued[STAGES] = {0, 0, 0, 0};
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int m0 = (tile % tiles_m) * TILE_M, n0 = (tile / tiles_m) * TILE_N;
+                const int t0 = (tile % tiles_t) * TILE_T, c0 = (tile / tiles_t) * TILE_C;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!(ok = mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x100u + s))) break;
                     mbar_arrive_expect_tx(bar(BAR_FULL + s), X_TILE_BYTES + P_TILE_BYTES);
-                    tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, m0, bar(BAR_FULL + s));
-                    // packed weights: bytes 32 (kb % 2) .. + 31 of the 16 rows of column tile kb / 2, for 16 row tiles
-                    tma_load_4d(sbase + OFF_P + s * P_TILE_BYTES, &tmap_w, (kb & 1) * 32, 0, kb >> 1, n0 >> 4,
+                    tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, t0, bar(BAR_FULL + s));
+                    // packed weights: bytes 32 (kb % 2) .. + 31 of the 16 rows of column tile kb / 2, for 8 row tiles
+                    tma_load_4d(sbase + OFF_P + s * P_TILE_BYTES, &tmap_w, (kb & 1) * 32, 0, kb >> 1, c0 >> 4,
                                 bar(BAR_FULL + s));
                     ++issued[s];
-                    if (++s == XSTAGES) { s = 0; ph ^= 1u; }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
             // drain: wait (bounded) until every copy this thread issued has landed, so that the CTA
             // never exits with a bulk copy in flight (immediate when the consumers ran to the end)
-            for (int q = 0; q < XSTAGES; ++q)
+            for (int q = 0; q < STAGES; ++q)
                 if (issued[q]) {
                     const uint32_t par = (issued[q] - 1u) & 1u;
                     for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_FULL + q), par); ++i) {}
@@ -266,91 +284,77 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        // Tile `it` accumulates into accumulator it % 2, so the epilogue of one tile runs under the
-        // main loop of the next.  With a correction, the epilogue first rewrites the accumulator as
-        // fp32 (dequantised), then this thread adds (H) (g B)^T into it with one more MMA, slipped in
-        // between the k blocks of the tile in progress as soon as the epilogue is ready for it.
         if (lane == 0) {
-            int s = 0, u = 0;
-            uint32_t ph = 0, bph = 0;
+            int s = 0;
+            uint32_t ph = 0;
             bool ok = true;
-            int it = 0, pend = -1;  // pend: tile whose correction MMA is still to be issued
-            auto issue_lora = [&](int t) {
-                const int b = t & 1;
-                tc_fence_after();
-                const uint64_t adesc = make_sw128_desc(sbase + OFF_LA);
-                const uint64_t bdesc = make_sw128_desc(sbase + OFF_LB);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)  // 64 fp16 = 4 x (K = 16), on top of the fp32 values
-                    mma_f16(tmem_base + b * ACC_COLS, adesc + 2u * kk, bdesc + 2u * kk, IDESC_F16, 1u);
-                tc_commit(bar(BAR_LORADONE + b));
-            };
+            int it = 0;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-                const int b = it & 1;
-                if (it >= 2 && !(ok = mbar_wait(bar(BAR_ACCEMPTY + b), (uint32_t)((it >> 1) - 1) & 1u, abort_flag, status, 0x200u)))
+                if (it > 0 && !(ok = mbar_wait(bar(BAR_ACCEMPTY), (uint32_t)(it - 1) & 1u, abort_flag, status, 0x200u)))
                     break;
                 tc_fence_after();
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (pend >= 0 && mbar_try_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u)) {
-                        issue_lora(pend);
-                        pend = -1;
-                    }
                     if (!(ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag, status, 0x210u + s))) break;
-                    if (!(ok = mbar_wait(bar(BAR_BFULL + u), bph, abort_flag, status, 0x220u + u))) break;
+                    if (!(ok = mbar_wait(bar(BAR_AFULL + s), ph, abort_flag, status, 0x220u + s))) break;
                     tc_fence_after();
-                    const uint64_t adesc = make_sw128_desc(sbase + OFF_X + s * X_TILE_BYTES);
-                    const uint64_t bdesc = make_sw128_desc(sbase + OFF_B + u * B_TILE_BYTES);
+                    const uint64_t bdesc = make_sw128_desc(sbase + OFF_X + s * X_TILE_BYTES);
+                    const uint32_t a_tmem = tmem_base + A_COL + s * A_STAGE_COLS;
 #pragma unroll
-                    for (int kk = 0; kk < KBLK / 32; ++kk)
-                        mma_i8(tmem_base + b * ACC_COLS, adesc + 2u * kk, bdesc + 2u * kk, IDESC_I8, (kb | kk) ? 1u : 0u);
+                    for (int kk = 0; kk < KBLK / 32; ++kk)  // 32 int8 = 8 columns of the weight operand, 32 bytes of a token row
+                        mma_i8_ts(tmem_base + ACC_COL, a_tmem + 8u * kk, bdesc + 2u * kk, IDESC_I8, (kb | kk) ? 1u : 0u);
                     tc_commit(bar(BAR_EMPTY + s));
-                    tc_commit(bar(BAR_BEMPTY + u));
-                    if (++s == XSTAGES) { s = 0; ph ^= 1u; }
-                    if (++u == BSTAGES) { u = 0; bph ^= 1u; }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit(bar(BAR_ACCFULL + b));
-                if (pend >= 0) {  // the previous tile's correction has to be out before its accumulator's next turn
-                    if (!(ok = mbar_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x230u)))
-                        break;
-                    issue_lora(pend);
-                    pend = -1;
+                tc_commit(bar(BAR_ACCFULL));
+                if (has_lora) {
+                    // the epilogue has rewritten the accumulator as fp32: add (g B) H^T on top
+                    if (!(ok = mbar_wait(bar(BAR_LORAREADY), (uint32_t)it & 1u, abort_flag, status, 0x230u))) break;
+                    tc_fence_after();
+                    const uint64_t adesc = make_sw128_desc(sbase + OFF_LB);
+                    const uint64_t bdesc = make_sw128_desc(sbase + OFF_LH);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)  // 64 fp16 = 4 x (K = 16)
+                        mma_f16(tmem_base + ACC_COL, adesc + 2u * kk, bdesc + 2u * kk, IDESC_F16, 1u);
+                    tc_commit(bar(BAR_LORADONE));
                 }
-                if (has_lora) pend = it;
             }
-            if (ok && pend >= 0 &&
-                mbar_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x231u))
-                issue_lora(pend);
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------------ epilogue warps
         const int e = warp - 2;          // staging role index
-        const int q = warp & 3;          // TMEM lane quarter this warp may read
-        uint8_t *stbuf = smem + OFF_ST + e * 2 * STORE_BUF_BYTES;
+        const int q = warp & 3;          // tensor-memory lane quarter this warp may access
+        int *tok_rs = reinterpret_cast<int *>(smem + OFF_TOKV + e * TOKV_BYTES);
+        float *tok_sc = reinterpret_cast<float *>(tok_rs + TILE_T);
         const float gw = p.gw_over_127;
-        constexpr int ES = OUT_BF16 ? 2 : 4;
-        constexpr int COLS_PER_STORE = 128 / ES;  // 32 fp32 or 64 bf16 columns per 128-byte row
+        uint8_t *buf = smem + OFF_ST + e * STORE_BUF_BYTES;
         bool ok = true;
-        int it = 0, sbuf = 0;
+        int it = 0;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-            const int m0 = (tile % tiles_m) * TILE_M, n0 = (tile / tiles_m) * TILE_N;
-            const int b = it & 1;
-            const uint32_t par = (uint32_t)(it >> 1) & 1u;
-            if (has_lora) {
-                // (the correction MMA of the previous tile has finished reading these buffers: this warp
-                // waited for it before the previous tile's second pass)
-                // H tile: rows 32 e .. 32 e + 31, 8 chunks of 16 bytes each
+            const int t0 = (tile % tiles_t) * TILE_T, c0 = (tile / tiles_t) * TILE_C;
+            const uint32_t par = (uint32_t)it & 1u;
+            // this warp's copy of the tile's per-token values
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int idx = i * 32 + lane, row = 32 * e + idx / 8, c = idx % 8, m = m0 + row;
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (m < p.M) v = *reinterpret_cast<const uint4 *>(p.h16 + (size_t)m * 64 + c * 8);
-                    *reinterpret_cast<uint4 *>(smem + OFF_LA + row * 128 + ((c ^ (row & 7)) << 4)) = v;
-                }
-                // (g B)^T tile: rows 64 e .. 64 e + 63, each row of B^T scaled by its channel's gate
+            for (int i = 0; i < TILE_T / 32; ++i) {
+                const int tl = 32 * i + lane, m = t0 + tl;
+                tok_rs[tl] = m < p.M ? p.row_sum[m] : 0;
+                tok_sc[tl] = m < p.M ? p.gamma_x[m] * gw : 0.0f;
+            }
+            if (has_lora) {
+                // (the previous tile's correction MMA has finished reading these buffers: this warp waited
+                // for it before its second pass)
+                // H tile: token rows 64 e .. 64 e + 63, 8 chunks of 16 bytes each
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const int idx = i * 32 + lane, row = 64 * e + idx / 8, c = idx % 8, n = n0 + row;
+                    const int idx = i * 32 + lane, row = 64 * e + idx / 8, c = idx % 8, m = t0 + row;
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (m < p.M) v = *reinterpret_cast<const uint4 *>(p.h16 + (size_t)m * 64 + c * 8);
+                    *reinterpret_cast<uint4 *>(smem + OFF_LH + row * 128 + ((c ^ (row & 7)) << 4)) = v;
+                }
+                // (g B)^T tile: channel rows 32 e .. 32 e + 31, each row of B^T scaled by its channel's gate
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int idx = i * 32 + lane, row = 32 * e + idx / 8, c = idx % 8, n = c0 + row;
                     uint4 v = make_uint4(0u, 0u, 0u, 0u);
                     if (n < p.N && c * 8 < p.r) {
                         v = *reinterpret_cast<const uint4 *>(p.Bt + (size_t)n * p.r + c * 8);
@@ -365,140 +369,115 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     *reinterpret_cast<uint4 *>(smem + OFF_LB + row * 128 + ((c ^ (row & 7)) << 4)) = v;
                 }
             }
+            __syncwarp();
 
-            const int m = m0 + 32 * q + lane;  // this thread's token = its TMEM lane
-            const float scale = m < p.M ? p.gamma_x[m] * gw : 0.0f;
-            const int rs = m < p.M ? p.row_sum[m] : 0;
+            const int n = c0 + 32 * q + lane;  // this thread's output channel = its tensor-memory lane
+            const bool n_ok = n < p.N;
 
-            ok = mbar_wait(bar(BAR_ACCFULL + b), par, abort_flag, status, 0x300u);
+            ok = mbar_wait(bar(BAR_ACCFULL), par, abort_flag, status, 0x300u);
             if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
             tc_fence_after();
-            const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16) + b * ACC_COLS;
+            const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16) + ACC_COL;
 
+            // (the per-token values are read as vectors ahead of the arithmetic: a shared-memory load per
+            // element in the dependent chain costs its full latency every time)
+            auto dequant_chunk = [&](int cc, uint32_t (&ai)[32]) {  // int32 sums -> fp32 (Y_int - row sum) * scale
+                if (p.dbg_y_int && n_ok) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (t0 + cc + j < p.M) p.dbg_y_int[(size_t)(t0 + cc + j) * p.N + n] = (int)ai[j] - tok_rs[cc + j];
+                }
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    const int4 rs4 = *reinterpret_cast<const int4 *>(tok_rs + cc + 4 * v);
+                    const float4 sc4 = *reinterpret_cast<const float4 *>(tok_sc + cc + 4 * v);
+                    ai[4 * v + 0] = __float_as_uint((float)((int)ai[4 * v + 0] - rs4.x) * sc4.x);
+                    ai[4 * v + 1] = __float_as_uint((float)((int)ai[4 * v + 1] - rs4.y) * sc4.y);
+                    ai[4 * v + 2] = __float_as_uint((float)((int)ai[4 * v + 2] - rs4.z) * sc4.z);
+                    ai[4 * v + 3] = __float_as_uint((float)((int)ai[4 * v + 3] - rs4.w) * sc4.w);
+                }
+            };
             if (has_lora) {
                 // first pass: dequantise in place (int32 -> fp32), then let the MMA warp add the correction
-                for (int cc = 0; cc < TILE_N; cc += 32) {
+                for (int cc = 0; cc < TILE_T; cc += 32) {
                     uint32_t ai[32];
                     tmem_ld32(lane_base + cc, ai);
                     tmem_ld_wait();
-                    if (p.dbg_y_int && m < p.M) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (n0 + cc + j < p.N) p.dbg_y_int[(size_t)m * p.N + n0 + cc + j] = (int)ai[j] - rs;
-                    }
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) ai[j] = __float_as_uint((float)((int)ai[j] - rs) * scale);
+                    dequant_chunk(cc, ai);
                     tmem_st32(lane_base + cc, ai);
                 }
                 tmem_st_wait();
                 tc_fence_before();
                 fence_proxy_async();  // the staged H and (g B)^T tiles
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_LORAREADY + b));
-                ok = mbar_wait(bar(BAR_LORADONE + b), par, abort_flag, status, 0x310u);
+                if (lane == 0) mbar_arrive(bar(BAR_LORAREADY));
+                ok = mbar_wait(bar(BAR_LORADONE), par, abort_flag, status, 0x310u);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;
                 tc_fence_after();
             }
 
-            for (int c0 = 0; c0 < TILE_N; c0 += COLS_PER_STORE) {
-                uint8_t *buf = stbuf + sbuf * STORE_BUF_BYTES;
-                // the buffer was handed to a TMA store two stores ago: wait until it was read
-                if (lane == 0) bulk_wait_read<1>();
+            // read the result, transpose it through shared memory (a thread holds one channel of 32
+            // tokens; y wants the channels of a token next to each other) and store with TMA
+            for (int cc = 0; cc < TILE_T; cc += 32) {
+                uint32_t ai[32];
+                tmem_ld32(lane_base + cc, ai);
+                tmem_ld_wait();
+                if (!has_lora) dequant_chunk(cc, ai);
+                // the buffer was handed to a TMA store one chunk ago: wait until it was read
+                if (lane == 0) bulk_wait_read<0>();
                 __syncwarp();
+                if (OUT_BF16) {
 #pragma unroll
-                for (int sub = 0; sub < COLS_PER_STORE / 32; ++sub) {
-                    const int cc = c0 + 32 * sub;
-                    uint32_t ai[32];
-                    tmem_ld32(lane_base + cc, ai);
-                    tmem_ld_wait();
-                    float yv[32];
-                    if (has_lora) {
+                    for (int j = 0; j < 32; ++j)
+                        reinterpret_cast<__nv_bfloat16 *>(buf)[j * 32 + lane] = __float2bfloat16_rn(__uint_as_float(ai[j]));
+                } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) yv[j] = __uint_as_float(ai[j]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            ai[j] = (uint32_t)((int)ai[j] - rs);
-                            yv[j] = (float)(int)ai[j] * scale;
-                        }
-                        if (p.dbg_y_int && m < p.M) {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (n0 + cc + j < p.N) p.dbg_y_int[(size_t)m * p.N + n0 + cc + j] = (int)ai[j];
-                        }
-                    }
-                    if (OUT_BF16) {
-#pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) {  // 8 bf16 per 16-byte chunk
-                            uint32_t w[4];
-#pragma unroll
-                            for (int h = 0; h < 4; ++h) {
-                                __nv_bfloat162 b2 = __floats2bfloat162_rn(yv[8 * ch + 2 * h], yv[8 * ch + 2 * h + 1]);
-                                w[h] = *reinterpret_cast<uint32_t *>(&b2);
-                            }
-                            const int chunk = 4 * sub + ch;
-                            *reinterpret_cast<uint4 *>(buf + lane * 128 + ((chunk ^ (lane & 7)) << 4)) =
-                                make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    } else {
-#pragma unroll
-                        for (int ch = 0; ch < 8; ++ch)  // 4 fp32 per 16-byte chunk
-                            *reinterpret_cast<uint4 *>(buf + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
-                                make_uint4(__float_as_uint(yv[4 * ch]), __float_as_uint(yv[4 * ch + 1]),
-                                           __float_as_uint(yv[4 * ch + 2]), __float_as_uint(yv[4 * ch + 3]));
-                    }
+                    for (int j = 0; j < 32; ++j) reinterpret_cast<uint32_t *>(buf)[j * 32 + lane] = ai[j];
                 }
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_2d(&tmap_y, n0 + c0, m0 + 32 * q, smem_u32(buf));
+                    tma_store_2d(&tmap_y, c0 + 32 * q, t0 + cc, smem_u32(buf));
                     bulk_commit();
                 }
-                sbuf ^= 1;
             }
-            // all TMEM reads of this tile are done: hand the accumulator back to the MMA warp
+            // all tensor-memory reads of this tile are done: hand the accumulator back to the MMA warp
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_ACCEMPTY + b));
+            if (lane == 0) mbar_arrive(bar(BAR_ACCEMPTY));
         }
         if (lane == 0) bulk_wait_read<0>();
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ unpack warps
-        const int ut = tid - 6 * 32;  // 0..127
-        int s = 0, u = 0;
-        uint32_t ph = 0, bph = 0;
+        const int q = warp & 3;              // tensor-memory lane quarter this warp may access
+        const int row = 32 * q + lane;       // this thread's channel row of the tile = its tensor-memory lane
+        int s = 0;
+        uint32_t ph = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < kblocks; ++kb) {
-                ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag, status, 0x400u + s) &&
-                     mbar_wait(bar(BAR_BEMPTY + u), bph ^ 1u, abort_flag, status, 0x410u + u);
+                // FULL also tells that the MMAs that read this stage's previous contents are complete
+                // (their commit was one of the arrivals the producer waited for before refilling it)
+                ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag, status, 0x400u + s);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
-                const uint8_t *psrc = smem + OFF_P + s * P_TILE_BYTES;
-                uint8_t *bdst = smem + OFF_B + u * B_TILE_BYTES;
+                const uint8_t *prow = smem + OFF_P + s * P_TILE_BYTES + row * 32;  // 128 codes of this row
+                const uint4 lo = *reinterpret_cast<const uint4 *>(prow), hi = *reinterpret_cast<const uint4 *>(prow + 16);
+                const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+                uint32_t a[32];  // register 4 i + j = columns 16 i + 4 j .. + 3 of the k block, one code per byte
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int idx = i * 128 + ut;          // 16-byte piece of the packed tile
-                    const int row = idx >> 1, half = idx & 1;  // 32 packed bytes per row
-                    const uint4 pk = *reinterpret_cast<const uint4 *>(psrc + idx * 16);
-                    const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
+                for (int i = 0; i < 8; ++i)
 #pragma unroll
-                    for (int qd = 0; qd < 4; ++qd) {
-                        // word qd holds 16 consecutive k; (w >> 2 j) & 0x03030303 = k 4 j .. 4 j + 3
-                        const uint4 o = make_uint4(w[qd] & 0x03030303u, (w[qd] >> 2) & 0x03030303u,
-                                                   (w[qd] >> 4) & 0x03030303u, (w[qd] >> 6) & 0x03030303u);
-                        const int chunk = 4 * half + qd;
-                        *reinterpret_cast<uint4 *>(bdst + row * 128 + ((chunk ^ (row & 7)) << 4)) = o;
-                    }
-                }
-                fence_proxy_async();
+                    for (int j = 0; j < 4; ++j) a[4 * i + j] = (w[i] >> (2 * j)) & 0x03030303u;
+                tmem_st32(tmem_base + ((uint32_t)(32 * q) << 16) + A_COL + s * A_STAGE_COLS, a);
+                tmem_st_wait();
+                tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(bar(BAR_BFULL + u));
+                    mbar_arrive(bar(BAR_AFULL + s));
                     mbar_arrive(bar(BAR_EMPTY + s));
                 }
-                if (++s == XSTAGES) { s = 0; ph ^= 1u; }
-                if (++u == BSTAGES) { u = 0; bph ^= 1u; }
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
         }
     }
@@ -561,7 +540,7 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
     }
     const bool bf16 = (p.flags & HGF_FLAG_OUT_BF16) != 0;
     CUtensorMap mx, mw, my;
-    if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.xq, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.K, KBLK, TILE_M,
+    if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.xq, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.K, KBLK, TILE_T,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;
     {   // packed weights as a 4-D byte tensor: (byte in row: 64, row in tile: 16, column tile, row tile)
@@ -570,7 +549,7 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
         const uint64_t steps = (uint64_t)padded_k(p.K) / 256;
         cuuint64_t dims[4] = {64, 16, steps, (uint64_t)row_tiles(p.N)};
         cuuint64_t strides[3] = {64, 1024, steps * 1024};
-        cuuint32_t box[4] = {KBLK / 4, 16, 1, TILE_N / 16};
+        cuuint32_t box[4] = {KBLK / 4, 16, 1, TILE_C / 16};
         cuuint32_t estr[4] = {1, 1, 1, 1};
         if (fn(&mw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<uint8_t *>(p.packed), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -578,9 +557,9 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
             return cudaErrorInvalidValue;
     }
     if (!make_map_2d(&my, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, p.y, (uint64_t)p.N,
-                     (uint64_t)p.M, (uint64_t)p.N * (bf16 ? 2 : 4), bf16 ? 64 : 32, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+                     (uint64_t)p.M, (uint64_t)p.N * (bf16 ? 2 : 4), 32, 32, CU_TENSOR_MAP_SWIZZLE_NONE))
         return cudaErrorInvalidValue;
-    const int tiles = ((p.M + TILE_M - 1) / TILE_M) * ((p.N + TILE_N - 1) / TILE_N);
+    const int tiles = ((p.M + TILE_T - 1) / TILE_T) * ((p.N + TILE_C - 1) / TILE_C);
     const int grid = tiles < sm_count ? tiles : sm_count;
     unsigned int *status = device_status_word();
     if (!status) return cudaErrorMemoryAllocation;
