@@ -44,9 +44,8 @@ static bool takes_gemm_path(int64_t M, int64_t d_in, uint32_t flags) {
 using namespace hgf;
 
 extern "C" size_t hgf_workspace_bytes(int64_t M, int64_t d_in, int64_t d_out, int32_t r, uint32_t flags) {
-    (void)d_out;
     if (M <= 0 || d_in <= 0 || d_in > 65536 || r < 0) return 256;
-    return ws_layout(M, d_in, r, takes_gemm_path(M, d_in, flags)).total;
+    return ws_layout(M, d_in, d_out, r, takes_gemm_path(M, d_in, flags)).total;
 }
 
 extern "C" hgf_status hgf_act_quant(const void *x, int64_t M, int64_t d_in, int8_t *xq, float *gamma_x,
@@ -98,6 +97,12 @@ static void fill_params(const void *x, int64_t M, const void *packed, float gamm
     pp->h_hi = gemm ? nullptr : (__half *)(ws + L.h_hi);
     pp->h_lo = gemm ? nullptr : (__half *)(ws + L.h_lo);
     pp->h16 = gemm ? (__half *)(ws + L.h16) : nullptr;
+    pp->tok_sc = gemm ? (float *)(ws + L.tok_sc) : nullptr;
+    pp->gb16 = (gemm && r) ? (__half *)(ws + L.gb16) : nullptr;
+    pp->Bt = (const __half *)Bt;
+    pp->gate = gate;
+    pp->gw_over_127 = (float)((double)gamma / 127.0);
+    pp->N = (int)d_out;
     pp->dbg_xq = dbg ? dbg->xq : nullptr;
     pp->dbg_gamma_x = dbg ? dbg->gamma_x : nullptr;
     pp->dbg_h = (dbg && r) ? dbg->h : nullptr;
@@ -139,7 +144,7 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
     if (st != HGF_OK) return st;
     if (dbg && (misaligned(dbg->xq) || misaligned(dbg->gamma_x) || misaligned(dbg->y_int) || misaligned(dbg->h)))
         return HGF_ERR_MISALIGNED;
-    const WsLayout L = ws_layout(M, d_in, r, gemm);
+    const WsLayout L = ws_layout(M, d_in, d_out, r, gemm);
     if (!workspace || workspace_bytes < L.total) return HGF_ERR_WORKSPACE;
     if (((uintptr_t)workspace) & 255u) return HGF_ERR_MISALIGNED;
     cudaStream_t stream = (cudaStream_t)stream_;
@@ -169,8 +174,8 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
     gp.gamma_x = pp.gamma_x;
     gp.row_sum = pp.row_sum;
     gp.h16 = pp.h16;
-    gp.Bt = (const __half *)Bt;
-    gp.gate = gate;
+    gp.tok_sc = pp.tok_sc;
+    gp.gb16 = pp.gb16;
     gp.y = y;
     gp.dbg_y_int = dbg ? dbg->y_int : nullptr;
     gp.gw_over_127 = dp.gw_over_127;
@@ -210,7 +215,7 @@ extern "C" hgf_status hgf_linear_forward_static(const void *x, int64_t M, const 
     if (flags & HGF_FLAG_FORCE_GEMM) return HGF_ERR_INVALID_ARG;
     if (d_in % 64 != 0 || d_in > 65536 || M > HGF_DECODE_MAX_M) return HGF_ERR_UNSUPPORTED_SHAPE;
     const int32_t r_eff = (At && Bt && gate) ? r : 0;
-    if (ws_layout(M, d_in, r_eff, false).total > (size_t)HGF_STATIC_SCRATCH_BYTES) return HGF_ERR_TOO_LARGE;
+    if (ws_layout(M, d_in, d_out, r_eff, false).total > (size_t)HGF_STATIC_SCRATCH_BYTES) return HGF_ERR_TOO_LARGE;
     if (takes_gemm_path(M, d_in, flags)) return HGF_ERR_UNSUPPORTED_SHAPE;
     void *scratch = static_scratch_address();
     if (!scratch) return HGF_ERR_CUDA;
@@ -254,7 +259,7 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         if (st != HGF_OK) return st;
         if (gemm) return HGF_ERR_UNSUPPORTED_SHAPE;  // groups hold decode-sized problems only
         ranks[i] = r;
-        lay[i] = ws_layout(q.M, q.d_in, r, false);
+        lay[i] = ws_layout(q.M, q.d_in, q.d_out, r, false);
         ws_total += lay[i].total;
         if (tiles > (1 << 30) - (1 << 21)) return HGF_ERR_UNSUPPORTED_SHAPE;
     }

@@ -35,23 +35,30 @@ static inline int64_t row_tiles(int64_t d_out) { return (d_out + 15) / 16; }
 //   h_hi     [M][r]      half     fp16 rounding of h          (decode path only)
 //   h_lo     [M][r]      half     fp16 rounding of h - h_hi   (decode path only)
 //   h16      [M][64]     half     h in fp16, zero-padded to 64 columns (GEMM path only)
+//   tok_sc   [M]         float    gamma_x[m] * gamma_W / 127 (GEMM path only)
+//   gb16     [N][64]     half     gate[n] * B[j][n], zero-padded to 64 columns (GEMM path only)
+// On the GEMM path the per-token arrays have room for M rounded up to 128: the kernel fetches them
+// 128 tokens at a time (what lies past M is never used).
 struct WsLayout {
-    size_t xq, gamma_x, row_sum, h, h_hi, h_lo, h16, total;
+    size_t xq, gamma_x, row_sum, h, h_hi, h_lo, h16, tok_sc, gb16, total;
 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-static inline WsLayout ws_layout(int64_t M, int64_t d_in, int32_t r, bool gemm_path) {
+static inline WsLayout ws_layout(int64_t M, int64_t d_in, int64_t d_out, int32_t r, bool gemm_path) {
     WsLayout L;
     size_t off = 0;
     const size_t rr = (size_t)(r > 0 ? r : 1);
     L.xq = off;      off += align_up((size_t)M * (size_t)d_in, 256);
     L.gamma_x = off; off += align_up((size_t)M * 4, 256);
-    L.row_sum = off; off += align_up((size_t)M * 4, 256);
+    const size_t Mp = gemm_path ? align_up((size_t)M, 128) : (size_t)M;
+    L.row_sum = off; off += align_up(Mp * 4, 256);
     L.h = off;       off += align_up((size_t)M * rr * 4, 256);
     L.h_hi = off;    off += gemm_path ? 0 : align_up((size_t)M * rr * 2, 256);
     L.h_lo = off;    off += gemm_path ? 0 : align_up((size_t)M * rr * 2, 256);
     L.h16 = off;     off += gemm_path ? align_up((size_t)M * 64 * 2, 256) : 0;
+    L.tok_sc = off;  off += gemm_path ? align_up(Mp * 4, 256) : 0;
+    L.gb16 = off;    off += (gemm_path && r > 0) ? align_up((size_t)d_out * 64 * 2, 256) : 0;
     L.total = off ? off : 256;
     return L;
 }
@@ -66,6 +73,12 @@ struct PrologueParams {
     float *h;                // [M][r]
     __half *h_hi, *h_lo;     // [M][r] each (decode path) or null
     __half *h16;             // [M][64] (GEMM path) or null
+    float *tok_sc;           // [M] gamma_x * gamma_W / 127 (GEMM path) or null
+    __half *gb16;            // [N][64] gate * B^T (GEMM path) or null
+    const __half *Bt;        // [N][r]  (GEMM path, for gb16)
+    const float *gate;       // [N]     (GEMM path, for gb16)
+    float gw_over_127;
+    int N;
     int8_t *dbg_xq;          // nullable debug copies
     float *dbg_gamma_x;
     float *dbg_h;
@@ -145,8 +158,8 @@ struct GemmParams {
     const float *gamma_x;    // [M]
     const int32_t *row_sum;  // [M]
     const __half *h16;       // [M][64]
-    const __half *Bt;        // [N][r]
-    const float *gate;       // [N]
+    const float *tok_sc;     // [M] (room for M rounded up to 128)
+    const __half *gb16;      // [N][64]
     void *y;                 // [M][N]
     int32_t *dbg_y_int;
     float gw_over_127;

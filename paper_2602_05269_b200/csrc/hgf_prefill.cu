@@ -10,14 +10,17 @@
 // registers (one 128-channel row per thread: a shift and a mask per register) and store it with one
 // tcgen05.st into the operand's place in tensor memory, so shared memory carries only the int8
 // activation tile (TMA in, MMA out) and the packed codes.  The output tile is therefore
-// 128 output channels (tensor-memory lanes, MMA M) x 256 tokens (columns, MMA N).
+// 128 output channels (tensor-memory lanes, MMA M) x 128 tokens (columns, MMA N); two accumulators
+// alternate, so the epilogue of a tile runs under the main loop of the next, and eight pipeline
+// stages cover the latency of the load -> expand -> MMA -> release round trip.
 //
 // One persistent CTA per SM, 10 warps with fixed roles:
-//   warp 0      TMA producer: per 128-wide k block the int8 activation tile (256 tokens x 128 B,
-//               128-byte swizzle) and the packed weight tile (128 rows x 32 B, gathered from 8
-//               consecutive row tiles of the tiled weight layout)
+//   warp 0      TMA producer: per 128-wide k block the int8 activation tile (128 tokens x 128 B,
+//               128-byte swizzle), per two k blocks the packed weights of 128 channels (eight
+//               contiguous 1 KiB tiles of the tiled weight layout, one bulk copy each), and per tile
+//               what its epilogue needs: row sums, scales, the H tile and the (g B)^T tile
 //   warp 1      allocates tensor memory; one lane issues the MMAs and commits to mbarriers
-//   warps 2-5   epilogue: stage the correction's operands, dequantise the accumulator in place
+//   warps 2-5   epilogue: dequantise the accumulator in place
 //               (tcgen05.ld / tcgen05.st), wait for the correction MMA, read the result, transpose it
 //               through shared memory and store y with TMA
 //   warps 6-9   expand the packed tile into tensor memory
@@ -34,33 +37,38 @@
 namespace hgf {
 
 constexpr int TILE_C = 128;   // output channels per tile (MMA M, tensor-memory lanes)
-constexpr int TILE_T = 256;   // tokens per tile (MMA N, accumulator columns)
+constexpr int TILE_T = 128;   // tokens per tile (MMA N, accumulator columns)
 constexpr int KBLK = 128;
-constexpr int STAGES = 4;
-constexpr int X_TILE_BYTES = TILE_T * KBLK;      // 32 KiB
-constexpr int P_TILE_BYTES = TILE_C * KBLK / 4;  // 4 KiB
-constexpr int LORA_H_BYTES = TILE_T * 128;       // 256 tokens x 64 fp16
+constexpr int STAGES = 6;      // activation tiles in shared memory and weight operands in tensor memory
+constexpr int X_TILE_BYTES = TILE_T * KBLK;      // 16 KiB
+constexpr int PSTAGES = 4;
+constexpr int P_TILE_BYTES = TILE_C * 256 / 4;   // 8 KiB: 8 weight tiles of 16 rows x 256 columns, i.e. two k blocks
+constexpr int LORA_H_BYTES = TILE_T * 128;       // 128 tokens x 64 fp16
 constexpr int LORA_B_BYTES = TILE_C * 128;       // 128 channels x 64 fp16
-constexpr int TOKV_BYTES = TILE_T * 8;           // per epilogue warp: row sum and scale of the tile's tokens
+constexpr int TOKV_BYTES = TILE_T * 8;           // row sums and scales of the tile's tokens
 constexpr int STORE_BUF_BYTES = 32 * 32 * 4;     // per epilogue warp: 32 tokens x 32 channels
 constexpr int GEMM_THREADS = 320;
-constexpr int TMEM_COLS = 512, ACC_COL = 0, A_COL = 256, A_STAGE_COLS = KBLK / 4;  // 32 columns = 128 int8 per lane
+// tensor memory: two accumulators of 128 columns, then STAGES weight operands of 32 columns (= 128 int8 per lane)
+constexpr int TMEM_COLS = 512, ACC_COLS = TILE_T, A_COL = 2 * ACC_COLS, A_STAGE_COLS = KBLK / 4;
+static_assert(A_COL + STAGES * A_STAGE_COLS <= TMEM_COLS, "tensor memory budget");
 
 constexpr int OFF_X = 0;
 constexpr int OFF_LH = OFF_X + STAGES * X_TILE_BYTES;
-constexpr int OFF_LB = OFF_LH + LORA_H_BYTES;
-constexpr int OFF_P = OFF_LB + LORA_B_BYTES;
-constexpr int OFF_TOKV = OFF_P + STAGES * P_TILE_BYTES;
-constexpr int OFF_ST = OFF_TOKV + 4 * TOKV_BYTES;
+constexpr int OFF_LB = OFF_LH + 2 * LORA_H_BYTES;   // the epilogue's operands are double-buffered like the accumulators
+constexpr int OFF_P = OFF_LB + 2 * LORA_B_BYTES;
+constexpr int OFF_TOKV = OFF_P + PSTAGES * P_TILE_BYTES;
+constexpr int OFF_ST = OFF_TOKV + 2 * TOKV_BYTES;
 constexpr int OFF_BAR = OFF_ST + 4 * STORE_BUF_BYTES;
-static_assert(OFF_BAR + 256 + 1024 <= 227 * 1024, "shared memory budget");
-constexpr int SMEM_USED = OFF_BAR + 256;
+static_assert(OFF_BAR + 512 + 1024 <= 227 * 1024, "shared memory budget");
+constexpr int SMEM_USED = OFF_BAR + 512;
 constexpr int SMEM_BYTES = SMEM_USED + 1024;  // slack for the 1024-byte alignment of the base
 
 // barrier slots (8 bytes each) inside the OFF_BAR block
-enum { BAR_FULL = 0, BAR_EMPTY = BAR_FULL + STAGES, BAR_AFULL = BAR_EMPTY + STAGES, BAR_ACCFULL = BAR_AFULL + STAGES,
-       BAR_ACCEMPTY, BAR_LORAREADY, BAR_LORADONE, BAR_COUNT };
-static_assert(BAR_COUNT * 8 + 16 <= 256, "barrier block too small");
+enum { BAR_FULL = 0, BAR_EMPTY = BAR_FULL + STAGES,
+       BAR_PFULL = BAR_EMPTY + STAGES, BAR_PEMPTY = BAR_PFULL + PSTAGES, BAR_ACCFULL = BAR_PEMPTY + PSTAGES,
+       BAR_ACCEMPTY = BAR_ACCFULL + 2, BAR_LORAREADY = BAR_ACCEMPTY + 2, BAR_LORADONE = BAR_LORAREADY + 2,
+       BAR_OPSFULL = BAR_LORADONE + 2, BAR_OPSEMPTY = BAR_OPSFULL + 2, BAR_COUNT = BAR_OPSEMPTY + 2 };
+static_assert(BAR_COUNT * 8 + 16 <= 512, "barrier block too small");
 
 constexpr uint32_t kSpinLimit = 1u << 22;            // polls of a drain loop
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // bounded waits give up after two seconds
@@ -129,6 +137,12 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
+}
+// Untiled bulk copy global -> shared (addresses 16-byte aligned, size a multiple of 16), completing on the mbarrier.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int x, int y, uint32_t src) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];\n"
@@ -213,8 +227,9 @@ constexpr uint32_t IDESC_F16 = (1u << 4) /*f32*/ | (0u << 7) /*A f16*/ | (0u << 
 
 template <bool OUT_BF16>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                    const __grid_constant__ CUtensorMap tmap_y, const GemmParams p, unsigned int *status) {
+prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_h,
+                    const __grid_constant__ CUtensorMap tmap_gb, const __grid_constant__ CUtensorMap tmap_y,
+                    const GemmParams p, unsigned int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -222,6 +237,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     auto bar = [&](int i) { return bar0 + 8u * i; };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + OFF_BAR + BAR_COUNT * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_BAR + BAR_COUNT * 8 + 4);
+    static_assert(TILE_T == 128, "the epilogue's staging loops are written for 128-token tiles");
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int tiles_t = (p.M + TILE_T - 1) / TILE_T, tiles_c = (p.N + TILE_C - 1) / TILE_C;
@@ -231,14 +247,26 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(bar(BAR_FULL + s), 1);
-            mbar_init(bar(BAR_EMPTY + s), 1 + 4);  // MMA commit (activations read) + four unpack warps (codes read)
-            mbar_init(bar(BAR_AFULL + s), 4);
+            // FULL: the activation tile has landed (producer's arrival + its bytes) and the four unpack warps
+            // have put the weight operand into tensor memory.  EMPTY: the MMAs that read both are complete
+            // (one commit; the producer and the unpack warps both wait on it).  One barrier each way keeps
+            // the MMA thread's loop short: it is a single thread and every barrier operation costs it a
+            // shared-memory round trip.
+            mbar_init(bar(BAR_FULL + s), 1 + 4);
+            mbar_init(bar(BAR_EMPTY + s), 1);
         }
-        mbar_init(bar(BAR_ACCFULL), 1);
-        mbar_init(bar(BAR_ACCEMPTY), 4);
-        mbar_init(bar(BAR_LORAREADY), 4);
-        mbar_init(bar(BAR_LORADONE), 1);
+        for (int j = 0; j < PSTAGES; ++j) {
+            mbar_init(bar(BAR_PFULL + j), 1);
+            mbar_init(bar(BAR_PEMPTY + j), 4);  // four unpack warps: the packed codes have been read
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(BAR_ACCFULL + b), 1);
+            mbar_init(bar(BAR_ACCEMPTY + b), 4);
+            mbar_init(bar(BAR_LORAREADY + b), 4);
+            mbar_init(bar(BAR_LORADONE + b), 1);
+            mbar_init(bar(BAR_OPSFULL + b), 1);
+            mbar_init(bar(BAR_OPSEMPTY + b), 4);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         fence_proxy_async();
@@ -256,128 +284,164 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
-            uint32_t issued[STAGES] = {0, 0, 0, 0};
+        // The whole warp walks the loop (a single thread issuing ten copies per two k blocks, each
+        // with its address arithmetic, cannot keep up with the MMAs): every lane polls the barriers,
+        // lane 0 posts the byte counts and the activation tile, lanes 0-7 one weight tile each.
+        {
+            int s = 0, pj = 0;
+            uint32_t ph = 0, pph = 0;
+            uint32_t issued[STAGES] = {}, pissued[PSTAGES] = {}, ops_issued[2] = {};
+            int pit = 0;
             bool ok = true;
+            const int steps = (p.K + 255) >> 8, n_row_tiles = (p.N + 15) >> 4;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                 const int t0 = (tile % tiles_t) * TILE_T, c0 = (tile / tiles_t) * TILE_C;
+                const int rt0 = c0 >> 4, nrt = n_row_tiles - rt0 < TILE_C / 16 ? n_row_tiles - rt0 : TILE_C / 16;
+                // this lane's weight tile of column tile 0 (row tiles past the matrix are left out)
+                const uint8_t *psrc = p.packed + (size_t)(rt0 + (lane < nrt ? lane : 0)) * steps * 1024;
+                {
+                    // what the tile's epilogue needs, into the buffer of the tile's accumulator: row sums and
+                    // scales of the 128 tokens, and with a correction the H tile and the (g B)^T tile
+                    const int b = pit & 1;
+                    ok = mbar_wait(bar(BAR_OPSEMPTY + b), ((uint32_t)(pit >> 1) & 1u) ^ 1u, abort_flag, status, 0x120u + b);
+                    if (!(ok = __all_sync(0xffffffffu, ok))) break;
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(bar(BAR_OPSFULL + b), 2u * TILE_T * 4u + (has_lora ? LORA_H_BYTES + LORA_B_BYTES : 0));
+                        bulk_load_1d(sbase + OFF_TOKV + b * TOKV_BYTES, p.row_sum + t0, TILE_T * 4u, bar(BAR_OPSFULL + b));
+                        bulk_load_1d(sbase + OFF_TOKV + b * TOKV_BYTES + TILE_T * 4, p.tok_sc + t0, TILE_T * 4u, bar(BAR_OPSFULL + b));
+                        if (has_lora) {
+                            tma_load_2d(sbase + OFF_LH + b * LORA_H_BYTES, &tmap_h, 0, t0, bar(BAR_OPSFULL + b));
+                            tma_load_2d(sbase + OFF_LB + b * LORA_B_BYTES, &tmap_gb, 0, c0, bar(BAR_OPSFULL + b));
+                        }
+                    }
+                    ++ops_issued[b];
+                    ++pit;
+                }
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!(ok = mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x100u + s))) break;
-                    mbar_arrive_expect_tx(bar(BAR_FULL + s), X_TILE_BYTES + P_TILE_BYTES);
-                    tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, t0, bar(BAR_FULL + s));
-                    // packed weights: bytes 32 (kb % 2) .. + 31 of the 16 rows of column tile kb / 2, for 8 row tiles
-                    tma_load_4d(sbase + OFF_P + s * P_TILE_BYTES, &tmap_w, (kb & 1) * 32, 0, kb >> 1, c0 >> 4,
-                                bar(BAR_FULL + s));
+                    if ((kb & 1) == 0) {
+                        // packed weights of two k blocks: the 1 KiB tiles (16 rows x 256 columns) of 8 consecutive
+                        // row tiles, each one contiguous in memory
+                        ok = mbar_wait(bar(BAR_PEMPTY + pj), pph ^ 1u, abort_flag, status, 0x110u + pj);
+                        if (!(ok = __all_sync(0xffffffffu, ok))) break;
+                        if (lane == 0) mbar_arrive_expect_tx(bar(BAR_PFULL + pj), (uint32_t)nrt * 1024u);
+                        __syncwarp();
+                        if (lane < nrt)
+                            bulk_load_1d(sbase + OFF_P + pj * P_TILE_BYTES + lane * 1024, psrc + (size_t)(kb >> 1) * 1024, 1024u,
+                                         bar(BAR_PFULL + pj));
+                        ++pissued[pj];
+                        if (++pj == PSTAGES) { pj = 0; pph ^= 1u; }
+                    }
+                    ok = mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x100u + s);
+                    if (!(ok = __all_sync(0xffffffffu, ok))) break;
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(bar(BAR_FULL + s), X_TILE_BYTES);
+                        tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, t0, bar(BAR_FULL + s));
+                    }
                     ++issued[s];
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
-            // drain: wait (bounded) until every copy this thread issued has landed, so that the CTA
+            // drain: wait (bounded) until every copy this warp issued has landed, so that the CTA
             // never exits with a bulk copy in flight (immediate when the consumers ran to the end)
             for (int q = 0; q < STAGES; ++q)
                 if (issued[q]) {
                     const uint32_t par = (issued[q] - 1u) & 1u;
                     for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_FULL + q), par); ++i) {}
                 }
+            for (int q = 0; q < PSTAGES; ++q)
+                if (pissued[q]) {
+                    const uint32_t par = (pissued[q] - 1u) & 1u;
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_PFULL + q), par); ++i) {}
+                }
+            for (int q = 0; q < 2; ++q)
+                if (ops_issued[q]) {
+                    const uint32_t par = (ops_issued[q] - 1u) & 1u;
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_OPSFULL + q), par); ++i) {}
+                }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
+        // Tile `it` accumulates into accumulator it % 2, so the epilogue of one tile runs under the main
+        // loop of the next.  With a correction, the epilogue first rewrites the accumulator as fp32
+        // (dequantised), then this thread adds (g B) H^T onto it with one more MMA, slipped in between
+        // the k blocks of the tile in progress as soon as the epilogue is ready for it.
         if (lane == 0) {
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
-            int it = 0;
+            int it = 0, pend = -1;  // pend: tile whose correction MMA is still to be issued
+            const uint64_t xdesc0 = make_sw128_desc(sbase + OFF_X);
+            auto issue_lora = [&](int t) {
+                const int b = t & 1;
+                tc_fence_after();
+                const uint64_t adesc = make_sw128_desc(sbase + OFF_LB + b * LORA_B_BYTES);
+                const uint64_t bdesc = make_sw128_desc(sbase + OFF_LH + b * LORA_H_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)  // 64 fp16 = 4 x (K = 16), on top of the fp32 values
+                    mma_f16(tmem_base + b * ACC_COLS, adesc + 2u * kk, bdesc + 2u * kk, IDESC_F16, 1u);
+                tc_commit(bar(BAR_LORADONE + b));
+            };
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-                if (it > 0 && !(ok = mbar_wait(bar(BAR_ACCEMPTY), (uint32_t)(it - 1) & 1u, abort_flag, status, 0x200u)))
+                const int b = it & 1;
+                const uint32_t acc = tmem_base + b * ACC_COLS;
+                if (it >= 2 && !(ok = mbar_wait(bar(BAR_ACCEMPTY + b), (uint32_t)((it >> 1) - 1) & 1u, abort_flag, status, 0x200u)))
                     break;
                 tc_fence_after();
                 for (int kb = 0; kb < kblocks; ++kb) {
+                    if (pend >= 0 && mbar_try_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u)) {
+                        issue_lora(pend);
+                        pend = -1;
+                    }
                     if (!(ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag, status, 0x210u + s))) break;
-                    if (!(ok = mbar_wait(bar(BAR_AFULL + s), ph, abort_flag, status, 0x220u + s))) break;
                     tc_fence_after();
-                    const uint64_t bdesc = make_sw128_desc(sbase + OFF_X + s * X_TILE_BYTES);
+                    const uint64_t bdesc = xdesc0 + (uint64_t)(s * (X_TILE_BYTES >> 4));
                     const uint32_t a_tmem = tmem_base + A_COL + s * A_STAGE_COLS;
-#pragma unroll
-                    for (int kk = 0; kk < KBLK / 32; ++kk)  // 32 int8 = 8 columns of the weight operand, 32 bytes of a token row
-                        mma_i8_ts(tmem_base + ACC_COL, a_tmem + 8u * kk, bdesc + 2u * kk, IDESC_I8, (kb | kk) ? 1u : 0u);
+                    // 32 int8 = 8 columns of the weight operand, 32 bytes of a token row
+                    mma_i8_ts(acc, a_tmem, bdesc, IDESC_I8, kb ? 1u : 0u);
+                    mma_i8_ts(acc, a_tmem + 8u, bdesc + 2u, IDESC_I8, 1u);
+                    mma_i8_ts(acc, a_tmem + 16u, bdesc + 4u, IDESC_I8, 1u);
+                    mma_i8_ts(acc, a_tmem + 24u, bdesc + 6u, IDESC_I8, 1u);
                     tc_commit(bar(BAR_EMPTY + s));
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit(bar(BAR_ACCFULL));
-                if (has_lora) {
-                    // the epilogue has rewritten the accumulator as fp32: add (g B) H^T on top
-                    if (!(ok = mbar_wait(bar(BAR_LORAREADY), (uint32_t)it & 1u, abort_flag, status, 0x230u))) break;
-                    tc_fence_after();
-                    const uint64_t adesc = make_sw128_desc(sbase + OFF_LB);
-                    const uint64_t bdesc = make_sw128_desc(sbase + OFF_LH);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)  // 64 fp16 = 4 x (K = 16)
-                        mma_f16(tmem_base + ACC_COL, adesc + 2u * kk, bdesc + 2u * kk, IDESC_F16, 1u);
-                    tc_commit(bar(BAR_LORADONE));
+                tc_commit(bar(BAR_ACCFULL + b));
+                if (pend >= 0) {  // the previous tile's correction has to be out before its accumulator's next turn
+                    if (!(ok = mbar_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x230u)))
+                        break;
+                    issue_lora(pend);
+                    pend = -1;
                 }
+                if (has_lora) pend = it;
             }
+            if (ok && pend >= 0 &&
+                mbar_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x231u))
+                issue_lora(pend);
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------------ epilogue warps
         const int e = warp - 2;          // staging role index
         const int q = warp & 3;          // tensor-memory lane quarter this warp may access
-        int *tok_rs = reinterpret_cast<int *>(smem + OFF_TOKV + e * TOKV_BYTES);
-        float *tok_sc = reinterpret_cast<float *>(tok_rs + TILE_T);
-        const float gw = p.gw_over_127;
         uint8_t *buf = smem + OFF_ST + e * STORE_BUF_BYTES;
         bool ok = true;
         int it = 0;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
             const int t0 = (tile % tiles_t) * TILE_T, c0 = (tile / tiles_t) * TILE_C;
-            const uint32_t par = (uint32_t)it & 1u;
-            // this warp's copy of the tile's per-token values
-#pragma unroll
-            for (int i = 0; i < TILE_T / 32; ++i) {
-                const int tl = 32 * i + lane, m = t0 + tl;
-                tok_rs[tl] = m < p.M ? p.row_sum[m] : 0;
-                tok_sc[tl] = m < p.M ? p.gamma_x[m] * gw : 0.0f;
-            }
-            if (has_lora) {
-                // (the previous tile's correction MMA has finished reading these buffers: this warp waited
-                // for it before its second pass)
-                // H tile: token rows 64 e .. 64 e + 63, 8 chunks of 16 bytes each
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int idx = i * 32 + lane, row = 64 * e + idx / 8, c = idx % 8, m = t0 + row;
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (m < p.M) v = *reinterpret_cast<const uint4 *>(p.h16 + (size_t)m * 64 + c * 8);
-                    *reinterpret_cast<uint4 *>(smem + OFF_LH + row * 128 + ((c ^ (row & 7)) << 4)) = v;
-                }
-                // (g B)^T tile: channel rows 32 e .. 32 e + 31, each row of B^T scaled by its channel's gate
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int idx = i * 32 + lane, row = 32 * e + idx / 8, c = idx % 8, n = c0 + row;
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (n < p.N && c * 8 < p.r) {
-                        v = *reinterpret_cast<const uint4 *>(p.Bt + (size_t)n * p.r + c * 8);
-                        const float g = p.gate[n];
-                        __half2 *h2 = reinterpret_cast<__half2 *>(&v);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const float2 f = __half22float2(h2[k]);
-                            h2[k] = __floats2half2_rn(g * f.x, g * f.y);
-                        }
-                    }
-                    *reinterpret_cast<uint4 *>(smem + OFF_LB + row * 128 + ((c ^ (row & 7)) << 4)) = v;
-                }
-            }
-            __syncwarp();
+            const int b = it & 1;
+            const uint32_t par = (uint32_t)(it >> 1) & 1u;
+            // the tile's row sums and scales (and the correction's operands) were fetched by the producer
+            const int *tok_rs = reinterpret_cast<const int *>(smem + OFF_TOKV + b * TOKV_BYTES);
+            const float *tok_sc = reinterpret_cast<const float *>(tok_rs + TILE_T);
+            ok = mbar_wait(bar(BAR_OPSFULL + b), par, abort_flag, status, 0x320u + b);
+            if (!(ok = __all_sync(0xffffffffu, ok))) break;
 
             const int n = c0 + 32 * q + lane;  // this thread's output channel = its tensor-memory lane
             const bool n_ok = n < p.N;
 
-            ok = mbar_wait(bar(BAR_ACCFULL), par, abort_flag, status, 0x300u);
+            ok = mbar_wait(bar(BAR_ACCFULL + b), par, abort_flag, status, 0x300u);
             if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
             tc_fence_after();
-            const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16) + ACC_COL;
+            const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16) + b * ACC_COLS;
 
             // (the per-token values are read as vectors ahead of the arithmetic: a shared-memory load per
             // element in the dependent chain costs its full latency every time)
@@ -408,10 +472,9 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
                 tmem_st_wait();
                 tc_fence_before();
-                fence_proxy_async();  // the staged H and (g B)^T tiles
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_LORAREADY));
-                ok = mbar_wait(bar(BAR_LORADONE), par, abort_flag, status, 0x310u);
+                if (lane == 0) mbar_arrive(bar(BAR_LORAREADY + b));
+                ok = mbar_wait(bar(BAR_LORADONE + b), par, abort_flag, status, 0x310u);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;
                 tc_fence_after();
             }
@@ -444,7 +507,10 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             // all tensor-memory reads of this tile are done: hand the accumulator back to the MMA warp
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_ACCEMPTY));
+            if (lane == 0) {
+                mbar_arrive(bar(BAR_ACCEMPTY + b));
+                mbar_arrive(bar(BAR_OPSEMPTY + b));
+            }
         }
         if (lane == 0) bulk_wait_read<0>();
         __syncwarp();
@@ -452,16 +518,18 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         // ------------------------------------------------------------------ unpack warps
         const int q = warp & 3;              // tensor-memory lane quarter this warp may access
         const int row = 32 * q + lane;       // this thread's channel row of the tile = its tensor-memory lane
-        int s = 0;
-        uint32_t ph = 0;
+        int s = 0, pj = 0;
+        uint32_t ph = 0, pph = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < kblocks; ++kb) {
-                // FULL also tells that the MMAs that read this stage's previous contents are complete
-                // (their commit was one of the arrivals the producer waited for before refilling it)
-                ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag, status, 0x400u + s);
+                // the packed codes of this k block have landed, and the MMAs that read this stage's previous
+                // operand are complete
+                ok = mbar_wait(bar(BAR_PFULL + pj), pph, abort_flag, status, 0x400u + pj) &&
+                     mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x410u + s);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
-                const uint8_t *prow = smem + OFF_P + s * P_TILE_BYTES + row * 32;  // 128 codes of this row
+                // this row's 64 bytes hold 256 columns: the k block's 128 codes are one half of them
+                const uint8_t *prow = smem + OFF_P + pj * P_TILE_BYTES + row * 64 + (kb & 1) * 32;
                 const uint4 lo = *reinterpret_cast<const uint4 *>(prow), hi = *reinterpret_cast<const uint4 *>(prow + 16);
                 const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
                 uint32_t a[32];  // register 4 i + j = columns 16 i + 4 j .. + 3 of the k block, one code per byte
@@ -474,8 +542,11 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(bar(BAR_AFULL + s));
-                    mbar_arrive(bar(BAR_EMPTY + s));
+                    mbar_arrive(bar(BAR_FULL + s));
+                    if ((kb & 1) || kb + 1 == kblocks) mbar_arrive(bar(BAR_PEMPTY + pj));
+                }
+                if ((kb & 1) || kb + 1 == kblocks) {
+                    if (++pj == PSTAGES) { pj = 0; pph ^= 1u; }
                 }
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
@@ -539,22 +610,18 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
         attr_set = true;
     }
     const bool bf16 = (p.flags & HGF_FLAG_OUT_BF16) != 0;
-    CUtensorMap mx, mw, my;
+    CUtensorMap mx, mh, mgb, my;
     if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.xq, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.K, KBLK, TILE_T,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;
-    {   // packed weights as a 4-D byte tensor: (byte in row: 64, row in tile: 16, column tile, row tile)
-        EncodeTiledFn fn = get_encode_fn();
-        if (!fn) return cudaErrorInvalidValue;
-        const uint64_t steps = (uint64_t)padded_k(p.K) / 256;
-        cuuint64_t dims[4] = {64, 16, steps, (uint64_t)row_tiles(p.N)};
-        cuuint64_t strides[3] = {64, 1024, steps * 1024};
-        cuuint32_t box[4] = {KBLK / 4, 16, 1, TILE_C / 16};
-        cuuint32_t estr[4] = {1, 1, 1, 1};
-        if (fn(&mw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<uint8_t *>(p.packed), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    if (p.r > 0) {  // H [M][64] and (g B)^T [N][64] fp16: 128-byte rows, tiles of 128 rows, 128-byte swizzle
+        if (!make_map_2d(&mh, CU_TENSOR_MAP_DATA_TYPE_UINT16, p.h16, 64, (uint64_t)p.M, 128, 64, TILE_T, CU_TENSOR_MAP_SWIZZLE_128B))
             return cudaErrorInvalidValue;
+        if (!make_map_2d(&mgb, CU_TENSOR_MAP_DATA_TYPE_UINT16, p.gb16, 64, (uint64_t)p.N, 128, 64, TILE_C, CU_TENSOR_MAP_SWIZZLE_128B))
+            return cudaErrorInvalidValue;
+    } else {
+        mh = mx;
+        mgb = mx;
     }
     if (!make_map_2d(&my, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, p.y, (uint64_t)p.N,
                      (uint64_t)p.M, (uint64_t)p.N * (bf16 ? 2 : 4), 32, 32, CU_TENSOR_MAP_SWIZZLE_NONE))
@@ -564,9 +631,9 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
     unsigned int *status = device_status_word();
     if (!status) return cudaErrorMemoryAllocation;
     if (bf16)
-        prefill_gemm_kernel<true><<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(mx, mw, my, p, status);
+        prefill_gemm_kernel<true><<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(mx, mh, mgb, my, p, status);
     else
-        prefill_gemm_kernel<false><<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(mx, mw, my, p, status);
+        prefill_gemm_kernel<false><<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(mx, mh, mgb, my, p, status);
     count_launch();
     return cudaGetLastError();
 }

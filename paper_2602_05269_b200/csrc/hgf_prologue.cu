@@ -114,6 +114,7 @@ __device__ void quant_row(const PrologueParams &p, int m) {
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) tot += s_red_i[w];
         if (p.row_sum) p.row_sum[m] = tot;
+        if (p.tok_sc) p.tok_sc[m] = g * p.gw_over_127;
         p.gamma_x[m] = g;
         if (p.dbg_gamma_x) p.dbg_gamma_x[m] = g;
     }
@@ -423,6 +424,27 @@ constexpr int kLdTokens = 32;
 template <int JT>  // r = 8 * JT column tiles
 __global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const PrologueParams p) {
     extern __shared__ float s_acc[];  // [4 warps][32 tokens][8*JT]
+    const int token_blocks = (p.M + kLdTokens - 1) / kLdTokens;
+    if ((int)blockIdx.x >= token_blocks) {
+        // the remaining blocks prepare the up-projection's operand: row n of B^T times its channel's
+        // gate, fp16, padded to 64 columns (one 16-byte piece per thread)
+        const int idx = ((int)blockIdx.x - token_blocks) * kLdThreads + (int)threadIdx.x, n = idx >> 3, c = idx & 7;
+        if (n < p.N) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (c * 8 < p.r) {
+                v = *reinterpret_cast<const uint4 *>(p.Bt + (size_t)n * p.r + c * 8);
+                const float g = p.gate[n];
+                __half2 *h2 = reinterpret_cast<__half2 *>(&v);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float2 f = __half22float2(h2[k]);
+                    h2[k] = __floats2half2_rn(g * f.x, g * f.y);
+                }
+            }
+            *reinterpret_cast<uint4 *>(p.gb16 + (size_t)n * 64 + c * 8) = v;
+        }
+        return;
+    }
     const int K = p.K, M = p.M, r = 8 * JT;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int m0 = blockIdx.x * kLdTokens;
@@ -568,7 +590,7 @@ cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_q
 }
 
 cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream) {
-    const int blocks = (p.M + kLdTokens - 1) / kLdTokens;
+    const int blocks = (p.M + kLdTokens - 1) / kLdTokens + (p.gb16 ? (p.N * 8 + kLdThreads - 1) / kLdThreads : 0);
     const size_t smem = (size_t)4 * kLdTokens * p.r * sizeof(float);
     switch (p.r) {
         case 16: lora_down_gemm_kernel<2><<<blocks, kLdThreads, smem, stream>>>(p); break;
