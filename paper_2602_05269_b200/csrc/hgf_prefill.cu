@@ -38,17 +38,17 @@ namespace hgf {
 
 constexpr int TILE_C = 128;   // output channels per tile (MMA M, tensor-memory lanes)
 constexpr int TILE_T = 128;   // tokens per tile (MMA N, accumulator columns)
-constexpr int KBLK = 128;
-constexpr int STAGES = 6;      // activation tiles in shared memory and weight operands in tensor memory
-constexpr int X_TILE_BYTES = TILE_T * KBLK;      // 16 KiB
-constexpr int PSTAGES = 4;
-constexpr int P_TILE_BYTES = TILE_C * 256 / 4;   // 8 KiB: 8 weight tiles of 16 rows x 256 columns, i.e. two k blocks
+constexpr int KBLK = 256;      // input columns per pipeline stage: one column tile of the packed layout
+constexpr int STAGES = 3;      // activation tiles + packed codes in shared memory, weight operands in tensor memory
+constexpr int X_HALF_BYTES = TILE_T * 128;       // 16 KiB: 128 tokens x 128 columns, one 128-byte-swizzled operand tile
+constexpr int X_TILE_BYTES = 2 * X_HALF_BYTES;   // 32 KiB per stage
+constexpr int P_TILE_BYTES = TILE_C * KBLK / 4;  // 8 KiB: 8 weight tiles of 16 rows x 256 columns
 constexpr int LORA_H_BYTES = TILE_T * 128;       // 128 tokens x 64 fp16
 constexpr int LORA_B_BYTES = TILE_C * 128;       // 128 channels x 64 fp16
 constexpr int TOKV_BYTES = TILE_T * 8;           // row sums and scales of the tile's tokens
 constexpr int STORE_BUF_BYTES = 32 * 32 * 4;     // per epilogue warp: 32 tokens x 32 channels
 constexpr int GEMM_THREADS = 320;
-// tensor memory: two accumulators of 128 columns, then STAGES weight operands of 32 columns (= 128 int8 per lane)
+// tensor memory: two accumulators of 128 columns, then STAGES weight operands of 64 columns (= 256 int8 per lane)
 constexpr int TMEM_COLS = 512, ACC_COLS = TILE_T, A_COL = 2 * ACC_COLS, A_STAGE_COLS = KBLK / 4;
 static_assert(A_COL + STAGES * A_STAGE_COLS <= TMEM_COLS, "tensor memory budget");
 
@@ -56,7 +56,7 @@ constexpr int OFF_X = 0;
 constexpr int OFF_LH = OFF_X + STAGES * X_TILE_BYTES;
 constexpr int OFF_LB = OFF_LH + 2 * LORA_H_BYTES;   // the epilogue's operands are double-buffered like the accumulators
 constexpr int OFF_P = OFF_LB + 2 * LORA_B_BYTES;
-constexpr int OFF_TOKV = OFF_P + PSTAGES * P_TILE_BYTES;
+constexpr int OFF_TOKV = OFF_P + STAGES * P_TILE_BYTES;
 constexpr int OFF_ST = OFF_TOKV + 2 * TOKV_BYTES;
 constexpr int OFF_BAR = OFF_ST + 4 * STORE_BUF_BYTES;
 static_assert(OFF_BAR + 512 + 1024 <= 227 * 1024, "shared memory budget");
@@ -65,7 +65,7 @@ constexpr int SMEM_BYTES = SMEM_USED + 1024;  // slack for the 1024-byte alignme
 
 // barrier slots (8 bytes each) inside the OFF_BAR block
 enum { BAR_FULL = 0, BAR_EMPTY = BAR_FULL + STAGES,
-       BAR_PFULL = BAR_EMPTY + STAGES, BAR_PEMPTY = BAR_PFULL + PSTAGES, BAR_ACCFULL = BAR_PEMPTY + PSTAGES,
+       BAR_LOADED = BAR_EMPTY + STAGES, BAR_ACCFULL = BAR_LOADED + STAGES,
        BAR_ACCEMPTY = BAR_ACCFULL + 2, BAR_LORAREADY = BAR_ACCEMPTY + 2, BAR_LORADONE = BAR_LORAREADY + 2,
        BAR_OPSFULL = BAR_LORADONE + 2, BAR_OPSEMPTY = BAR_OPSFULL + 2, BAR_COUNT = BAR_OPSEMPTY + 2 };
 static_assert(BAR_COUNT * 8 + 16 <= 512, "barrier block too small");
@@ -247,17 +247,14 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            // FULL: the activation tile has landed (producer's arrival + its bytes) and the four unpack warps
-            // have put the weight operand into tensor memory.  EMPTY: the MMAs that read both are complete
-            // (one commit; the producer and the unpack warps both wait on it).  One barrier each way keeps
-            // the MMA thread's loop short: it is a single thread and every barrier operation costs it a
-            // shared-memory round trip.
-            mbar_init(bar(BAR_FULL + s), 1 + 4);
+            // LOADED: the stage's activation tile and packed codes have landed (producer's arrival + bytes).
+            // FULL: the four unpack warps have seen LOADED and put the weight operand into tensor memory,
+            // so the MMA thread waits on this one barrier only (it is a single thread and every barrier
+            // operation costs it a shared-memory round trip).  EMPTY: the MMAs that read the stage are
+            // complete (one commit; the producer and the unpack warps both wait on it).
+            mbar_init(bar(BAR_LOADED + s), 1);
+            mbar_init(bar(BAR_FULL + s), 4);
             mbar_init(bar(BAR_EMPTY + s), 1);
-        }
-        for (int j = 0; j < PSTAGES; ++j) {
-            mbar_init(bar(BAR_PFULL + j), 1);
-            mbar_init(bar(BAR_PEMPTY + j), 4);  // four unpack warps: the packed codes have been read
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(BAR_ACCFULL + b), 1);
@@ -288,9 +285,9 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         // with its address arithmetic, cannot keep up with the MMAs): every lane polls the barriers,
         // lane 0 posts the byte counts and the activation tile, lanes 0-7 one weight tile each.
         {
-            int s = 0, pj = 0;
-            uint32_t ph = 0, pph = 0;
-            uint32_t issued[STAGES] = {}, pissued[PSTAGES] = {}, ops_issued[2] = {};
+            int s = 0;
+            uint32_t ph = 0;
+            uint32_t issued[STAGES] = {}, ops_issued[2] = {};
             int pit = 0;
             bool ok = true;
             const int steps = (p.K + 255) >> 8, n_row_tiles = (p.N + 15) >> 4;
@@ -318,25 +315,19 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     ++pit;
                 }
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if ((kb & 1) == 0) {
-                        // packed weights of two k blocks: the 1 KiB tiles (16 rows x 256 columns) of 8 consecutive
-                        // row tiles, each one contiguous in memory
-                        ok = mbar_wait(bar(BAR_PEMPTY + pj), pph ^ 1u, abort_flag, status, 0x110u + pj);
-                        if (!(ok = __all_sync(0xffffffffu, ok))) break;
-                        if (lane == 0) mbar_arrive_expect_tx(bar(BAR_PFULL + pj), (uint32_t)nrt * 1024u);
-                        __syncwarp();
-                        if (lane < nrt)
-                            bulk_load_1d(sbase + OFF_P + pj * P_TILE_BYTES + lane * 1024, psrc + (size_t)(kb >> 1) * 1024, 1024u,
-                                         bar(BAR_PFULL + pj));
-                        ++pissued[pj];
-                        if (++pj == PSTAGES) { pj = 0; pph ^= 1u; }
-                    }
                     ok = mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x100u + s);
                     if (!(ok = __all_sync(0xffffffffu, ok))) break;
                     if (lane == 0) {
-                        mbar_arrive_expect_tx(bar(BAR_FULL + s), X_TILE_BYTES);
-                        tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, t0, bar(BAR_FULL + s));
+                        // 256 columns of 128 tokens as two 128-byte-swizzled tiles (columns past K read as zeros),
+                        // and the 1 KiB tiles (16 rows x 256 columns) of 8 consecutive row tiles
+                        mbar_arrive_expect_tx(bar(BAR_LOADED + s), X_TILE_BYTES + (uint32_t)nrt * 1024u);
+                        tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, t0, bar(BAR_LOADED + s));
+                        tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES + X_HALF_BYTES, &tmap_x, kb * KBLK + 128, t0, bar(BAR_LOADED + s));
                     }
+                    __syncwarp();
+                    if (lane < nrt)
+                        bulk_load_1d(sbase + OFF_P + s * P_TILE_BYTES + lane * 1024, psrc + (size_t)kb * 1024, 1024u,
+                                     bar(BAR_LOADED + s));
                     ++issued[s];
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -346,12 +337,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             for (int q = 0; q < STAGES; ++q)
                 if (issued[q]) {
                     const uint32_t par = (issued[q] - 1u) & 1u;
-                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_FULL + q), par); ++i) {}
-                }
-            for (int q = 0; q < PSTAGES; ++q)
-                if (pissued[q]) {
-                    const uint32_t par = (pissued[q] - 1u) & 1u;
-                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_PFULL + q), par); ++i) {}
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_LOADED + q), par); ++i) {}
                 }
             for (int q = 0; q < 2; ++q)
                 if (ops_issued[q]) {
@@ -396,11 +382,16 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     tc_fence_after();
                     const uint64_t bdesc = xdesc0 + (uint64_t)(s * (X_TILE_BYTES >> 4));
                     const uint32_t a_tmem = tmem_base + A_COL + s * A_STAGE_COLS;
-                    // 32 int8 = 8 columns of the weight operand, 32 bytes of a token row
+                    // per MMA 32 int8: 8 columns of the weight operand, 32 bytes of a token row; the stage's
+                    // second 128 columns sit in the second swizzled tile
                     mma_i8_ts(acc, a_tmem, bdesc, IDESC_I8, kb ? 1u : 0u);
                     mma_i8_ts(acc, a_tmem + 8u, bdesc + 2u, IDESC_I8, 1u);
                     mma_i8_ts(acc, a_tmem + 16u, bdesc + 4u, IDESC_I8, 1u);
                     mma_i8_ts(acc, a_tmem + 24u, bdesc + 6u, IDESC_I8, 1u);
+                    mma_i8_ts(acc, a_tmem + 32u, bdesc + (X_HALF_BYTES >> 4), IDESC_I8, 1u);
+                    mma_i8_ts(acc, a_tmem + 40u, bdesc + (X_HALF_BYTES >> 4) + 2u, IDESC_I8, 1u);
+                    mma_i8_ts(acc, a_tmem + 48u, bdesc + (X_HALF_BYTES >> 4) + 4u, IDESC_I8, 1u);
+                    mma_i8_ts(acc, a_tmem + 56u, bdesc + (X_HALF_BYTES >> 4) + 6u, IDESC_I8, 1u);
                     tc_commit(bar(BAR_EMPTY + s));
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -518,36 +509,35 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         // ------------------------------------------------------------------ unpack warps
         const int q = warp & 3;              // tensor-memory lane quarter this warp may access
         const int row = 32 * q + lane;       // this thread's channel row of the tile = its tensor-memory lane
-        int s = 0, pj = 0;
-        uint32_t ph = 0, pph = 0;
+        int s = 0;
+        uint32_t ph = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < kblocks; ++kb) {
-                // the packed codes of this k block have landed, and the MMAs that read this stage's previous
-                // operand are complete
-                ok = mbar_wait(bar(BAR_PFULL + pj), pph, abort_flag, status, 0x400u + pj) &&
-                     mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x410u + s);
+                // the stage's packed codes have landed; and the MMAs that read this stage's previous operand
+                // are complete (the producer waited for their commit before it refilled the stage)
+                ok = mbar_wait(bar(BAR_LOADED + s), ph, abort_flag, status, 0x400u + s);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
-                // this row's 64 bytes hold 256 columns: the k block's 128 codes are one half of them
-                const uint8_t *prow = smem + OFF_P + pj * P_TILE_BYTES + row * 64 + (kb & 1) * 32;
-                const uint4 lo = *reinterpret_cast<const uint4 *>(prow), hi = *reinterpret_cast<const uint4 *>(prow + 16);
-                const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-                uint32_t a[32];  // register 4 i + j = columns 16 i + 4 j .. + 3 of the k block, one code per byte
+                // this row's 64 bytes hold the stage's 256 columns; register 4 i + j of a half = columns
+                // 16 i + 4 j .. + 3, one code per byte
+                const uint8_t *prow = smem + OFF_P + s * P_TILE_BYTES + row * 64;
+                const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + A_COL + s * A_STAGE_COLS;
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
+                for (int half = 0; half < 2; ++half) {
+                    const uint4 lo = *reinterpret_cast<const uint4 *>(prow + 32 * half);
+                    const uint4 hi = *reinterpret_cast<const uint4 *>(prow + 32 * half + 16);
+                    const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+                    uint32_t a[32];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) a[4 * i + j] = (w[i] >> (2 * j)) & 0x03030303u;
-                tmem_st32(tmem_base + ((uint32_t)(32 * q) << 16) + A_COL + s * A_STAGE_COLS, a);
+                    for (int i = 0; i < 8; ++i)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) a[4 * i + j] = (w[i] >> (2 * j)) & 0x03030303u;
+                    tmem_st32(taddr + 32 * half, a);
+                }
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(bar(BAR_FULL + s));
-                    if ((kb & 1) || kb + 1 == kblocks) mbar_arrive(bar(BAR_PEMPTY + pj));
-                }
-                if ((kb & 1) || kb + 1 == kblocks) {
-                    if (++pj == PSTAGES) { pj = 0; pph ^= 1u; }
-                }
+                if (lane == 0) mbar_arrive(bar(BAR_FULL + s));
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
         }
@@ -611,7 +601,7 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
     }
     const bool bf16 = (p.flags & HGF_FLAG_OUT_BF16) != 0;
     CUtensorMap mx, mh, mgb, my;
-    if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.xq, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.K, KBLK, TILE_T,
+    if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.xq, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.K, 128, TILE_T,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;
     if (p.r > 0) {  // H [M][64] and (g B)^T [N][64] fp16: 128-byte rows, tiles of 128 rows, 128-byte swizzle
