@@ -418,12 +418,13 @@ decode_prologue_group_kernel(const QuantItem *quant_items, int n_quant, const Lo
 // the products are formed from exact inputs and accumulated in fp32.
 // Block = 4 warps, tile = 32 tokens x r columns; the warps split K in 32-element chunks and the
 // partial sums are reduced through shared memory.
-constexpr int kLdThreads = 128;
+constexpr int kLdWarps = 8;
+constexpr int kLdThreads = kLdWarps * 32;
 constexpr int kLdTokens = 32;
 
 template <int JT>  // r = 8 * JT column tiles
 __global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const PrologueParams p) {
-    extern __shared__ float s_acc[];  // [4 warps][32 tokens][8*JT]
+    extern __shared__ float s_acc[];  // [warps][32 tokens][8*JT]
     const int token_blocks = (p.M + kLdTokens - 1) / kLdTokens;
     if ((int)blockIdx.x >= token_blocks) {
         // the remaining blocks prepare the up-projection's operand: row n of B^T times its channel's
@@ -469,7 +470,7 @@ __global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const Prolog
         }
 
     const int nchunks = K / 32;
-    for (int c = warp; c < nchunks; c += 4) {
+    for (int c = warp; c < nchunks; c += kLdWarps) {
         const int k = c * 32 + 8 * t;  // this thread's 8 consecutive k
         uint4 xa[2][2];
 #pragma unroll
@@ -508,7 +509,9 @@ __global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const Prolog
     __syncthreads();
     for (int e = tid; e < kLdTokens * r; e += kLdThreads) {
         int ml = e / r, j = e % r, m = m0 + ml;
-        float z = s_acc[e] + s_acc[kLdTokens * r + e] + s_acc[2 * kLdTokens * r + e] + s_acc[3 * kLdTokens * r + e];
+        float z = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kLdWarps; ++w) z += s_acc[w * kLdTokens * r + e];
         float h = (p.flags & HGF_FLAG_NO_SILU) ? z : silu_f(z);
         if (m < M) {
             p.h[(size_t)m * r + j] = h;
@@ -591,7 +594,14 @@ cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_q
 
 cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream) {
     const int blocks = (p.M + kLdTokens - 1) / kLdTokens + (p.gb16 ? (p.N * 8 + kLdThreads - 1) / kLdThreads : 0);
-    const size_t smem = (size_t)4 * kLdTokens * p.r * sizeof(float);
+    const size_t smem = (size_t)kLdWarps * kLdTokens * p.r * sizeof(float);
+    static bool attr_set = false;
+    if (!attr_set) {  // the widest variant needs more than the default dynamic shared memory
+        cudaError_t e = cudaFuncSetAttribute(lora_down_gemm_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kLdWarps * kLdTokens * 64 * (int)sizeof(float));
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
     switch (p.r) {
         case 16: lora_down_gemm_kernel<2><<<blocks, kLdThreads, smem, stream>>>(p); break;
         case 32: lora_down_gemm_kernel<4><<<blocks, kLdThreads, smem, stream>>>(p); break;
