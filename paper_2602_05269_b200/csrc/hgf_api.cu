@@ -60,7 +60,7 @@ extern "C" hgf_status hgf_act_quant(const void *x, int64_t M, int64_t d_in, int8
     pp.row_sum = row_sum;
     pp.M = (int)M;
     pp.K = (int)d_in;
-    return launch_quant(pp, (cudaStream_t)stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
+    return launch_quant(pp, GemmPrologueExtra{}, (cudaStream_t)stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
 }
 
 namespace hgf {
@@ -97,12 +97,6 @@ static void fill_params(const void *x, int64_t M, const void *packed, float gamm
     pp->h_hi = gemm ? nullptr : (__half *)(ws + L.h_hi);
     pp->h_lo = gemm ? nullptr : (__half *)(ws + L.h_lo);
     pp->h16 = gemm ? (__half *)(ws + L.h16) : nullptr;
-    pp->tok_sc = gemm ? (float *)(ws + L.tok_sc) : nullptr;
-    pp->gb16 = (gemm && r) ? (__half *)(ws + L.gb16) : nullptr;
-    pp->Bt = (const __half *)Bt;
-    pp->gate = gate;
-    pp->gw_over_127 = (float)((double)gamma / 127.0);
-    pp->N = (int)d_out;
     pp->dbg_xq = dbg ? dbg->xq : nullptr;
     pp->dbg_gamma_x = dbg ? dbg->gamma_x : nullptr;
     pp->dbg_h = (dbg && r) ? dbg->h : nullptr;
@@ -166,16 +160,23 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
         return launch_decode_gemv(dl, &dp, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
     }
 
-    if (launch_quant(pp, stream) != cudaSuccess) return HGF_ERR_CUDA;
-    if (r && launch_lora_down_gemm(pp, stream) != cudaSuccess) return HGF_ERR_CUDA;
+    GemmPrologueExtra gx = {};
+    gx.tok_sc = (float *)((char *)workspace + L.tok_sc);
+    gx.gb16 = r ? (__half *)((char *)workspace + L.gb16) : nullptr;
+    gx.Bt = (const __half *)Bt;
+    gx.gate = gate;
+    gx.gw_over_127 = dp.gw_over_127;
+    gx.N = (int)d_out;
+    if (launch_quant(pp, gx, stream) != cudaSuccess) return HGF_ERR_CUDA;
+    if (r && launch_lora_down_gemm(pp, gx, stream) != cudaSuccess) return HGF_ERR_CUDA;
     GemmParams gp = {};
     gp.xq = pp.xq;
     gp.packed = (const uint8_t *)packed;
     gp.gamma_x = pp.gamma_x;
     gp.row_sum = pp.row_sum;
     gp.h16 = pp.h16;
-    gp.tok_sc = pp.tok_sc;
-    gp.gb16 = pp.gb16;
+    gp.tok_sc = gx.tok_sc;
+    gp.gb16 = gx.gb16;
     gp.y = y;
     gp.dbg_y_int = dbg ? dbg->y_int : nullptr;
     gp.gw_over_127 = dp.gw_over_127;

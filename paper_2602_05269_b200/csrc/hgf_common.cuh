@@ -73,17 +73,22 @@ struct PrologueParams {
     float *h;                // [M][r]
     __half *h_hi, *h_lo;     // [M][r] each (decode path) or null
     __half *h16;             // [M][64] (GEMM path) or null
-    float *tok_sc;           // [M] gamma_x * gamma_W / 127 (GEMM path) or null
-    __half *gb16;            // [N][64] gate * B^T (GEMM path) or null
-    const __half *Bt;        // [N][r]  (GEMM path, for gb16)
-    const float *gate;       // [N]     (GEMM path, for gb16)
-    float gw_over_127;
-    int N;
     int8_t *dbg_xq;          // nullable debug copies
     float *dbg_gamma_x;
     float *dbg_h;
     int M, K, r;
     uint32_t flags;
+};
+
+// What the GEMM path's prologue kernels produce beyond PrologueParams (kept apart so that the decode
+// kernels' parameter block stays as small as it was).
+struct GemmPrologueExtra {
+    float *tok_sc;           // [M] gamma_x * gamma_W / 127, or null
+    __half *gb16;            // [N][64] gate * B^T, or null
+    const __half *Bt;        // [N][r]
+    const float *gate;       // [N]
+    float gw_over_127;
+    int N;
 };
 
 // One layer problem of a decode launch (M <= 16).  tile_begin = index of its first 16-row tile in
@@ -120,7 +125,7 @@ struct DecodeLaunch {
 };
 
 // host-side launchers (each enqueues on `stream` and returns the CUDA error of the launch)
-cudaError_t launch_quant(const PrologueParams &p, cudaStream_t stream);
+cudaError_t launch_quant(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream);
 cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream_t stream);
 // Group prologue.  A quantisation item is one token row.  A LoRA item is 16 columns of H (rows
 // 16 jt .. 16 jt + 15 of A^T) over one K slice of a problem; its 16 x 16 partial sums of x A go to
@@ -144,7 +149,7 @@ static inline int prologue_slice_k(int max_M) { return max_M <= 8 ? 512 : 256; }
 cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_quant,
                                          const LoraItem *d_lora_items, int n_lora, int max_M, bool pdl,
                                          cudaStream_t stream);
-cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream);
+cudaError_t launch_lora_down_gemm(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream);
 cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream);
 // Shared memory the decode kernel needs for one problem's activations, and the largest it accepts.
 int decode_xq_smem_bytes(int M, int K);

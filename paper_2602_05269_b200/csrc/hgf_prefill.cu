@@ -6,23 +6,24 @@
 // The ternary weights are the MMA's first operand and are read from TENSOR MEMORY: the tensor core
 // cannot read 2-bit codes, and expanding them to int8 in shared memory costs four times their bytes
 // in shared-memory writes plus the same again when the MMA reads them - more than the port has.
-// Here four warps expand a packed 128 x 128 tile straight from its 4 KiB in shared memory into
-// registers (one 128-channel row per thread: a shift and a mask per register) and store it with one
+// Here four warps expand a packed 128 x 256 tile straight from its 8 KiB in shared memory into
+// registers (one 128-channel row per thread: a shift and a mask per register) and store it with two
 // tcgen05.st into the operand's place in tensor memory, so shared memory carries only the int8
 // activation tile (TMA in, MMA out) and the packed codes.  The output tile is therefore
 // 128 output channels (tensor-memory lanes, MMA M) x 128 tokens (columns, MMA N); two accumulators
-// alternate, so the epilogue of a tile runs under the main loop of the next, and eight pipeline
-// stages cover the latency of the load -> expand -> MMA -> release round trip.
+// alternate, so the epilogue of a tile runs under the main loop of the next.  A pipeline stage is
+// 256 input columns (eight MMAs): every hand-over between the roles costs a shared-memory round
+// trip, and the single MMA-issuing thread can only afford one per 512 tensor-core clocks.
 //
 // One persistent CTA per SM, 10 warps with fixed roles:
-//   warp 0      TMA producer: per 128-wide k block the int8 activation tile (128 tokens x 128 B,
-//               128-byte swizzle), per two k blocks the packed weights of 128 channels (eight
-//               contiguous 1 KiB tiles of the tiled weight layout, one bulk copy each), and per tile
-//               what its epilogue needs: row sums, scales, the H tile and the (g B)^T tile
+//   warp 0      producer (all lanes): per stage the int8 activation tile as two 128 tokens x 128 B
+//               boxes (128-byte swizzle) and the packed weights of 128 channels (eight contiguous
+//               1 KiB tiles of the tiled weight layout, one bulk copy each); per tile what its
+//               epilogue needs: row sums, scales, the H tile and the (g B)^T tile
 //   warp 1      allocates tensor memory; one lane issues the MMAs and commits to mbarriers
-//   warps 2-5   epilogue: dequantise the accumulator in place
-//               (tcgen05.ld / tcgen05.st), wait for the correction MMA, read the result, transpose it
-//               through shared memory and store y with TMA
+//   warps 2-5   epilogue: dequantise the accumulator in place (tcgen05.ld / tcgen05.st), wait for
+//               the correction MMA, read the result, transpose it through shared memory and store
+//               y with TMA
 //   warps 6-9   expand the packed tile into tensor memory
 // Codes are c = t + 1 (both operands are declared signed 8-bit; 0, 1, 2 read the same either way);
 // sum_k t x~ = sum_k c x~ - sum_k x~ is restored in the epilogue from the row sums.
@@ -102,7 +103,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     return t;
 }
 // Bounded wait: gives up after kWaitLimitNs of wall time.  Returns false if it gave up or another
-// role already aborted.  A waiting warp sleeps between polls (20 ns, growing to 320 ns): the roles of
+// role already aborted.  A waiting warp sleeps between polls (20 ns, growing to 80 ns): the roles of
 // this kernel share the SM's schedulers and its shared-memory pipe, and warps that poll without a
 // pause slow the ones that have work.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
@@ -112,7 +113,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     unsigned int ns = 20;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         __nanosleep(ns);
-        if (ns < 320) ns *= 2;
+        if (ns < 80) ns *= 2;
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63u) == 63u) {
             if (*abort_flag) return false;
@@ -130,12 +131,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
 // Untiled bulk copy global -> shared (addresses 16-byte aligned, size a multiple of 16), completing on the mbarrier.

@@ -62,7 +62,7 @@ __device__ __forceinline__ int quant1(float x, const QuantScale &s) {
 }
 
 // One block quantises one token row.
-__device__ void quant_row(const PrologueParams &p, int m) {
+__device__ __forceinline__ void quant_row(const PrologueParams &p, int m, float *tok_sc = nullptr, float gw_over_127 = 0.0f) {
     __shared__ float s_red_f[kWarps];
     __shared__ int s_red_i[kWarps];
     const int K = p.K, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -114,7 +114,7 @@ __device__ void quant_row(const PrologueParams &p, int m) {
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) tot += s_red_i[w];
         if (p.row_sum) p.row_sum[m] = tot;
-        if (p.tok_sc) p.tok_sc[m] = g * p.gw_over_127;
+        if (tok_sc) tok_sc[m] = g * gw_over_127;
         p.gamma_x[m] = g;
         if (p.dbg_gamma_x) p.dbg_gamma_x[m] = g;
     }
@@ -143,7 +143,7 @@ __device__ __forceinline__ uint4 ldg_nc_u4(const void *ptr) {
 // 8-column operand; the warps split K in 32-element chunks and their partial sums are added in a
 // fixed order through shared memory.  NT = number of 8-token tiles.
 template <int NT>
-__device__ void lora_down_tile(const PrologueParams &p, int jt) {
+__device__ __forceinline__ void lora_down_tile(const PrologueParams &p, int jt) {
     __shared__ float s_red[kWarps][NT * 4][32];
     const int K = p.K, M = p.M, r = p.r, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const __half *rowA = p.At + (size_t)(16 * jt + g) * K + 8 * t;
@@ -227,8 +227,8 @@ __device__ __forceinline__ void lora_down_block(const PrologueParams &p, int jt)
     if (p.M <= 8) lora_down_tile<1>(p, jt); else lora_down_tile<2>(p, jt);
 }
 
-__global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p) {
-    quant_row(p, blockIdx.x);
+__global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p, const GemmPrologueExtra x) {
+    quant_row(p, blockIdx.x, x.tok_sc, x.gw_over_127);
 }
 
 // Programmatic dependent launch: no-ops when the launch carries no such attribute.
@@ -423,18 +423,18 @@ constexpr int kLdThreads = kLdWarps * 32;
 constexpr int kLdTokens = 32;
 
 template <int JT>  // r = 8 * JT column tiles
-__global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const PrologueParams p) {
+__global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const PrologueParams p, const GemmPrologueExtra x) {
     extern __shared__ float s_acc[];  // [warps][32 tokens][8*JT]
     const int token_blocks = (p.M + kLdTokens - 1) / kLdTokens;
     if ((int)blockIdx.x >= token_blocks) {
         // the remaining blocks prepare the up-projection's operand: row n of B^T times its channel's
         // gate, fp16, padded to 64 columns (one 16-byte piece per thread)
         const int idx = ((int)blockIdx.x - token_blocks) * kLdThreads + (int)threadIdx.x, n = idx >> 3, c = idx & 7;
-        if (n < p.N) {
+        if (n < x.N) {
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
             if (c * 8 < p.r) {
-                v = *reinterpret_cast<const uint4 *>(p.Bt + (size_t)n * p.r + c * 8);
-                const float g = p.gate[n];
+                v = *reinterpret_cast<const uint4 *>(x.Bt + (size_t)n * p.r + c * 8);
+                const float g = x.gate[n];
                 __half2 *h2 = reinterpret_cast<__half2 *>(&v);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
@@ -442,7 +442,7 @@ __global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const Prolog
                     h2[k] = __floats2half2_rn(g * f.x, g * f.y);
                 }
             }
-            *reinterpret_cast<uint4 *>(p.gb16 + (size_t)n * 64 + c * 8) = v;
+            *reinterpret_cast<uint4 *>(x.gb16 + (size_t)n * 64 + c * 8) = v;
         }
         return;
     }
@@ -528,8 +528,8 @@ __global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const Prolog
     }
 }
 
-cudaError_t launch_quant(const PrologueParams &p, cudaStream_t stream) {
-    quant_kernel<<<p.M, kThreads, 0, stream>>>(p);
+cudaError_t launch_quant(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
+    quant_kernel<<<p.M, kThreads, 0, stream>>>(p, x);
     count_launch();
     return cudaGetLastError();
 }
@@ -592,8 +592,8 @@ cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_q
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream) {
-    const int blocks = (p.M + kLdTokens - 1) / kLdTokens + (p.gb16 ? (p.N * 8 + kLdThreads - 1) / kLdThreads : 0);
+cudaError_t launch_lora_down_gemm(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
+    const int blocks = (p.M + kLdTokens - 1) / kLdTokens + (x.gb16 ? (x.N * 8 + kLdThreads - 1) / kLdThreads : 0);
     const size_t smem = (size_t)kLdWarps * kLdTokens * p.r * sizeof(float);
     static bool attr_set = false;
     if (!attr_set) {  // the widest variant needs more than the default dynamic shared memory
@@ -603,10 +603,10 @@ cudaError_t launch_lora_down_gemm(const PrologueParams &p, cudaStream_t stream) 
         attr_set = true;
     }
     switch (p.r) {
-        case 16: lora_down_gemm_kernel<2><<<blocks, kLdThreads, smem, stream>>>(p); break;
-        case 32: lora_down_gemm_kernel<4><<<blocks, kLdThreads, smem, stream>>>(p); break;
-        case 48: lora_down_gemm_kernel<6><<<blocks, kLdThreads, smem, stream>>>(p); break;
-        case 64: lora_down_gemm_kernel<8><<<blocks, kLdThreads, smem, stream>>>(p); break;
+        case 16: lora_down_gemm_kernel<2><<<blocks, kLdThreads, smem, stream>>>(p, x); break;
+        case 32: lora_down_gemm_kernel<4><<<blocks, kLdThreads, smem, stream>>>(p, x); break;
+        case 48: lora_down_gemm_kernel<6><<<blocks, kLdThreads, smem, stream>>>(p, x); break;
+        case 64: lora_down_gemm_kernel<8><<<blocks, kLdThreads, smem, stream>>>(p, x); break;
         default: return cudaErrorInvalidValue;
     }
     count_launch();
