@@ -218,6 +218,16 @@ class Workload:
         return t0.elapsed_time(t1) / steps
 
 
+def reduce_max_over_ranks(ms, world, dist, device):
+    """The step time of the job = the slowest rank's (every rank runs its own replica of the workload)."""
+    if world == 1:
+        return ms
+    import torch
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -236,11 +246,7 @@ def run_ours(args):
     peaks = measured_peaks()
 
     def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_max_over_ranks(ms, world, dist, "cuda")
 
     def barrier():
         if world > 1:
