@@ -32,30 +32,63 @@ __device__ __forceinline__ int quant1_div(float x, float gamma) {
     q = fminf(fmaxf(q, -127.0f), 127.0f);
     return __float2int_rn(q);
 }
-// Division-free form, for gamma = max |x| over bf16 values (so gamma is a bf16 value itself, i.e. not
-// the 1e-5 floor).  A candidate q = rint(x * (127 / gamma)) is within one of the answer.  The
-// residual 127 x - q gamma is exact in one fma (127 x and q gamma each have at most 15 significant
-// bits), and the exact quotient is q + residual / gamma: the candidate stands iff
-// 2 |residual| < gamma, or = gamma with q even (a tie goes to the even neighbour); otherwise it
-// moves one step towards the residual's sign.
+// Division- and conversion-free form, for gamma = max |x| over bf16 values (so gamma is a bf16 value
+// itself, i.e. not the 1e-5 floor).  Adding 1.5 * 2^23 in one fma rounds x * (127 / gamma) to an
+// integer (nearest, ties to even) in the low mantissa bits - a candidate that can only be wrong on
+// an exact tie of the true quotient.  The residual 127 x - q gamma is exact in one fma (127 x and
+// q gamma each have at most 15 significant bits), and the exact quotient is q + residual / gamma:
+// off a tie the candidate is always right (checked over every pair of bf16 mantissas and every
+// exponent gap in exact arithmetic), so it stands unless 2 |residual| = gamma with q odd: a tie goes
+// to the even neighbour, one step towards the residual's sign.  No F2I / FRND: those run at an
+// eighth of the FMA rate and bounded the quantisation kernels.
 struct QuantScale {
-    float gamma, inv127;  // inv127 = 127 / gamma
-    bool fast;            // gamma is a bf16 value
+    float gamma, half_gamma, inv127;  // inv127 = 127 / gamma
+    bool fast;                        // gamma is a bf16 value
 };
 __device__ __forceinline__ QuantScale make_quant_scale(float gamma) {
     QuantScale s;
     s.gamma = gamma;
+    s.half_gamma = 0.5f * gamma;
     s.inv127 = __fdiv_rn(127.0f, gamma);
     s.fast = (__float_as_uint(gamma) & 0xffffu) == 0u;
     return s;
 }
 __device__ __forceinline__ int quant1_fast(float x, const QuantScale &s) {
-    float q = rintf(x * s.inv127);
+    constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: integers in [-2^22, 2^22] sit in the mantissa
+    const float tm = fmaf(x, s.inv127, kMagic);
+    int qi = __float_as_int(tm) - 0x4B400000;
+    const float q = tm - kMagic;
     const float res = fmaf(-q, s.gamma, 127.0f * x);
-    const float two = 2.0f * fabsf(res);
-    const bool odd = (__float2int_rn(q) & 1) != 0;
-    if (two > s.gamma || (two == s.gamma && odd)) q += copysignf(1.0f, res);
-    return __float2int_rn(q);
+    const float ar = fabsf(res);
+    if (ar == s.half_gamma && (qi & 1)) qi += res > 0.0f ? 1 : -1;  // (2 |residual| > gamma cannot occur)
+    return qi;
+}
+// Largest magnitude of the eight bf16 values of a 16-byte unit, on the bit patterns: without the sign
+// bit a bf16 pattern orders like its magnitude, so a packed 16-bit maximum does two values at a time.
+__device__ __forceinline__ uint32_t absmax8_bits(uint32_t acc, const uint4 &v) {
+    acc = __vmaxu2(acc, v.x & 0x7fff7fffu);
+    acc = __vmaxu2(acc, v.y & 0x7fff7fffu);
+    acc = __vmaxu2(acc, v.z & 0x7fff7fffu);
+    return __vmaxu2(acc, v.w & 0x7fff7fffu);
+}
+__device__ __forceinline__ float absmax_bits_to_float(uint32_t acc) {
+    const uint32_t hi = acc >> 16, lo = acc & 0xffffu;
+    return __uint_as_float((hi > lo ? hi : lo) << 16);
+}
+__device__ __forceinline__ int quant1(float x, const QuantScale &s);
+// The eight values of a 16-byte unit -> eight int8 (two words), their sum added to `sum`.
+__device__ __forceinline__ uint2 quant8(const uint4 &v, const QuantScale &s, int &sum) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int q0 = quant1(bf16lo_to_float(w[2 * h]), s), q1 = quant1(bf16hi_to_float(w[2 * h]), s);
+        const int q2 = quant1(bf16lo_to_float(w[2 * h + 1]), s), q3 = quant1(bf16hi_to_float(w[2 * h + 1]), s);
+        const uint32_t p01 = __byte_perm((uint32_t)q0, (uint32_t)q1, 0x0040), p23 = __byte_perm((uint32_t)q2, (uint32_t)q3, 0x0040);
+        o[h] = __byte_perm(p01, p23, 0x5410);
+        sum = __dp4a((int)o[h], 0x01010101, sum);
+    }
+    return make_uint2(o[0], o[1]);
 }
 __device__ __forceinline__ int quant1(float x, const QuantScale &s) {
     return s.fast ? quant1_fast(x, s) : quant1_div(x, s.gamma);
@@ -69,17 +102,9 @@ __device__ __forceinline__ void quant_row(const PrologueParams &p, int m, float 
     const uint4 *xv = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K);
     const int nv = K / 8;
 
-    float amax = 0.0f;
-    for (int i = tid; i < nv; i += kThreads) {
-        uint4 v = xv[i];
-        uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            amax = fmaxf(amax, fabsf(bf16lo_to_float(w[j])));
-            amax = fmaxf(amax, fabsf(bf16hi_to_float(w[j])));
-        }
-    }
-    amax = warp_max(amax);
+    uint32_t abits = 0u;
+    for (int i = tid; i < nv; i += kThreads) abits = absmax8_bits(abits, xv[i]);
+    float amax = warp_max(absmax_bits_to_float(abits));
     if (lane == 0) s_red_f[warp] = amax;
     __syncthreads();
     float g = s_red_f[0];
@@ -92,19 +117,9 @@ __device__ __forceinline__ void quant_row(const PrologueParams &p, int m, float 
     uint2 *qv = reinterpret_cast<uint2 *>(p.xq + (size_t)m * K);
     uint2 *dq = p.dbg_xq ? reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * K) : nullptr;
     for (int i = tid; i < nv; i += kThreads) {
-        uint4 v = xv[i];
-        uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        uint32_t o[2] = {0u, 0u};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            int q0 = quant1(bf16lo_to_float(w[j]), qs);
-            int q1 = quant1(bf16hi_to_float(w[j]), qs);
-            sum += q0 + q1;
-            o[j >> 1] |= (uint32_t)(q0 & 0xff) << (16 * (j & 1));
-            o[j >> 1] |= (uint32_t)(q1 & 0xff) << (16 * (j & 1) + 8);
-        }
-        qv[i] = make_uint2(o[0], o[1]);
-        if (dq) dq[i] = make_uint2(o[0], o[1]);
+        const uint2 o = quant8(xv[i], qs, sum);
+        qv[i] = o;
+        if (dq) dq[i] = o;
     }
     sum = warp_sum_i(sum);
     if (lane == 0) s_red_i[warp] = sum;
@@ -227,6 +242,43 @@ __device__ __forceinline__ void lora_down_block(const PrologueParams &p, int jt)
     if (p.M <= 8) lora_down_tile<1>(p, jt); else lora_down_tile<2>(p, jt);
 }
 
+// Many rows of up to 4096 elements (GEMM path): one warp per token row, the row held in registers between the maximum and
+// the rounding (U 16-byte units per lane), so a row costs one trip to memory, no block-wide
+// synchronisation, and the per-row overhead (scale, reductions) is spread over 8 U elements per lane.
+template <int U>
+__global__ void __launch_bounds__(kThreads) quant_rows_kernel(const PrologueParams p, const GemmPrologueExtra x) {
+    const int lane = threadIdx.x & 31, m = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (m >= p.M) return;
+    const int K = p.K, nv = K / 8;
+    const uint4 *xv = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K);
+    uint4 v[U];
+    uint32_t abits = 0u;
+#pragma unroll
+    for (int u = 0; u < U; ++u) v[u] = lane + 32 * u < nv ? xv[lane + 32 * u] : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int u = 0; u < U; ++u) abits = absmax8_bits(abits, v[u]);
+    const float g = fmaxf(warp_max(absmax_bits_to_float(abits)), 1e-5f);
+    const QuantScale qs = make_quant_scale(g);
+    int sum = 0;
+    uint2 *qv = reinterpret_cast<uint2 *>(p.xq + (size_t)m * K);
+    uint2 *dq = p.dbg_xq ? reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * K) : nullptr;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        if (lane + 32 * u < nv) {
+            const uint2 o = quant8(v[u], qs, sum);
+            qv[lane + 32 * u] = o;
+            if (dq) dq[lane + 32 * u] = o;
+        }
+    }
+    sum = warp_sum_i(sum);
+    if (lane == 0) {
+        if (p.row_sum) p.row_sum[m] = sum;
+        if (x.tok_sc) x.tok_sc[m] = g * x.gw_over_127;
+        p.gamma_x[m] = g;
+        if (p.dbg_gamma_x) p.dbg_gamma_x[m] = g;
+    }
+}
+
 __global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p, const GemmPrologueExtra x) {
     quant_row(p, blockIdx.x, x.tok_sc, x.gw_over_127);
 }
@@ -281,39 +333,19 @@ __device__ void warp_quant_row(const QuantItem &q, uint32_t buf_u32, const uint8
         asm volatile("cp.async.wait_all;\n" ::: "memory");
         return n;
     };
-    float amax = 0.0f;
+    uint32_t abits = 0u;
     int n = 0;
     for (int pc = 0; pc < npieces; ++pc) {
         n = fetch(pc);
-        for (int i = lane; i < n; i += 32) {
-            const uint4 v = *reinterpret_cast<const uint4 *>(buf + 16 * i);
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                amax = fmaxf(amax, fabsf(bf16lo_to_float(w[j])));
-                amax = fmaxf(amax, fabsf(bf16hi_to_float(w[j])));
-            }
-        }
+        for (int i = lane; i < n; i += 32) abits = absmax8_bits(abits, *reinterpret_cast<const uint4 *>(buf + 16 * i));
     }
-    const float g = fmaxf(warp_max(amax), 1e-5f);
+    const float g = fmaxf(warp_max(absmax_bits_to_float(abits)), 1e-5f);
     const QuantScale qs = make_quant_scale(g);
     int sum = 0;
     for (int pc = 0; pc < npieces; ++pc) {
         if (npieces > 1) n = fetch(pc);
         uint2 *qv = reinterpret_cast<uint2 *>(q.xq + (size_t)pc * piece);
-        for (int i = lane; i < n; i += 32) {
-            const uint4 v = *reinterpret_cast<const uint4 *>(buf + 16 * i);
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-            uint32_t o[2] = {0u, 0u};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int q0 = quant1(bf16lo_to_float(w[j]), qs), q1 = quant1(bf16hi_to_float(w[j]), qs);
-                sum += q0 + q1;
-                o[j >> 1] |= (uint32_t)(q0 & 0xff) << (16 * (j & 1));
-                o[j >> 1] |= (uint32_t)(q1 & 0xff) << (16 * (j & 1) + 8);
-            }
-            qv[i] = make_uint2(o[0], o[1]);
-        }
+        for (int i = lane; i < n; i += 32) qv[i] = quant8(*reinterpret_cast<const uint4 *>(buf + 16 * i), qs, sum);
     }
     sum = warp_sum_i(sum);
     if (lane == 0) {
@@ -529,7 +561,13 @@ __global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const Prolog
 }
 
 cudaError_t launch_quant(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
-    quant_kernel<<<p.M, kThreads, 0, stream>>>(p, x);
+    const int nv = p.K / 8, row_blocks = (p.M + kWarps - 1) / kWarps;
+    if (p.M >= 256 && nv <= 32 * 8)
+        quant_rows_kernel<8><<<row_blocks, kThreads, 0, stream>>>(p, x);
+    else if (p.M >= 256 && nv <= 32 * 16)
+        quant_rows_kernel<16><<<row_blocks, kThreads, 0, stream>>>(p, x);
+    else
+        quant_kernel<<<p.M, kThreads, 0, stream>>>(p, x);
     count_launch();
     return cudaGetLastError();
 }
