@@ -40,36 +40,39 @@ namespace hgf {
 constexpr int TILE_C = 128;   // output channels per tile (MMA M, tensor-memory lanes)
 constexpr int TILE_T = 128;   // tokens per tile (MMA N, accumulator columns)
 constexpr int KBLK = 256;      // input columns per pipeline stage: one column tile of the packed layout
-constexpr int STAGES = 3;      // activation tiles + packed codes in shared memory, weight operands in tensor memory
 constexpr int X_HALF_BYTES = TILE_T * 128;       // 16 KiB: 128 tokens x 128 columns, one 128-byte-swizzled operand tile
 constexpr int X_TILE_BYTES = 2 * X_HALF_BYTES;   // 32 KiB per stage
 constexpr int P_TILE_BYTES = TILE_C * KBLK / 4;  // 8 KiB: 8 weight tiles of 16 rows x 256 columns
-constexpr int LORA_H_BYTES = TILE_T * 128;       // 128 tokens x 64 fp16
-constexpr int LORA_B_BYTES = TILE_C * 128;       // 128 channels x 64 fp16
 constexpr int TOKV_BYTES = TILE_T * 8;           // row sums and scales of the tile's tokens
 constexpr int STORE_BUF_BYTES = 32 * 32 * 4;     // per epilogue warp: 32 tokens x 32 channels
 constexpr int GEMM_THREADS = 320;
-// tensor memory: two accumulators of 128 columns, then STAGES weight operands of 64 columns (= 256 int8 per lane)
+// tensor memory: two accumulators of 128 columns, then one weight operand of 64 columns (= 256 int8 per lane) per stage
 constexpr int TMEM_COLS = 512, ACC_COLS = TILE_T, A_COL = 2 * ACC_COLS, A_STAGE_COLS = KBLK / 4;
-static_assert(A_COL + STAGES * A_STAGE_COLS <= TMEM_COLS, "tensor memory budget");
 
-constexpr int OFF_X = 0;
-constexpr int OFF_LH = OFF_X + STAGES * X_TILE_BYTES;
-constexpr int OFF_LB = OFF_LH + 2 * LORA_H_BYTES;   // the epilogue's operands are double-buffered like the accumulators
-constexpr int OFF_P = OFF_LB + 2 * LORA_B_BYTES;
-constexpr int OFF_TOKV = OFF_P + STAGES * P_TILE_BYTES;
-constexpr int OFF_ST = OFF_TOKV + 2 * TOKV_BYTES;
-constexpr int OFF_BAR = OFF_ST + 4 * STORE_BUF_BYTES;
-static_assert(OFF_BAR + 512 + 1024 <= 227 * 1024, "shared memory budget");
-constexpr int SMEM_USED = OFF_BAR + 512;
-constexpr int SMEM_BYTES = SMEM_USED + 1024;  // slack for the 1024-byte alignment of the base
-
-// barrier slots (8 bytes each) inside the OFF_BAR block
-enum { BAR_FULL = 0, BAR_EMPTY = BAR_FULL + STAGES,
-       BAR_LOADED = BAR_EMPTY + STAGES, BAR_ACCFULL = BAR_LOADED + STAGES,
-       BAR_ACCEMPTY = BAR_ACCFULL + 2, BAR_LORAREADY = BAR_ACCEMPTY + 2, BAR_LORADONE = BAR_LORAREADY + 2,
-       BAR_OPSFULL = BAR_LORADONE + 2, BAR_OPSEMPTY = BAR_OPSFULL + 2, BAR_COUNT = BAR_OPSEMPTY + 2 };
-static_assert(BAR_COUNT * 8 + 16 <= 512, "barrier block too small");
+// Shared-memory map and barrier slots of a kernel variant.  NS = pipeline stages (activation tile +
+// packed codes in shared memory, weight operand in tensor memory).  OPSB = bytes per row of the
+// correction's two operand tiles: 128 (64 fp16, any rank), or 64 when r <= 32 - which leaves room
+// for a fourth stage.
+template <int NS, int OPSB>
+struct Cfg {
+    static constexpr int STAGES = NS;
+    static constexpr int LORA_H_BYTES = TILE_T * OPSB, LORA_B_BYTES = TILE_C * OPSB;
+    static constexpr int OFF_X = 0;
+    static constexpr int OFF_LH = OFF_X + NS * X_TILE_BYTES;
+    static constexpr int OFF_LB = OFF_LH + 2 * LORA_H_BYTES;  // the epilogue's operands are double-buffered like the accumulators
+    static constexpr int OFF_P = OFF_LB + 2 * LORA_B_BYTES;
+    static constexpr int OFF_TOKV = OFF_P + NS * P_TILE_BYTES;
+    static constexpr int OFF_ST = OFF_TOKV + 2 * TOKV_BYTES;
+    static constexpr int OFF_BAR = OFF_ST + 4 * STORE_BUF_BYTES;
+    static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;  // + slack for the 1024-byte alignment of the base
+    // barrier slots (8 bytes each) inside the OFF_BAR block
+    static constexpr int BAR_FULL = 0, BAR_EMPTY = BAR_FULL + NS, BAR_LOADED = BAR_EMPTY + NS, BAR_ACCFULL = BAR_LOADED + NS,
+                         BAR_ACCEMPTY = BAR_ACCFULL + 2, BAR_LORAREADY = BAR_ACCEMPTY + 2, BAR_LORADONE = BAR_LORAREADY + 2,
+                         BAR_OPSFULL = BAR_LORADONE + 2, BAR_OPSEMPTY = BAR_OPSFULL + 2, BAR_COUNT = BAR_OPSEMPTY + 2;
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+    static_assert(BAR_COUNT * 8 + 16 <= 512, "barrier block too small");
+    static_assert(A_COL + NS * A_STAGE_COLS <= TMEM_COLS, "tensor memory budget");
+};
 
 constexpr uint32_t kSpinLimit = 1u << 22;            // polls of a drain loop
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // bounded waits give up after two seconds
@@ -215,23 +218,29 @@ __device__ __forceinline__ void mma_i8_ts(uint32_t d, uint32_t a_tmem, uint64_t 
 
 // Instruction descriptor: D format (bits 4-5), A format (7-9), B format (10-12), K-major A and B,
 // N >> 3 (17-22), M >> 4 (24-28).
+// The same for K-major rows of 64 bytes with 64-byte swizzle (groups of 8 rows 512 bytes apart, layout type 4).
+__device__ __forceinline__ uint64_t make_sw64_desc(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(512 >> 4) << 32) | (1ull << 46) |
+           (4ull << 61);
+}
 constexpr uint32_t IDESC_I8 = (2u << 4) /*s32*/ | (1u << 7) /*A s8*/ | (1u << 10) /*B s8*/ |
                               ((uint32_t)(TILE_T >> 3) << 17) | ((uint32_t)(TILE_C >> 4) << 24);
 constexpr uint32_t IDESC_F16 = (1u << 4) /*f32*/ | (0u << 7) /*A f16*/ | (0u << 10) /*B f16*/ |
                                ((uint32_t)(TILE_T >> 3) << 17) | ((uint32_t)(TILE_C >> 4) << 24);
 
-template <bool OUT_BF16>
+template <bool OUT_BF16, int NS, int OPSB>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_h,
                     const __grid_constant__ CUtensorMap tmap_gb, const __grid_constant__ CUtensorMap tmap_y,
                     const GemmParams p, unsigned int *status) {
+    using C = Cfg<NS, OPSB>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t bar0 = sbase + OFF_BAR;
+    const uint32_t bar0 = sbase + C::OFF_BAR;
     auto bar = [&](int i) { return bar0 + 8u * i; };
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + OFF_BAR + BAR_COUNT * 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_BAR + BAR_COUNT * 8 + 4);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::OFF_BAR + C::BAR_COUNT * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_BAR + C::BAR_COUNT * 8 + 4);
     static_assert(TILE_T == 128, "the epilogue's staging loops are written for 128-token tiles");
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -241,23 +250,23 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const bool has_lora = p.r > 0;
 
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < C::STAGES; ++s) {
             // LOADED: the stage's activation tile and packed codes have landed (producer's arrival + bytes).
             // FULL: the four unpack warps have seen LOADED and put the weight operand into tensor memory,
             // so the MMA thread waits on this one barrier only (it is a single thread and every barrier
             // operation costs it a shared-memory round trip).  EMPTY: the MMAs that read the stage are
             // complete (one commit; the producer and the unpack warps both wait on it).
-            mbar_init(bar(BAR_LOADED + s), 1);
-            mbar_init(bar(BAR_FULL + s), 4);
-            mbar_init(bar(BAR_EMPTY + s), 1);
+            mbar_init(bar(C::BAR_LOADED + s), 1);
+            mbar_init(bar(C::BAR_FULL + s), 4);
+            mbar_init(bar(C::BAR_EMPTY + s), 1);
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(bar(BAR_ACCFULL + b), 1);
-            mbar_init(bar(BAR_ACCEMPTY + b), 4);
-            mbar_init(bar(BAR_LORAREADY + b), 4);
-            mbar_init(bar(BAR_LORADONE + b), 1);
-            mbar_init(bar(BAR_OPSFULL + b), 1);
-            mbar_init(bar(BAR_OPSEMPTY + b), 4);
+            mbar_init(bar(C::BAR_ACCFULL + b), 1);
+            mbar_init(bar(C::BAR_ACCEMPTY + b), 4);
+            mbar_init(bar(C::BAR_LORAREADY + b), 4);
+            mbar_init(bar(C::BAR_LORADONE + b), 1);
+            mbar_init(bar(C::BAR_OPSFULL + b), 1);
+            mbar_init(bar(C::BAR_OPSEMPTY + b), 4);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -282,7 +291,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         {
             int s = 0;
             uint32_t ph = 0;
-            uint32_t issued[STAGES] = {}, ops_issued[2] = {};
+            uint32_t issued[C::STAGES] = {}, ops_issued[2] = {};
             int pit = 0;
             bool ok = true;
             const int steps = (p.K + 255) >> 8, n_row_tiles = (p.N + 15) >> 4;
@@ -295,49 +304,49 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     // what the tile's epilogue needs, into the buffer of the tile's accumulator: row sums and
                     // scales of the 128 tokens, and with a correction the H tile and the (g B)^T tile
                     const int b = pit & 1;
-                    ok = mbar_wait(bar(BAR_OPSEMPTY + b), ((uint32_t)(pit >> 1) & 1u) ^ 1u, abort_flag, status, 0x120u + b);
+                    ok = mbar_wait(bar(C::BAR_OPSEMPTY + b), ((uint32_t)(pit >> 1) & 1u) ^ 1u, abort_flag, status, 0x120u + b);
                     if (!(ok = __all_sync(0xffffffffu, ok))) break;
                     if (lane == 0) {
-                        mbar_arrive_expect_tx(bar(BAR_OPSFULL + b), 2u * TILE_T * 4u + (has_lora ? LORA_H_BYTES + LORA_B_BYTES : 0));
-                        bulk_load_1d(sbase + OFF_TOKV + b * TOKV_BYTES, p.row_sum + t0, TILE_T * 4u, bar(BAR_OPSFULL + b));
-                        bulk_load_1d(sbase + OFF_TOKV + b * TOKV_BYTES + TILE_T * 4, p.tok_sc + t0, TILE_T * 4u, bar(BAR_OPSFULL + b));
+                        mbar_arrive_expect_tx(bar(C::BAR_OPSFULL + b), 2u * TILE_T * 4u + (has_lora ? C::LORA_H_BYTES + C::LORA_B_BYTES : 0));
+                        bulk_load_1d(sbase + C::OFF_TOKV + b * TOKV_BYTES, p.row_sum + t0, TILE_T * 4u, bar(C::BAR_OPSFULL + b));
+                        bulk_load_1d(sbase + C::OFF_TOKV + b * TOKV_BYTES + TILE_T * 4, p.tok_sc + t0, TILE_T * 4u, bar(C::BAR_OPSFULL + b));
                         if (has_lora) {
-                            tma_load_2d(sbase + OFF_LH + b * LORA_H_BYTES, &tmap_h, 0, t0, bar(BAR_OPSFULL + b));
-                            tma_load_2d(sbase + OFF_LB + b * LORA_B_BYTES, &tmap_gb, 0, c0, bar(BAR_OPSFULL + b));
+                            tma_load_2d(sbase + C::OFF_LH + b * C::LORA_H_BYTES, &tmap_h, 0, t0, bar(C::BAR_OPSFULL + b));
+                            tma_load_2d(sbase + C::OFF_LB + b * C::LORA_B_BYTES, &tmap_gb, 0, c0, bar(C::BAR_OPSFULL + b));
                         }
                     }
                     ++ops_issued[b];
                     ++pit;
                 }
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    ok = mbar_wait(bar(BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x100u + s);
+                    ok = mbar_wait(bar(C::BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x100u + s);
                     if (!(ok = __all_sync(0xffffffffu, ok))) break;
                     if (lane == 0) {
                         // 256 columns of 128 tokens as two 128-byte-swizzled tiles (columns past K read as zeros),
                         // and the 1 KiB tiles (16 rows x 256 columns) of 8 consecutive row tiles
-                        mbar_arrive_expect_tx(bar(BAR_LOADED + s), X_TILE_BYTES + (uint32_t)nrt * 1024u);
-                        tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, t0, bar(BAR_LOADED + s));
-                        tma_load_2d(sbase + OFF_X + s * X_TILE_BYTES + X_HALF_BYTES, &tmap_x, kb * KBLK + 128, t0, bar(BAR_LOADED + s));
+                        mbar_arrive_expect_tx(bar(C::BAR_LOADED + s), X_TILE_BYTES + (uint32_t)nrt * 1024u);
+                        tma_load_2d(sbase + C::OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, t0, bar(C::BAR_LOADED + s));
+                        tma_load_2d(sbase + C::OFF_X + s * X_TILE_BYTES + X_HALF_BYTES, &tmap_x, kb * KBLK + 128, t0, bar(C::BAR_LOADED + s));
                     }
                     __syncwarp();
                     if (lane < nrt)
-                        bulk_load_1d(sbase + OFF_P + s * P_TILE_BYTES + lane * 1024, psrc + (size_t)kb * 1024, 1024u,
-                                     bar(BAR_LOADED + s));
+                        bulk_load_1d(sbase + C::OFF_P + s * P_TILE_BYTES + lane * 1024, psrc + (size_t)kb * 1024, 1024u,
+                                     bar(C::BAR_LOADED + s));
                     ++issued[s];
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    if (++s == C::STAGES) { s = 0; ph ^= 1u; }
                 }
             }
             // drain: wait (bounded) until every copy this warp issued has landed, so that the CTA
             // never exits with a bulk copy in flight (immediate when the consumers ran to the end)
-            for (int q = 0; q < STAGES; ++q)
+            for (int q = 0; q < C::STAGES; ++q)
                 if (issued[q]) {
                     const uint32_t par = (issued[q] - 1u) & 1u;
-                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_LOADED + q), par); ++i) {}
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(C::BAR_LOADED + q), par); ++i) {}
                 }
             for (int q = 0; q < 2; ++q)
                 if (ops_issued[q]) {
                     const uint32_t par = (ops_issued[q] - 1u) & 1u;
-                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(BAR_OPSFULL + q), par); ++i) {}
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(C::BAR_OPSFULL + q), par); ++i) {}
                 }
         }
     } else if (warp == 1) {
@@ -351,29 +360,30 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             uint32_t ph = 0;
             bool ok = true;
             int it = 0, pend = -1;  // pend: tile whose correction MMA is still to be issued
-            const uint64_t xdesc0 = make_sw128_desc(sbase + OFF_X);
+            const uint64_t xdesc0 = make_sw128_desc(sbase + C::OFF_X);
             auto issue_lora = [&](int t) {
                 const int b = t & 1;
                 tc_fence_after();
-                const uint64_t adesc = make_sw128_desc(sbase + OFF_LB + b * LORA_B_BYTES);
-                const uint64_t bdesc = make_sw128_desc(sbase + OFF_LH + b * LORA_H_BYTES);
+                const uint32_t la = sbase + C::OFF_LB + b * C::LORA_B_BYTES, lh = sbase + C::OFF_LH + b * C::LORA_H_BYTES;
+                const uint64_t adesc = OPSB == 128 ? make_sw128_desc(la) : make_sw64_desc(la);
+                const uint64_t bdesc = OPSB == 128 ? make_sw128_desc(lh) : make_sw64_desc(lh);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)  // 64 fp16 = 4 x (K = 16), on top of the fp32 values
+                for (int kk = 0; kk < OPSB / 32; ++kk)  // K = 16 fp16 (32 bytes of a row) per MMA, on top of the fp32 values
                     mma_f16(tmem_base + b * ACC_COLS, adesc + 2u * kk, bdesc + 2u * kk, IDESC_F16, 1u);
-                tc_commit(bar(BAR_LORADONE + b));
+                tc_commit(bar(C::BAR_LORADONE + b));
             };
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
                 const int b = it & 1;
                 const uint32_t acc = tmem_base + b * ACC_COLS;
-                if (it >= 2 && !(ok = mbar_wait(bar(BAR_ACCEMPTY + b), (uint32_t)((it >> 1) - 1) & 1u, abort_flag, status, 0x200u)))
+                if (it >= 2 && !(ok = mbar_wait(bar(C::BAR_ACCEMPTY + b), (uint32_t)((it >> 1) - 1) & 1u, abort_flag, status, 0x200u)))
                     break;
                 tc_fence_after();
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (pend >= 0 && mbar_try_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u)) {
+                    if (pend >= 0 && mbar_try_wait(bar(C::BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u)) {
                         issue_lora(pend);
                         pend = -1;
                     }
-                    if (!(ok = mbar_wait(bar(BAR_FULL + s), ph, abort_flag, status, 0x210u + s))) break;
+                    if (!(ok = mbar_wait(bar(C::BAR_FULL + s), ph, abort_flag, status, 0x210u + s))) break;
                     tc_fence_after();
                     const uint64_t bdesc = xdesc0 + (uint64_t)(s * (X_TILE_BYTES >> 4));
                     const uint32_t a_tmem = tmem_base + A_COL + s * A_STAGE_COLS;
@@ -387,13 +397,13 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     mma_i8_ts(acc, a_tmem + 40u, bdesc + (X_HALF_BYTES >> 4) + 2u, IDESC_I8, 1u);
                     mma_i8_ts(acc, a_tmem + 48u, bdesc + (X_HALF_BYTES >> 4) + 4u, IDESC_I8, 1u);
                     mma_i8_ts(acc, a_tmem + 56u, bdesc + (X_HALF_BYTES >> 4) + 6u, IDESC_I8, 1u);
-                    tc_commit(bar(BAR_EMPTY + s));
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    tc_commit(bar(C::BAR_EMPTY + s));
+                    if (++s == C::STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit(bar(BAR_ACCFULL + b));
+                tc_commit(bar(C::BAR_ACCFULL + b));
                 if (pend >= 0) {  // the previous tile's correction has to be out before its accumulator's next turn
-                    if (!(ok = mbar_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x230u)))
+                    if (!(ok = mbar_wait(bar(C::BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x230u)))
                         break;
                     issue_lora(pend);
                     pend = -1;
@@ -401,14 +411,14 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 if (has_lora) pend = it;
             }
             if (ok && pend >= 0 &&
-                mbar_wait(bar(BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x231u))
+                mbar_wait(bar(C::BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x231u))
                 issue_lora(pend);
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------------ epilogue warps
         const int e = warp - 2;          // staging role index
         const int q = warp & 3;          // tensor-memory lane quarter this warp may access
-        uint8_t *buf = smem + OFF_ST + e * STORE_BUF_BYTES;
+        uint8_t *buf = smem + C::OFF_ST + e * STORE_BUF_BYTES;
         bool ok = true;
         int it = 0;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
@@ -416,15 +426,15 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const int b = it & 1;
             const uint32_t par = (uint32_t)(it >> 1) & 1u;
             // the tile's row sums and scales (and the correction's operands) were fetched by the producer
-            const int *tok_rs = reinterpret_cast<const int *>(smem + OFF_TOKV + b * TOKV_BYTES);
+            const int *tok_rs = reinterpret_cast<const int *>(smem + C::OFF_TOKV + b * TOKV_BYTES);
             const float *tok_sc = reinterpret_cast<const float *>(tok_rs + TILE_T);
-            ok = mbar_wait(bar(BAR_OPSFULL + b), par, abort_flag, status, 0x320u + b);
+            ok = mbar_wait(bar(C::BAR_OPSFULL + b), par, abort_flag, status, 0x320u + b);
             if (!(ok = __all_sync(0xffffffffu, ok))) break;
 
             const int n = c0 + 32 * q + lane;  // this thread's output channel = its tensor-memory lane
             const bool n_ok = n < p.N;
 
-            ok = mbar_wait(bar(BAR_ACCFULL + b), par, abort_flag, status, 0x300u);
+            ok = mbar_wait(bar(C::BAR_ACCFULL + b), par, abort_flag, status, 0x300u);
             if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
             tc_fence_after();
             const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16) + b * ACC_COLS;
@@ -459,8 +469,8 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_LORAREADY + b));
-                ok = mbar_wait(bar(BAR_LORADONE + b), par, abort_flag, status, 0x310u);
+                if (lane == 0) mbar_arrive(bar(C::BAR_LORAREADY + b));
+                ok = mbar_wait(bar(C::BAR_LORADONE + b), par, abort_flag, status, 0x310u);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;
                 tc_fence_after();
             }
@@ -494,8 +504,8 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(bar(BAR_ACCEMPTY + b));
-                mbar_arrive(bar(BAR_OPSEMPTY + b));
+                mbar_arrive(bar(C::BAR_ACCEMPTY + b));
+                mbar_arrive(bar(C::BAR_OPSEMPTY + b));
             }
         }
         if (lane == 0) bulk_wait_read<0>();
@@ -511,11 +521,11 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             for (int kb = 0; kb < kblocks; ++kb) {
                 // the stage's packed codes have landed; and the MMAs that read this stage's previous operand
                 // are complete (the producer waited for their commit before it refilled the stage)
-                ok = mbar_wait(bar(BAR_LOADED + s), ph, abort_flag, status, 0x400u + s);
+                ok = mbar_wait(bar(C::BAR_LOADED + s), ph, abort_flag, status, 0x400u + s);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
                 // this row's 64 bytes hold the stage's 256 columns; register 4 i + j of a half = columns
                 // 16 i + 4 j .. + 3, one code per byte
-                const uint8_t *prow = smem + OFF_P + s * P_TILE_BYTES + row * 64;
+                const uint8_t *prow = smem + C::OFF_P + s * P_TILE_BYTES + row * 64;
                 const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + A_COL + s * A_STAGE_COLS;
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
@@ -532,8 +542,8 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_FULL + s));
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
+                if (lane == 0) mbar_arrive(bar(C::BAR_FULL + s));
+                if (++s == C::STAGES) { s = 0; ph ^= 1u; }
             }
         }
     }
@@ -577,9 +587,22 @@ static bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, const void *ba
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <bool OUT_BF16, int NS, int OPSB>
+static cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &mh, const CUtensorMap &mgb, const CUtensorMap &my,
+                                  const GemmParams &p, int grid, unsigned int *status, cudaStream_t stream) {
+    static bool attr_set = false;
+    constexpr int smem = Cfg<NS, OPSB>::SMEM_BYTES;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(prefill_gemm_kernel<OUT_BF16, NS, OPSB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    prefill_gemm_kernel<OUT_BF16, NS, OPSB><<<grid, GEMM_THREADS, smem, stream>>>(mx, mh, mgb, my, p, status);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
     static int sm_count = 0;
-    static bool attr_set = false;
     if (!sm_count) {
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
@@ -587,23 +610,17 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
         e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
     }
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(prefill_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
     const bool bf16 = (p.flags & HGF_FLAG_OUT_BF16) != 0;
+    const bool narrow = p.r <= 32;  // 64-byte operand rows for the correction, and room for a fourth stage
     CUtensorMap mx, mh, mgb, my;
     if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, p.xq, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.K, 128, TILE_T,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;
-    if (p.r > 0) {  // H [M][64] and (g B)^T [N][64] fp16: 128-byte rows, tiles of 128 rows, 128-byte swizzle
-        if (!make_map_2d(&mh, CU_TENSOR_MAP_DATA_TYPE_UINT16, p.h16, 64, (uint64_t)p.M, 128, 64, TILE_T, CU_TENSOR_MAP_SWIZZLE_128B))
-            return cudaErrorInvalidValue;
-        if (!make_map_2d(&mgb, CU_TENSOR_MAP_DATA_TYPE_UINT16, p.gb16, 64, (uint64_t)p.N, 128, 64, TILE_C, CU_TENSOR_MAP_SWIZZLE_128B))
-            return cudaErrorInvalidValue;
+    if (p.r > 0) {  // H [M][64] and (g B)^T [N][64] fp16: tiles of 128 rows; the first 32 or all 64 columns
+        const uint32_t cols = narrow ? 32 : 64;
+        const CUtensorMapSwizzle sw = narrow ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
+        if (!make_map_2d(&mh, CU_TENSOR_MAP_DATA_TYPE_UINT16, p.h16, 64, (uint64_t)p.M, 128, cols, TILE_T, sw)) return cudaErrorInvalidValue;
+        if (!make_map_2d(&mgb, CU_TENSOR_MAP_DATA_TYPE_UINT16, p.gb16, 64, (uint64_t)p.N, 128, cols, TILE_C, sw)) return cudaErrorInvalidValue;
     } else {
         mh = mx;
         mgb = mx;
@@ -615,12 +632,15 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
     const int grid = tiles < sm_count ? tiles : sm_count;
     unsigned int *status = device_status_word();
     if (!status) return cudaErrorMemoryAllocation;
-    if (bf16)
-        prefill_gemm_kernel<true><<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(mx, mh, mgb, my, p, status);
+    cudaError_t e;
+    if (narrow)
+        e = bf16 ? launch_variant<true, 4, 64>(mx, mh, mgb, my, p, grid, status, stream)
+                 : launch_variant<false, 4, 64>(mx, mh, mgb, my, p, grid, status, stream);
     else
-        prefill_gemm_kernel<false><<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(mx, mh, mgb, my, p, status);
+        e = bf16 ? launch_variant<true, 3, 128>(mx, mh, mgb, my, p, grid, status, stream)
+                 : launch_variant<false, 3, 128>(mx, mh, mgb, my, p, grid, status, stream);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace hgf
