@@ -15,7 +15,7 @@
 // 256 input columns (eight MMAs): every hand-over between the roles costs a shared-memory round
 // trip, and the single MMA-issuing thread can only afford one per 512 tensor-core clocks.
 //
-// One persistent CTA per SM, 10 warps with fixed roles:
+// One persistent CTA per SM, 11 warps with fixed roles:
 //   warp 0      producer (all lanes): per stage the int8 activation tile as two 128 tokens x 128 B
 //               boxes (128-byte swizzle) and the packed weights of 128 channels (eight contiguous
 //               1 KiB tiles of the tiled weight layout, one bulk copy each); per tile what its
@@ -25,6 +25,8 @@
 //               the correction MMA, read the result, transpose it through shared memory and store
 //               y with TMA
 //   warps 6-9   expand the packed tile into tensor memory
+//   warp 10     producer of the packed codes (eight contiguous 1 KiB tiles of the tiled weight layout
+//               per stage, one bulk copy each), in a ring that runs ahead of the activations'
 // Codes are c = t + 1 (both operands are declared signed 8-bit; 0, 1, 2 read the same either way);
 // sum_k t x~ = sum_k c x~ - sum_k x~ is restored in the epilogue from the row sums.
 //
@@ -45,7 +47,7 @@ constexpr int X_TILE_BYTES = 2 * X_HALF_BYTES;   // 32 KiB per stage
 constexpr int P_TILE_BYTES = TILE_C * KBLK / 4;  // 8 KiB: 8 weight tiles of 16 rows x 256 columns
 constexpr int TOKV_BYTES = TILE_T * 8;           // row sums and scales of the tile's tokens
 constexpr int STORE_BUF_BYTES = 32 * 32 * 4;     // per epilogue warp: 32 tokens x 32 channels
-constexpr int GEMM_THREADS = 320;
+constexpr int GEMM_THREADS = 352;  // 11 warps
 // tensor memory: two accumulators of 128 columns, then one weight operand of 64 columns (= 256 int8 per lane) per stage
 constexpr int TMEM_COLS = 512, ACC_COLS = TILE_T, A_COL = 2 * ACC_COLS, A_STAGE_COLS = KBLK / 4;
 
@@ -56,17 +58,19 @@ constexpr int TMEM_COLS = 512, ACC_COLS = TILE_T, A_COL = 2 * ACC_COLS, A_STAGE_
 template <int NS, int OPSB>
 struct Cfg {
     static constexpr int STAGES = NS;
+    static constexpr int PSTAGES = NS + 1;  // the packed codes run one stage further ahead than the activations
     static constexpr int LORA_H_BYTES = TILE_T * OPSB, LORA_B_BYTES = TILE_C * OPSB;
     static constexpr int OFF_X = 0;
     static constexpr int OFF_LH = OFF_X + NS * X_TILE_BYTES;
     static constexpr int OFF_LB = OFF_LH + 2 * LORA_H_BYTES;  // the epilogue's operands are double-buffered like the accumulators
     static constexpr int OFF_P = OFF_LB + 2 * LORA_B_BYTES;
-    static constexpr int OFF_TOKV = OFF_P + NS * P_TILE_BYTES;
+    static constexpr int OFF_TOKV = OFF_P + PSTAGES * P_TILE_BYTES;
     static constexpr int OFF_ST = OFF_TOKV + 2 * TOKV_BYTES;
     static constexpr int OFF_BAR = OFF_ST + 4 * STORE_BUF_BYTES;
     static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;  // + slack for the 1024-byte alignment of the base
     // barrier slots (8 bytes each) inside the OFF_BAR block
-    static constexpr int BAR_FULL = 0, BAR_EMPTY = BAR_FULL + NS, BAR_LOADED = BAR_EMPTY + NS, BAR_ACCFULL = BAR_LOADED + NS,
+    static constexpr int BAR_FULL = 0, BAR_EMPTY = BAR_FULL + NS, BAR_PFULL = BAR_EMPTY + NS, BAR_PEMPTY = BAR_PFULL + PSTAGES,
+                         BAR_ACCFULL = BAR_PEMPTY + PSTAGES,
                          BAR_ACCEMPTY = BAR_ACCFULL + 2, BAR_LORAREADY = BAR_ACCEMPTY + 2, BAR_LORADONE = BAR_LORAREADY + 2,
                          BAR_OPSFULL = BAR_LORADONE + 2, BAR_OPSEMPTY = BAR_OPSFULL + 2, BAR_COUNT = BAR_OPSEMPTY + 2;
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
@@ -251,14 +255,20 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
-            // LOADED: the stage's activation tile and packed codes have landed (producer's arrival + bytes).
-            // FULL: the four unpack warps have seen LOADED and put the weight operand into tensor memory,
-            // so the MMA thread waits on this one barrier only (it is a single thread and every barrier
-            // operation costs it a shared-memory round trip).  EMPTY: the MMAs that read the stage are
-            // complete (one commit; the producer and the unpack warps both wait on it).
-            mbar_init(bar(C::BAR_LOADED + s), 1);
-            mbar_init(bar(C::BAR_FULL + s), 4);
+            // FULL: the stage's activation tile has landed (producer's arrival + bytes) and the four unpack
+            // warps have put the weight operand into tensor memory, so the MMA thread waits on this one
+            // barrier only (it is a single thread and every barrier operation costs it a shared-memory
+            // round trip).  EMPTY: the MMAs that read the stage are complete (one commit; the producer
+            // and the unpack warps both wait on it).
+            mbar_init(bar(C::BAR_FULL + s), 1 + 4);
             mbar_init(bar(C::BAR_EMPTY + s), 1);
+        }
+        for (int j = 0; j < C::PSTAGES; ++j) {
+            // the packed codes have a ring of their own, filled ahead of the activations: the expansion into
+            // tensor memory then starts the moment a stage's MMAs are complete, in parallel with the reload
+            // of the activation tile, instead of after it
+            mbar_init(bar(C::BAR_PFULL + j), 1);
+            mbar_init(bar(C::BAR_PEMPTY + j), 4);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(C::BAR_ACCFULL + b), 1);
@@ -294,12 +304,8 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             uint32_t issued[C::STAGES] = {}, ops_issued[2] = {};
             int pit = 0;
             bool ok = true;
-            const int steps = (p.K + 255) >> 8, n_row_tiles = (p.N + 15) >> 4;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                 const int t0 = (tile % tiles_t) * TILE_T, c0 = (tile / tiles_t) * TILE_C;
-                const int rt0 = c0 >> 4, nrt = n_row_tiles - rt0 < TILE_C / 16 ? n_row_tiles - rt0 : TILE_C / 16;
-                // this lane's weight tile of column tile 0 (row tiles past the matrix are left out)
-                const uint8_t *psrc = p.packed + (size_t)(rt0 + (lane < nrt ? lane : 0)) * steps * 1024;
                 {
                     // what the tile's epilogue needs, into the buffer of the tile's accumulator: row sums and
                     // scales of the 128 tokens, and with a correction the H tile and the (g B)^T tile
@@ -322,16 +328,11 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     ok = mbar_wait(bar(C::BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x100u + s);
                     if (!(ok = __all_sync(0xffffffffu, ok))) break;
                     if (lane == 0) {
-                        // 256 columns of 128 tokens as two 128-byte-swizzled tiles (columns past K read as zeros),
-                        // and the 1 KiB tiles (16 rows x 256 columns) of 8 consecutive row tiles
-                        mbar_arrive_expect_tx(bar(C::BAR_LOADED + s), X_TILE_BYTES + (uint32_t)nrt * 1024u);
-                        tma_load_2d(sbase + C::OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, t0, bar(C::BAR_LOADED + s));
-                        tma_load_2d(sbase + C::OFF_X + s * X_TILE_BYTES + X_HALF_BYTES, &tmap_x, kb * KBLK + 128, t0, bar(C::BAR_LOADED + s));
+                        // 256 columns of 128 tokens as two 128-byte-swizzled tiles (columns past K read as zeros)
+                        mbar_arrive_expect_tx(bar(C::BAR_FULL + s), X_TILE_BYTES);
+                        tma_load_2d(sbase + C::OFF_X + s * X_TILE_BYTES, &tmap_x, kb * KBLK, t0, bar(C::BAR_FULL + s));
+                        tma_load_2d(sbase + C::OFF_X + s * X_TILE_BYTES + X_HALF_BYTES, &tmap_x, kb * KBLK + 128, t0, bar(C::BAR_FULL + s));
                     }
-                    __syncwarp();
-                    if (lane < nrt)
-                        bulk_load_1d(sbase + C::OFF_P + s * P_TILE_BYTES + lane * 1024, psrc + (size_t)kb * 1024, 1024u,
-                                     bar(C::BAR_LOADED + s));
                     ++issued[s];
                     if (++s == C::STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -341,7 +342,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             for (int q = 0; q < C::STAGES; ++q)
                 if (issued[q]) {
                     const uint32_t par = (issued[q] - 1u) & 1u;
-                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(C::BAR_LOADED + q), par); ++i) {}
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(C::BAR_FULL + q), par); ++i) {}
                 }
             for (int q = 0; q < 2; ++q)
                 if (ops_issued[q]) {
@@ -510,22 +511,54 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
         if (lane == 0) bulk_wait_read<0>();
         __syncwarp();
+    } else if (warp == 10) {
+        // ------------------------------------------------------------------ packed-code producer
+        // Its own warp and ring: the codes run ahead of the activations, so the expansion into tensor
+        // memory starts the moment a stage's MMAs are complete, in parallel with the reload of the
+        // activation tile.  Per stage the 1 KiB tiles (16 rows x 256 columns) of 8 consecutive row tiles,
+        // one bulk copy per lane (row tiles past the matrix are left out).
+        int pj = 0;
+        uint32_t pph = 0;
+        uint32_t pissued[C::PSTAGES] = {};
+        bool ok = true;
+        const int steps = (p.K + 255) >> 8, n_row_tiles = (p.N + 15) >> 4;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            const int rt0 = ((tile / tiles_t) * TILE_C) >> 4;
+            const int nrt = n_row_tiles - rt0 < TILE_C / 16 ? n_row_tiles - rt0 : TILE_C / 16;
+            const uint8_t *psrc = p.packed + (size_t)(rt0 + (lane < nrt ? lane : 0)) * steps * 1024;
+            for (int kb = 0; kb < kblocks; ++kb) {
+                ok = mbar_wait(bar(C::BAR_PEMPTY + pj), pph ^ 1u, abort_flag, status, 0x110u + pj);
+                if (!(ok = __all_sync(0xffffffffu, ok))) break;
+                if (lane == 0) mbar_arrive_expect_tx(bar(C::BAR_PFULL + pj), (uint32_t)nrt * 1024u);
+                __syncwarp();
+                if (lane < nrt)
+                    bulk_load_1d(sbase + C::OFF_P + pj * P_TILE_BYTES + lane * 1024, psrc + (size_t)kb * 1024, 1024u, bar(C::BAR_PFULL + pj));
+                ++pissued[pj];
+                if (++pj == C::PSTAGES) { pj = 0; pph ^= 1u; }
+            }
+        }
+        for (int q = 0; q < C::PSTAGES; ++q)
+            if (pissued[q]) {
+                const uint32_t par = (pissued[q] - 1u) & 1u;
+                for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(C::BAR_PFULL + q), par); ++i) {}
+            }
     } else {
         // ------------------------------------------------------------------ unpack warps
         const int q = warp & 3;              // tensor-memory lane quarter this warp may access
         const int row = 32 * q + lane;       // this thread's channel row of the tile = its tensor-memory lane
-        int s = 0;
-        uint32_t ph = 0;
+        int s = 0, pj = 0;
+        uint32_t ph = 0, pph = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < kblocks; ++kb) {
-                // the stage's packed codes have landed; and the MMAs that read this stage's previous operand
-                // are complete (the producer waited for their commit before it refilled the stage)
-                ok = mbar_wait(bar(C::BAR_LOADED + s), ph, abort_flag, status, 0x400u + s);
+                // the stage's packed codes have landed, and the MMAs that read this stage's previous operand
+                // are complete
+                ok = mbar_wait(bar(C::BAR_PFULL + pj), pph, abort_flag, status, 0x400u + pj) &&
+                     mbar_wait(bar(C::BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x410u + s);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the whole warp leaves together
                 // this row's 64 bytes hold the stage's 256 columns; register 4 i + j of a half = columns
                 // 16 i + 4 j .. + 3, one code per byte
-                const uint8_t *prow = smem + C::OFF_P + s * P_TILE_BYTES + row * 64;
+                const uint8_t *prow = smem + C::OFF_P + pj * P_TILE_BYTES + row * 64;
                 const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + A_COL + s * A_STAGE_COLS;
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
@@ -542,7 +575,11 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(C::BAR_FULL + s));
+                if (lane == 0) {
+                    mbar_arrive(bar(C::BAR_FULL + s));
+                    mbar_arrive(bar(C::BAR_PEMPTY + pj));
+                }
+                if (++pj == C::PSTAGES) { pj = 0; pph ^= 1u; }
                 if (++s == C::STAGES) { s = 0; ph ^= 1u; }
             }
         }
