@@ -391,6 +391,17 @@ def run_extra(hgf, torch, syn, stream, args, peaks):
                                      "frac_2x_measured_bf16": tops / int8_peak_2x_bf16})
             del w
             torch.cuda.empty_cache()
+    # config 4 prefill: the seven projections of one 7B-class block at M = 4096 (the stack is 32 such blocks)
+    blk = Workload(hgf, torch, syn.CONFIGS[4]["layers"], 4096, 1, flags=hgf.FLAG_OUT_BF16)
+    blk.capture(stream)
+    ms = blk.time_steps(stream, 20, args.warmup)
+    extra["prefill_config4_block"] = {"workload": "config4 7B-class block (7 projections, r=64), prefill M=4096, bf16 y",
+                                      "ms_per_block": ms, "TOPS": blk.ops / (ms * 1e-3) / 1e12,
+                                      "frac_nominal_4500": blk.ops / (ms * 1e-3) / 1e12 / int8_peak_nominal,
+                                      "frac_2x_measured_bf16": blk.ops / (ms * 1e-3) / 1e12 / int8_peak_2x_bf16,
+                                      "prefill_tokens_per_s_32_blocks": 4096 / (32 * ms * 1e-3)}
+    del blk
+    torch.cuda.empty_cache()
     return extra
 
 
