@@ -371,13 +371,18 @@ decode_prologue_group_kernel(const QuantItem *quant_items, int n_quant, const Lo
         d0 = reinterpret_cast<const uint4 *>(lora + gw)[0];
         d1 = reinterpret_cast<const uint4 *>(lora + gw)[1];
     }
-    pdl_wait();  // x, and the scratch this kernel overwrites, belong to earlier work
-
     // LoRA items are dealt from the first warp up, quantisation items from the last warp down, so the
     // warps with one LoRA item fewer take the rows
-    for (int i = nw - 1 - gw; i < n_quant; i += nw) {
-        const QuantItem q = quant_items[i];
+    const int q_first = nw - 1 - gw;
+    QuantItem q = {nullptr, nullptr, nullptr, nullptr, 0, 0};
+    if (q_first < n_quant) q = quant_items[q_first];
+    pdl_wait();  // x, and the scratch this kernel overwrites, belong to earlier work
+
+    for (int i = q_first; i < n_quant; i += nw) {
+        QuantItem q_next = q;
+        if (i + nw < n_quant) q_next = quant_items[i + nw];  // travels while this row is worked on
         warp_quant_row(q, buf - 16 * lane, pg_smem + warp * kWarpBytes, kWarpBytes, lane);
+        q = q_next;
     }
 
     for (int i = gw; i < n_lora; i += nw) {
