@@ -154,7 +154,7 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
         dl.probs = nullptr;
         dl.n_probs = 1;
         dl.total_tiles = (int)row_tiles(d_out);
-        dl.total_cost = (long long)dl.total_tiles * (long long)(padded_k(d_in) / 256);
+        dl.total_cost = (long long)dl.total_tiles * row_tile_cost((int)d_in);
         dl.max_M = (int)M;
         dl.xq_smem_bytes = decode_xq_smem_bytes((int)M, (int)d_in);
         return launch_decode_gemv(dl, &dp, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
@@ -314,7 +314,7 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
             hpart += (size_t)jts * slices * 8 * 32;
         }
         tiles += (int)row_tiles(q.d_out);
-        cost += (long long)row_tiles(q.d_out) * (long long)(padded_k(q.d_in) / 256);
+        cost += (long long)row_tiles(q.d_out) * row_tile_cost((int)q.d_in);
         blocks += (int)q.M + ranks[i] / 16;
         max_M = q.M > max_M ? (int)q.M : max_M;
         const int xb = decode_xq_smem_bytes((int)q.M, (int)q.d_in);
@@ -343,7 +343,7 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
                 const int mid = (lo + hi + 1) >> 1;
                 if (dps[mid].cost_begin <= c) lo = mid; else hi = mid - 1;
             }
-            const long long steps = padded_k(dps[lo].K) / 256, tl = row_tiles(dps[lo].N);
+            const long long steps = row_tile_cost(dps[lo].K), tl = row_tiles(dps[lo].N);
             long long local = (c - dps[lo].cost_begin + steps - 1) / steps;
             if (local > tl) local = tl;
             *prob = lo;

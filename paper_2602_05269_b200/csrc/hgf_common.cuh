@@ -91,8 +91,15 @@ struct GemmPrologueExtra {
     int N;
 };
 
+// Cost of one 16-row tile of a decode problem, the unit in which a launch is cut into equal shares:
+// its 1 KiB weight tiles, plus what the switch to the row tile and its epilogue take, counted in
+// weight tiles (measured: a layer with short rows runs slower per byte than one with long rows by
+// about this much per row tile).
+constexpr int kRowTileOverhead = 6;
+__host__ __device__ inline long long row_tile_cost(int K) { return (long long)((K + 255) >> 8) + kRowTileOverhead; }
+
 // One layer problem of a decode launch (M <= 16).  tile_begin = index of its first 16-row tile in
-// the launch-wide tile numbering; cost_begin = number of 1 KiB weight tiles of all earlier problems.
+// the launch-wide tile numbering; cost_begin = sum of the costs of all row tiles of earlier problems.
 struct DecodeProblem {
     const uint8_t *packed;   // tiled layout, see above
     const int8_t *xq;        // [M][K]
@@ -117,7 +124,7 @@ struct DecodeLaunch {
     const DecodeProblem *probs;  // device array, or null for a single problem passed by value
     int n_probs;
     int total_tiles;
-    long long total_cost;        // 1 KiB weight tiles of all problems
+    long long total_cost;        // cost of all row tiles of all problems
     int max_M;                   // largest token count of any problem
     int xq_smem_bytes;           // shared memory for the largest problem's activations
     int ring_slots;              // weight-ring slots per warp (set by the launcher)

@@ -4,8 +4,8 @@
 //
 // The kernel is bound by the packed-weight stream from HBM, so it is built around keeping that
 // stream busy.  One persistent CTA of 16 warps per SM.  The weights of all problems of the launch
-// form one long sequence of 1 KiB tiles (16 output rows x 256 input columns); it is cut into equal
-// contiguous shares, one per CTA.  Every warp owns a private ring of 1 KiB shared-memory slots
+// form one long sequence of 1 KiB tiles (16 output rows x 256 input columns); it is cut into
+// contiguous shares of equal cost (weight tiles plus a fixed charge per row tile), one per CTA.  Every warp owns a private ring of 1 KiB shared-memory slots
 // that one of its lanes keeps filled with bulk asynchronous copies (cp.async.bulk, completion on an
 // mbarrier), several tiles ahead of their use and across row-tile, layer and (under programmatic
 // dependent launch) kernel boundaries, so the number of bytes in flight does not depend on what
@@ -142,7 +142,7 @@ __device__ __forceinline__ const DecodeProblem &problem_of(const DecodeLaunch &L
 __device__ __forceinline__ int steps_of(int K) { return (K + 255) >> 8; }
 __device__ __forceinline__ int tiles_of(int N) { return (N + 15) >> 4; }
 
-// Smallest launch-wide tile index whose first 1 KiB tile has sequence number >= cost.
+// Smallest launch-wide tile index at which the cost of all earlier row tiles is >= cost.
 __device__ int tile_of_cost(const DecodeLaunch &L, const DecodeProblem &single, long long cost) {
     int lo = 0, hi = L.n_probs - 1;
     while (lo < hi) {  // last problem with cost_begin <= cost
@@ -150,7 +150,8 @@ __device__ int tile_of_cost(const DecodeLaunch &L, const DecodeProblem &single, 
         if (problem_of(L, single, mid).cost_begin <= cost) lo = mid; else hi = mid - 1;
     }
     const DecodeProblem &P = problem_of(L, single, lo);
-    const int steps = steps_of(P.K), tiles = tiles_of(P.N);
+    const long long steps = row_tile_cost(P.K);
+    const int tiles = tiles_of(P.N);
     long long local = (cost - P.cost_begin + steps - 1) / steps;
     if (local > tiles) local = tiles;
     return P.tile_begin + (int)local;
@@ -361,7 +362,13 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
                     const int idx = 4 * (m >> 3) + 2 * (jl >> 3) + (m & 1), ln = 4 * (jl & 7) + ((m & 7) >> 1);
                     const float *src = hp + ((size_t)jt * ns * 8 + idx) * 32 + ln;
                     float z = 0.0f;
-                    for (int sl = 0; sl < ns; ++sl) z += __ldcg(src + (size_t)sl * 256);
+                    int sl = 0;
+                    for (; sl + 4 <= ns; sl += 4) {  // four loads in flight, added in slice order
+                        const float z0 = __ldcg(src + (size_t)sl * 256), z1 = __ldcg(src + (size_t)(sl + 1) * 256);
+                        const float z2 = __ldcg(src + (size_t)(sl + 2) * 256), z3 = __ldcg(src + (size_t)(sl + 3) * 256);
+                        z += z0; z += z1; z += z2; z += z3;
+                    }
+                    for (; sl < ns; ++sl) z += __ldcg(src + (size_t)sl * 256);
                     const float h = no_silu ? z : silu_f(z);
                     const __half hi = __float2half_rn(h);
                     sm.h_hi[m][j] = hi;
