@@ -157,6 +157,7 @@ cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_q
                                          const LoraItem *d_lora_items, int n_lora, int max_M, bool pdl,
                                          cudaStream_t stream);
 cudaError_t launch_lora_down_gemm(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream);
+cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream);
 cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream);
 // Shared memory the decode kernel needs for one problem's activations, and the largest it accepts.
 int decode_xq_smem_bytes(int M, int K);

@@ -39,8 +39,8 @@ __device__ __forceinline__ int quant1_div(float x, float gamma) {
 // q gamma each have at most 15 significant bits), and the exact quotient is q + residual / gamma:
 // off a tie the candidate is always right (checked over every pair of bf16 mantissas and every
 // exponent gap in exact arithmetic), so it stands unless 2 |residual| = gamma with q odd: a tie goes
-// to the even neighbour, one step towards the residual's sign.  No F2I / FRND: those run at an
-// eighth of the FMA rate and bounded the quantisation kernels.
+// to the even neighbour, one step towards the residual's sign (2 |residual| > gamma cannot occur).
+// No F2I / FRND: those run at an eighth of the FMA rate and bounded the quantisation kernels.
 struct QuantScale {
     float gamma, half_gamma, inv127;  // inv127 = 127 / gamma
     bool fast;                        // gamma is a bf16 value
@@ -52,16 +52,6 @@ __device__ __forceinline__ QuantScale make_quant_scale(float gamma) {
     s.inv127 = __fdiv_rn(127.0f, gamma);
     s.fast = (__float_as_uint(gamma) & 0xffffu) == 0u;
     return s;
-}
-__device__ __forceinline__ int quant1_fast(float x, const QuantScale &s) {
-    constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: integers in [-2^22, 2^22] sit in the mantissa
-    const float tm = fmaf(x, s.inv127, kMagic);
-    int qi = __float_as_int(tm) - 0x4B400000;
-    const float q = tm - kMagic;
-    const float res = fmaf(-q, s.gamma, 127.0f * x);
-    const float ar = fabsf(res);
-    if (ar == s.half_gamma && (qi & 1)) qi += res > 0.0f ? 1 : -1;  // (2 |residual| > gamma cannot occur)
-    return qi;
 }
 // Largest magnitude of the eight bf16 values of a 16-byte unit, on the bit patterns: without the sign
 // bit a bf16 pattern orders like its magnitude, so a packed 16-bit maximum does two values at a time.
@@ -75,23 +65,45 @@ __device__ __forceinline__ float absmax_bits_to_float(uint32_t acc) {
     const uint32_t hi = acc >> 16, lo = acc & 0xffffu;
     return __uint_as_float((hi > lo ? hi : lo) << 16);
 }
-__device__ __forceinline__ int quant1(float x, const QuantScale &s);
 // The eight values of a 16-byte unit -> eight int8 (two words), their sum added to `sum`.
+// The fast form, arranged for throughput: the candidate's low byte is already the low
+// byte of the magic-constant sum's bit pattern (its mantissa holds 2^22 + q in two's complement), so
+// the bytes are packed straight from those patterns, and the tie test of all eight values is one
+// predicate; only a unit that holds an exact tie (rare) goes back over its values to move the odd
+// candidates to their even neighbours.
 __device__ __forceinline__ uint2 quant8(const uint4 &v, const QuantScale &s, int &sum) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t b[8];
+    if (s.fast) {
+        constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23
+        float xf[8], res[8];
+        bool tie = false;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            xf[e] = (e & 1) ? bf16hi_to_float(w[e >> 1]) : bf16lo_to_float(w[e >> 1]);
+            const float tm = fmaf(xf[e], s.inv127, kMagic);
+            res[e] = fmaf(kMagic - tm, s.gamma, 127.0f * xf[e]);  // 127 x - q gamma, exact
+            tie = tie || fabsf(res[e]) == s.half_gamma;
+            b[e] = __float_as_uint(tm);
+        }
+        if (tie) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                if (fabsf(res[e]) == s.half_gamma && (b[e] & 1u)) b[e] += res[e] > 0.0f ? 1u : 0xffffffffu;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            b[e] = (uint32_t)quant1_div((e & 1) ? bf16hi_to_float(w[e >> 1]) : bf16lo_to_float(w[e >> 1]), s.gamma);
+    }
     uint32_t o[2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        const int q0 = quant1(bf16lo_to_float(w[2 * h]), s), q1 = quant1(bf16hi_to_float(w[2 * h]), s);
-        const int q2 = quant1(bf16lo_to_float(w[2 * h + 1]), s), q3 = quant1(bf16hi_to_float(w[2 * h + 1]), s);
-        const uint32_t p01 = __byte_perm((uint32_t)q0, (uint32_t)q1, 0x0040), p23 = __byte_perm((uint32_t)q2, (uint32_t)q3, 0x0040);
+        const uint32_t p01 = __byte_perm(b[4 * h], b[4 * h + 1], 0x0040), p23 = __byte_perm(b[4 * h + 2], b[4 * h + 3], 0x0040);
         o[h] = __byte_perm(p01, p23, 0x5410);
         sum = __dp4a((int)o[h], 0x01010101, sum);
     }
     return make_uint2(o[0], o[1]);
-}
-__device__ __forceinline__ int quant1(float x, const QuantScale &s) {
-    return s.fast ? quant1_fast(x, s) : quant1_div(x, s.gamma);
 }
 
 // One block quantises one token row.
@@ -563,6 +575,249 @@ __global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const Prolog
             if (m < M) p.h16[(size_t)m * 64 + j] = __float2half_rn(0.0f);
         }
     }
+}
+
+// ---- GEMM-path prologue in one kernel -------------------------------------------------------------
+// Quantisation (Algorithm 1, steps 1-2) and the LoRA down-projection (steps 5-6) of a block of 32
+// tokens, reading x from HBM once.  First pass: x and the rows of A^T travel through a three-stage
+// ring of 256-column chunks (16-byte asynchronous copies); every warp takes 32 columns of a chunk,
+// feeds them to the tf32 MMA (tokens are the 16-row operand, 8 columns of H the 8-column operand;
+// bf16 and fp16 values are exact in tf32) and, since every element of x passes through exactly one
+// lane's registers on the way, keeps the running maximum of |x| of its rows.  Then the warps' partial
+// sums of x A are added in a fixed order, and the block's rows - still in L2 - are read again and
+// rounded with the now known scales.  JT = r / 8 column tiles of H; JT = 0 quantises only.
+constexpr int kFpThreads = 256;
+constexpr int kFpWarps = kFpThreads / 32;
+constexpr int kFpTokens = 32;
+constexpr int kFpChunk = 256;                        // columns per stage
+constexpr int kFpPitch = kFpChunk * 2 + 64;          // bytes per staged row: neighbouring rows on the other 16 banks
+constexpr int kFpStages = 3;
+__host__ __device__ constexpr int fp_stage_bytes(int r) { return (kFpTokens + r) * kFpPitch; }
+__host__ __device__ constexpr int fp_smem_bytes(int r) {
+    return kFpStages * fp_stage_bytes(r) > kFpWarps * kFpTokens * r * 4 ? kFpStages * fp_stage_bytes(r)
+                                                                         : kFpWarps * kFpTokens * r * 4;
+}
+
+template <int JT>
+__global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const PrologueParams p, const GemmPrologueExtra x) {
+    extern __shared__ __align__(128) uint8_t fp_smem[];
+    __shared__ float s_amax[kFpWarps][kFpTokens];
+    __shared__ float s_gamma[kFpTokens];
+    constexpr int r = 8 * JT;
+    const int token_blocks = (p.M + kFpTokens - 1) / kFpTokens;
+    if ((int)blockIdx.x >= token_blocks) {
+        // the remaining blocks prepare the up-projection's operand: row n of B^T times its channel's
+        // gate, fp16, padded to 64 columns (one 16-byte piece per thread)
+        if constexpr (JT > 0) {
+            const int idx = ((int)blockIdx.x - token_blocks) * kFpThreads + (int)threadIdx.x, n = idx >> 3, c = idx & 7;
+            if (n < x.N) {
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (c * 8 < r) {
+                    v = *reinterpret_cast<const uint4 *>(x.Bt + (size_t)n * r + c * 8);
+                    const float g = x.gate[n];
+                    __half2 *h2 = reinterpret_cast<__half2 *>(&v);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 f = __half22float2(h2[k]);
+                        h2[k] = __floats2half2_rn(g * f.x, g * f.y);
+                    }
+                }
+                *reinterpret_cast<uint4 *>(x.gb16 + (size_t)n * 64 + c * 8) = v;
+            }
+        }
+        return;
+    }
+    const int K = p.K, M = p.M;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    const int m0 = blockIdx.x * kFpTokens;
+    const uint32_t smem_u32 = (uint32_t)__cvta_generic_to_shared(fp_smem);
+    constexpr int kStage = fp_stage_bytes(r);
+    const int nchunks = (K + kFpChunk - 1) / kFpChunk;
+
+    // one chunk into one stage: 32 (+ r) rows of 32 16-byte units; rows past M and columns past K are zeros
+    auto fetch = [&](int c, int stage) {
+        const uint32_t dst0 = smem_u32 + stage * kStage;
+        const int k0 = c * kFpChunk;
+        for (int u = tid; u < (kFpTokens + r) * 32; u += kFpThreads) {
+            const int row = u >> 5, unit = u & 31, k = k0 + 8 * unit;
+            const void *src;
+            bool in = k < K;
+            if (row < kFpTokens) {
+                in = in && m0 + row < M;
+                src = p.x + (size_t)(in ? m0 + row : 0) * K + (in ? k : 0);
+            } else {
+                src = p.At + (size_t)(row - kFpTokens) * K + (in ? k : 0);
+            }
+            cp_async_16(dst0 + row * kFpPitch + 16 * unit, src, in ? 16u : 0u);
+        }
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+    };
+
+    float acc[2][JT > 0 ? JT : 1][4];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < (JT > 0 ? JT : 1); ++b)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.0f;
+    uint32_t amax[2][2] = {{0u, 0u}, {0u, 0u}};  // rows 16 mt + 8 hh + g, packed maxima of the bit patterns
+
+#pragma unroll
+    for (int sg = 0; sg < kFpStages - 1; ++sg) {
+        if (sg < nchunks) fetch(sg, sg);
+        else asm volatile("cp.async.commit_group;\n" ::: "memory");
+    }
+    for (int c = 0; c < nchunks; ++c) {
+        asm volatile("cp.async.wait_group %0;\n" ::"n"(kFpStages - 2) : "memory");
+        __syncthreads();  // chunk c has landed for every thread, and everyone is done with chunk c - 1
+        if (c + kFpStages - 1 < nchunks) fetch(c + kFpStages - 1, (c + kFpStages - 1) % kFpStages);
+        else asm volatile("cp.async.commit_group;\n" ::: "memory");
+
+        const uint32_t st = smem_u32 + (c % kFpStages) * kStage + 64 * warp + 16 * t;
+        uint4 xa[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                xa[mt][hh] = pg_lds_u4(st + (16 * mt + 8 * hh + g) * kFpPitch);
+                amax[mt][hh] = absmax8_bits(amax[mt][hh], xa[mt][hh]);
+            }
+        if constexpr (JT > 0) {
+#pragma unroll
+            for (int jt = 0; jt < JT; ++jt) {
+                const uint4 a4 = pg_lds_u4(st + (kFpTokens + 8 * jt + g) * kFpPitch);
+                const uint32_t aw[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    // elements 2 i and 2 i + 1 of this lane's eight take the k slots t and t + 4 of the MMA
+                    const float2 bf = __half22float2(*reinterpret_cast<const __half2 *>(&aw[i]));
+                    const uint32_t b0 = __float_as_uint(bf.x), b1 = __float_as_uint(bf.y);
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt) {
+                        const uint32_t x0 = (&xa[mt][0].x)[i], x1 = (&xa[mt][1].x)[i];
+                        mma_tf32(acc[mt][jt], x0 << 16, x1 << 16, x0 & 0xffff0000u, x1 & 0xffff0000u, b0, b1);
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("cp.async.wait_all;\n" ::: "memory");
+
+    // the rows' maxima: over the four lanes that share a row, then over the warps
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            float a = absmax_bits_to_float(amax[mt][hh]);
+            a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+            a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
+            if (t == 0) s_amax[warp][16 * mt + 8 * hh + g] = a;
+        }
+    __syncthreads();  // also: every warp is done with the ring, which the partial sums now reuse
+    if (tid < kFpTokens) {
+        float a = s_amax[0][tid];
+#pragma unroll
+        for (int w = 1; w < kFpWarps; ++w) a = fmaxf(a, s_amax[w][tid]);
+        s_gamma[tid] = fmaxf(a, 1e-5f);
+    }
+    if constexpr (JT > 0) {
+        float *s_acc = reinterpret_cast<float *>(fp_smem);  // [warps][32 tokens][r]
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int jt = 0; jt < JT; ++jt) {
+                float *base = s_acc + ((size_t)warp * kFpTokens + 16 * mt) * r + 8 * jt;
+                base[g * r + 2 * t] = acc[mt][jt][0];
+                base[g * r + 2 * t + 1] = acc[mt][jt][1];
+                base[(g + 8) * r + 2 * t] = acc[mt][jt][2];
+                base[(g + 8) * r + 2 * t + 1] = acc[mt][jt][3];
+            }
+    }
+    __syncthreads();
+    if constexpr (JT > 0) {
+        const float *s_acc = reinterpret_cast<const float *>(fp_smem);
+        for (int e = tid; e < kFpTokens * r; e += kFpThreads) {
+            const int ml = e / r, j = e % r, m = m0 + ml;
+            float z = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kFpWarps; ++w) z += s_acc[w * kFpTokens * r + e];
+            const float h = (p.flags & HGF_FLAG_NO_SILU) ? z : silu_f(z);
+            if (m < M) {
+                p.h[(size_t)m * r + j] = h;
+                if (p.dbg_h) p.dbg_h[(size_t)m * r + j] = h;
+                if (p.h16) p.h16[(size_t)m * 64 + j] = __float2half_rn(h);
+            }
+        }
+        if constexpr (JT < 8) {  // zero padding of the fp16 copy up to 64 columns
+            if (p.h16)
+                for (int e = tid; e < kFpTokens * (64 - r); e += kFpThreads) {
+                    const int ml = e / (64 - r), j = r + e % (64 - r), m = m0 + ml;
+                    if (m < M) p.h16[(size_t)m * 64 + j] = __float2half_rn(0.0f);
+                }
+        }
+    }
+
+    // second pass: each warp rounds four of the block's rows
+    const int nv = K / 8;
+#pragma unroll 1
+    for (int rr = 0; rr < kFpTokens / kFpWarps; ++rr) {
+        const int ml = warp * (kFpTokens / kFpWarps) + rr, m = m0 + ml;
+        if (m >= M) break;
+        const float gm = s_gamma[ml];
+        const QuantScale qs = make_quant_scale(gm);
+        const uint4 *xv = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K);
+        uint2 *qv = reinterpret_cast<uint2 *>(p.xq + (size_t)m * K);
+        uint2 *dq = p.dbg_xq ? reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * K) : nullptr;
+        int sum = 0;
+        int i = lane;
+        for (; i + 96 < nv; i += 128) {  // four units in flight per lane
+            const uint4 v0 = xv[i], v1 = xv[i + 32], v2 = xv[i + 64], v3 = xv[i + 96];
+            const uint2 o0 = quant8(v0, qs, sum), o1 = quant8(v1, qs, sum), o2 = quant8(v2, qs, sum), o3 = quant8(v3, qs, sum);
+            qv[i] = o0; qv[i + 32] = o1; qv[i + 64] = o2; qv[i + 96] = o3;
+            if (dq) { dq[i] = o0; dq[i + 32] = o1; dq[i + 64] = o2; dq[i + 96] = o3; }
+        }
+        for (; i < nv; i += 32) {
+            const uint2 o = quant8(xv[i], qs, sum);
+            qv[i] = o;
+            if (dq) dq[i] = o;
+        }
+        sum = warp_sum_i(sum);
+        if (lane == 0) {
+            if (p.row_sum) p.row_sum[m] = sum;
+            if (x.tok_sc) x.tok_sc[m] = gm * x.gw_over_127;
+            p.gamma_x[m] = gm;
+            if (p.dbg_gamma_x) p.dbg_gamma_x[m] = gm;
+        }
+    }
+}
+
+template <int JT>
+static cudaError_t launch_gemm_prologue_jt(const PrologueParams &p, const GemmPrologueExtra &x, int blocks, cudaStream_t stream) {
+    constexpr int smem = fp_smem_bytes(8 * JT);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_prologue_kernel<JT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    gemm_prologue_kernel<JT><<<blocks, kFpThreads, smem, stream>>>(p, x);
+    return cudaGetLastError();
+}
+
+// Quantisation and (r > 0) LoRA down-projection of the GEMM path, plus gate * B^T for its epilogue.
+cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
+    const int blocks = (p.M + kFpTokens - 1) / kFpTokens + ((p.r > 0 && x.gb16) ? (x.N * 8 + kFpThreads - 1) / kFpThreads : 0);
+    cudaError_t e;
+    switch (p.r) {
+        case 0: e = launch_gemm_prologue_jt<0>(p, x, blocks, stream); break;
+        case 16: e = launch_gemm_prologue_jt<2>(p, x, blocks, stream); break;
+        case 32: e = launch_gemm_prologue_jt<4>(p, x, blocks, stream); break;
+        case 48: e = launch_gemm_prologue_jt<6>(p, x, blocks, stream); break;
+        case 64: e = launch_gemm_prologue_jt<8>(p, x, blocks, stream); break;
+        default: return cudaErrorInvalidValue;
+    }
+    count_launch();
+    return e;
 }
 
 cudaError_t launch_quant(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
