@@ -156,7 +156,6 @@ static inline int prologue_slice_k(int max_M) { return max_M <= 8 ? 512 : 256; }
 cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_quant,
                                          const LoraItem *d_lora_items, int n_lora, int max_M, bool pdl,
                                          cudaStream_t stream);
-cudaError_t launch_lora_down_gemm(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream);
 cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream);
 cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream);
 // Shared memory the decode kernel needs for one problem's activations, and the largest it accepts.

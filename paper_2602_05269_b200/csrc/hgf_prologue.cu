@@ -254,43 +254,6 @@ __device__ __forceinline__ void lora_down_block(const PrologueParams &p, int jt)
     if (p.M <= 8) lora_down_tile<1>(p, jt); else lora_down_tile<2>(p, jt);
 }
 
-// Many rows of up to 4096 elements (GEMM path): one warp per token row, the row held in registers between the maximum and
-// the rounding (U 16-byte units per lane), so a row costs one trip to memory, no block-wide
-// synchronisation, and the per-row overhead (scale, reductions) is spread over 8 U elements per lane.
-template <int U>
-__global__ void __launch_bounds__(kThreads) quant_rows_kernel(const PrologueParams p, const GemmPrologueExtra x) {
-    const int lane = threadIdx.x & 31, m = blockIdx.x * kWarps + (threadIdx.x >> 5);
-    if (m >= p.M) return;
-    const int K = p.K, nv = K / 8;
-    const uint4 *xv = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K);
-    uint4 v[U];
-    uint32_t abits = 0u;
-#pragma unroll
-    for (int u = 0; u < U; ++u) v[u] = lane + 32 * u < nv ? xv[lane + 32 * u] : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-    for (int u = 0; u < U; ++u) abits = absmax8_bits(abits, v[u]);
-    const float g = fmaxf(warp_max(absmax_bits_to_float(abits)), 1e-5f);
-    const QuantScale qs = make_quant_scale(g);
-    int sum = 0;
-    uint2 *qv = reinterpret_cast<uint2 *>(p.xq + (size_t)m * K);
-    uint2 *dq = p.dbg_xq ? reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * K) : nullptr;
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-        if (lane + 32 * u < nv) {
-            const uint2 o = quant8(v[u], qs, sum);
-            qv[lane + 32 * u] = o;
-            if (dq) dq[lane + 32 * u] = o;
-        }
-    }
-    sum = warp_sum_i(sum);
-    if (lane == 0) {
-        if (p.row_sum) p.row_sum[m] = sum;
-        if (x.tok_sc) x.tok_sc[m] = g * x.gw_over_127;
-        p.gamma_x[m] = g;
-        if (p.dbg_gamma_x) p.dbg_gamma_x[m] = g;
-    }
-}
-
 __global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p, const GemmPrologueExtra x) {
     quant_row(p, blockIdx.x, x.tok_sc, x.gw_over_127);
 }
@@ -462,121 +425,6 @@ decode_prologue_group_kernel(const QuantItem *quant_items, int n_quant, const Lo
     }
 }
 
-// ---- GEMM-path LoRA down-projection on tensor cores (legacy warp MMA, tf32 inputs) -----------
-// bf16 and fp16 values are both exactly representable in tf32 (8 exponent, 10 mantissa bits), so
-// the products are formed from exact inputs and accumulated in fp32.
-// Block = 4 warps, tile = 32 tokens x r columns; the warps split K in 32-element chunks and the
-// partial sums are reduced through shared memory.
-constexpr int kLdWarps = 8;
-constexpr int kLdThreads = kLdWarps * 32;
-constexpr int kLdTokens = 32;
-
-template <int JT>  // r = 8 * JT column tiles
-__global__ void __launch_bounds__(kLdThreads) lora_down_gemm_kernel(const PrologueParams p, const GemmPrologueExtra x) {
-    extern __shared__ float s_acc[];  // [warps][32 tokens][8*JT]
-    const int token_blocks = (p.M + kLdTokens - 1) / kLdTokens;
-    if ((int)blockIdx.x >= token_blocks) {
-        // the remaining blocks prepare the up-projection's operand: row n of B^T times its channel's
-        // gate, fp16, padded to 64 columns (one 16-byte piece per thread)
-        const int idx = ((int)blockIdx.x - token_blocks) * kLdThreads + (int)threadIdx.x, n = idx >> 3, c = idx & 7;
-        if (n < x.N) {
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (c * 8 < p.r) {
-                v = *reinterpret_cast<const uint4 *>(x.Bt + (size_t)n * p.r + c * 8);
-                const float g = x.gate[n];
-                __half2 *h2 = reinterpret_cast<__half2 *>(&v);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float2 f = __half22float2(h2[k]);
-                    h2[k] = __floats2half2_rn(g * f.x, g * f.y);
-                }
-            }
-            *reinterpret_cast<uint4 *>(x.gb16 + (size_t)n * 64 + c * 8) = v;
-        }
-        return;
-    }
-    const int K = p.K, M = p.M, r = 8 * JT;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-    const int m0 = blockIdx.x * kLdTokens;
-
-    float acc[2][JT][4];
-#pragma unroll
-    for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int b = 0; b < JT; ++b)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.0f;
-
-    // rows this thread feeds: tokens m0 + 16 mt + g and + 8 (clamped; clamped rows are not stored)
-    const __nv_bfloat16 *xrow[2][2];
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-            int m = m0 + 16 * mt + 8 * hh + g;
-            m = m < M ? m : M - 1;
-            xrow[mt][hh] = p.x + (size_t)m * K;
-        }
-
-    const int nchunks = K / 32;
-    for (int c = warp; c < nchunks; c += kLdWarps) {
-        const int k = c * 32 + 8 * t;  // this thread's 8 consecutive k
-        uint4 xa[2][2];
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) xa[mt][hh] = *reinterpret_cast<const uint4 *>(xrow[mt][hh] + k);
-#pragma unroll
-        for (int jt = 0; jt < JT; ++jt) {
-            uint4 a4 = *reinterpret_cast<const uint4 *>(p.At + (size_t)(8 * jt + g) * K + k);
-            const uint32_t aw[4] = {a4.x, a4.y, a4.z, a4.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                __half2 hv = *reinterpret_cast<const __half2 *>(&aw[i]);
-                float2 bf = __half22float2(hv);
-                uint32_t b0 = __float_as_uint(bf.x), b1 = __float_as_uint(bf.y);
-#pragma unroll
-                for (int mt = 0; mt < 2; ++mt) {
-                    const uint32_t x0 = (&xa[mt][0].x)[i], x1 = (&xa[mt][1].x)[i];
-                    mma_tf32(acc[mt][jt], x0 << 16, x1 << 16, x0 & 0xffff0000u, x1 & 0xffff0000u, b0, b1);
-                }
-            }
-        }
-    }
-
-    // cross-warp reduction
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int jt = 0; jt < JT; ++jt) {
-            float *base = s_acc + ((size_t)warp * kLdTokens + 16 * mt) * r + 8 * jt;
-            base[(g)*r + 2 * t] = acc[mt][jt][0];
-            base[(g)*r + 2 * t + 1] = acc[mt][jt][1];
-            base[(g + 8) * r + 2 * t] = acc[mt][jt][2];
-            base[(g + 8) * r + 2 * t + 1] = acc[mt][jt][3];
-        }
-    __syncthreads();
-    for (int e = tid; e < kLdTokens * r; e += kLdThreads) {
-        int ml = e / r, j = e % r, m = m0 + ml;
-        float z = 0.0f;
-#pragma unroll
-        for (int w = 0; w < kLdWarps; ++w) z += s_acc[w * kLdTokens * r + e];
-        float h = (p.flags & HGF_FLAG_NO_SILU) ? z : silu_f(z);
-        if (m < M) {
-            p.h[(size_t)m * r + j] = h;
-            if (p.dbg_h) p.dbg_h[(size_t)m * r + j] = h;
-            if (p.h16) p.h16[(size_t)m * 64 + j] = __float2half_rn(h);
-        }
-    }
-    if constexpr (JT < 8) {  // zero padding of the fp16 copy up to 64 columns
-        if (p.h16)
-        for (int e = tid; e < kLdTokens * (64 - r); e += kLdThreads) {
-            int ml = e / (64 - r), j = r + e % (64 - r), m = m0 + ml;
-            if (m < M) p.h16[(size_t)m * 64 + j] = __float2half_rn(0.0f);
-        }
-    }
-}
-
 // ---- GEMM-path prologue in one kernel -------------------------------------------------------------
 // Quantisation (Algorithm 1, steps 1-2) and the LoRA down-projection (steps 5-6) of a block of 32
 // tokens, reading x from HBM once.  First pass: x and the rows of A^T travel through a three-stage
@@ -634,21 +482,30 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
     constexpr int kStage = fp_stage_bytes(r);
     const int nchunks = (K + kFpChunk - 1) / kFpChunk;
 
-    // one chunk into one stage: 32 (+ r) rows of 32 16-byte units; rows past M and columns past K are zeros
+    // One chunk into one stage: 32 (+ r) rows of 32 16-byte units; rows past M and columns past K are
+    // zeros.  A thread copies unit `lane` of rows warp, warp + 8, ...: the same ones in every chunk.
+    constexpr int kRowsPerThread = (kFpTokens + r) / kFpWarps;
+    const uint8_t *src_row[kRowsPerThread];
+    bool row_ok[kRowsPerThread];
+#pragma unroll
+    for (int q = 0; q < kRowsPerThread; ++q) {
+        const int row = warp + kFpWarps * q;
+        if (row < kFpTokens) {
+            row_ok[q] = m0 + row < M;
+            src_row[q] = reinterpret_cast<const uint8_t *>(p.x + (size_t)(row_ok[q] ? m0 + row : 0) * K) + 16 * lane;
+        } else {
+            row_ok[q] = true;
+            src_row[q] = reinterpret_cast<const uint8_t *>(p.At + (size_t)(row - kFpTokens) * K) + 16 * lane;
+        }
+    }
     auto fetch = [&](int c, int stage) {
-        const uint32_t dst0 = smem_u32 + stage * kStage;
-        const int k0 = c * kFpChunk;
-        for (int u = tid; u < (kFpTokens + r) * 32; u += kFpThreads) {
-            const int row = u >> 5, unit = u & 31, k = k0 + 8 * unit;
-            const void *src;
-            bool in = k < K;
-            if (row < kFpTokens) {
-                in = in && m0 + row < M;
-                src = p.x + (size_t)(in ? m0 + row : 0) * K + (in ? k : 0);
-            } else {
-                src = p.At + (size_t)(row - kFpTokens) * K + (in ? k : 0);
-            }
-            cp_async_16(dst0 + row * kFpPitch + 16 * unit, src, in ? 16u : 0u);
+        const uint32_t dst = smem_u32 + stage * kStage + warp * kFpPitch + 16 * lane;
+        const int k = c * kFpChunk + 8 * lane;
+        const bool col_ok = k < K;
+#pragma unroll
+        for (int q = 0; q < kRowsPerThread; ++q) {
+            const bool in = col_ok && row_ok[q];
+            cp_async_16(dst + q * kFpWarps * kFpPitch, src_row[q] + (in ? (size_t)c * kFpChunk * 2 : 0), in ? 16u : 0u);
         }
         asm volatile("cp.async.commit_group;\n" ::: "memory");
     };
@@ -674,28 +531,26 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
         else asm volatile("cp.async.commit_group;\n" ::: "memory");
 
         const uint32_t st = smem_u32 + (c % kFpStages) * kStage + 64 * warp + 16 * t;
-        uint4 xa[2][2];
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                xa[mt][hh] = pg_lds_u4(st + (16 * mt + 8 * hh + g) * kFpPitch);
-                amax[mt][hh] = absmax8_bits(amax[mt][hh], xa[mt][hh]);
-            }
-        if constexpr (JT > 0) {
-#pragma unroll
-            for (int jt = 0; jt < JT; ++jt) {
-                const uint4 a4 = pg_lds_u4(st + (kFpTokens + 8 * jt + g) * kFpPitch);
-                const uint32_t aw[4] = {a4.x, a4.y, a4.z, a4.w};
+        for (int mt = 0; mt < 2; ++mt) {
+            const uint4 x0 = pg_lds_u4(st + (16 * mt + g) * kFpPitch), x1 = pg_lds_u4(st + (16 * mt + 8 + g) * kFpPitch);
+            amax[mt][0] = absmax8_bits(amax[mt][0], x0);
+            amax[mt][1] = absmax8_bits(amax[mt][1], x1);
+            if constexpr (JT > 0) {
+                // elements 2 i and 2 i + 1 of this lane's eight take the k slots t and t + 4 of MMA i
+                uint32_t xs[4][4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    // elements 2 i and 2 i + 1 of this lane's eight take the k slots t and t + 4 of the MMA
-                    const float2 bf = __half22float2(*reinterpret_cast<const __half2 *>(&aw[i]));
-                    const uint32_t b0 = __float_as_uint(bf.x), b1 = __float_as_uint(bf.y);
+                    const uint32_t w0 = (&x0.x)[i], w1 = (&x1.x)[i];
+                    xs[i][0] = w0 << 16; xs[i][1] = w1 << 16; xs[i][2] = w0 & 0xffff0000u; xs[i][3] = w1 & 0xffff0000u;
+                }
 #pragma unroll
-                    for (int mt = 0; mt < 2; ++mt) {
-                        const uint32_t x0 = (&xa[mt][0].x)[i], x1 = (&xa[mt][1].x)[i];
-                        mma_tf32(acc[mt][jt], x0 << 16, x1 << 16, x0 & 0xffff0000u, x1 & 0xffff0000u, b0, b1);
+                for (int jt = 0; jt < JT; ++jt) {
+                    const uint4 a4 = pg_lds_u4(st + (kFpTokens + 8 * jt + g) * kFpPitch);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 bf = __half22float2(*reinterpret_cast<const __half2 *>(&(&a4.x)[i]));
+                        mma_tf32(acc[mt][jt], xs[i][0], xs[i][1], xs[i][2], xs[i][3], __float_as_uint(bf.x), __float_as_uint(bf.y));
                     }
                 }
             }
@@ -820,14 +675,15 @@ cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtr
     return e;
 }
 
+// Stand-alone quantisation: the GEMM path's prologue kernel without its LoRA part for many rows, one
+// block per row otherwise.
 cudaError_t launch_quant(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
-    const int nv = p.K / 8, row_blocks = (p.M + kWarps - 1) / kWarps;
-    if (p.M >= 256 && nv <= 32 * 8)
-        quant_rows_kernel<8><<<row_blocks, kThreads, 0, stream>>>(p, x);
-    else if (p.M >= 256 && nv <= 32 * 16)
-        quant_rows_kernel<16><<<row_blocks, kThreads, 0, stream>>>(p, x);
-    else
-        quant_kernel<<<p.M, kThreads, 0, stream>>>(p, x);
+    if (p.M >= 2 * kFpTokens) {
+        PrologueParams q = p;
+        q.r = 0;
+        return launch_gemm_prologue(q, x, stream);
+    }
+    quant_kernel<<<p.M, kThreads, 0, stream>>>(p, x);
     count_launch();
     return cudaGetLastError();
 }
@@ -888,27 +744,6 @@ cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_q
     }
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
-}
-
-cudaError_t launch_lora_down_gemm(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
-    const int blocks = (p.M + kLdTokens - 1) / kLdTokens + (x.gb16 ? (x.N * 8 + kLdThreads - 1) / kLdThreads : 0);
-    const size_t smem = (size_t)kLdWarps * kLdTokens * p.r * sizeof(float);
-    static bool attr_set = false;
-    if (!attr_set) {  // the widest variant needs more than the default dynamic shared memory
-        cudaError_t e = cudaFuncSetAttribute(lora_down_gemm_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kLdWarps * kLdTokens * 64 * (int)sizeof(float));
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
-    switch (p.r) {
-        case 16: lora_down_gemm_kernel<2><<<blocks, kLdThreads, smem, stream>>>(p, x); break;
-        case 32: lora_down_gemm_kernel<4><<<blocks, kLdThreads, smem, stream>>>(p, x); break;
-        case 48: lora_down_gemm_kernel<6><<<blocks, kLdThreads, smem, stream>>>(p, x); break;
-        case 64: lora_down_gemm_kernel<8><<<blocks, kLdThreads, smem, stream>>>(p, x); break;
-        default: return cudaErrorInvalidValue;
-    }
-    count_launch();
-    return cudaGetLastError();
 }
 
 }  // namespace hgf
