@@ -167,7 +167,7 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
     gx.gate = gate;
     gx.gw_over_127 = dp.gw_over_127;
     gx.N = (int)d_out;
-    if (launch_gemm_prologue(pp, gx, stream) != cudaSuccess) return HGF_ERR_CUDA;
+    if ((r ? launch_gemm_prologue(pp, gx, stream) : launch_quant(pp, gx, stream)) != cudaSuccess) return HGF_ERR_CUDA;
     GemmParams gp = {};
     gp.xq = pp.xq;
     gp.packed = (const uint8_t *)packed;

@@ -254,6 +254,43 @@ __device__ __forceinline__ void lora_down_block(const PrologueParams &p, int jt)
     if (p.M <= 8) lora_down_tile<1>(p, jt); else lora_down_tile<2>(p, jt);
 }
 
+// Many rows of up to 4096 elements (quantisation alone): one warp per token row, the row held in registers between the maximum and
+// the rounding (U 16-byte units per lane), so a row costs one trip to memory, no block-wide
+// synchronisation, and the per-row overhead (scale, reductions) is spread over 8 U elements per lane.
+template <int U>
+__global__ void __launch_bounds__(kThreads) quant_rows_kernel(const PrologueParams p, const GemmPrologueExtra x) {
+    const int lane = threadIdx.x & 31, m = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (m >= p.M) return;
+    const int K = p.K, nv = K / 8;
+    const uint4 *xv = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K);
+    uint4 v[U];
+    uint32_t abits = 0u;
+#pragma unroll
+    for (int u = 0; u < U; ++u) v[u] = lane + 32 * u < nv ? xv[lane + 32 * u] : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int u = 0; u < U; ++u) abits = absmax8_bits(abits, v[u]);
+    const float g = fmaxf(warp_max(absmax_bits_to_float(abits)), 1e-5f);
+    const QuantScale qs = make_quant_scale(g);
+    int sum = 0;
+    uint2 *qv = reinterpret_cast<uint2 *>(p.xq + (size_t)m * K);
+    uint2 *dq = p.dbg_xq ? reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * K) : nullptr;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        if (lane + 32 * u < nv) {
+            const uint2 o = quant8(v[u], qs, sum);
+            qv[lane + 32 * u] = o;
+            if (dq) dq[lane + 32 * u] = o;
+        }
+    }
+    sum = warp_sum_i(sum);
+    if (lane == 0) {
+        if (p.row_sum) p.row_sum[m] = sum;
+        if (x.tok_sc) x.tok_sc[m] = g * x.gw_over_127;
+        p.gamma_x[m] = g;
+        if (p.dbg_gamma_x) p.dbg_gamma_x[m] = g;
+    }
+}
+
 __global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p, const GemmPrologueExtra x) {
     quant_row(p, blockIdx.x, x.tok_sc, x.gw_over_127);
 }
@@ -675,15 +712,21 @@ cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtr
     return e;
 }
 
-// Stand-alone quantisation: the GEMM path's prologue kernel without its LoRA part for many rows, one
-// block per row otherwise.
+// Quantisation alone.  Many rows: one warp per row while a row fits its registers, else the GEMM
+// path's prologue kernel without its LoRA part; few rows: one block per row.
 cudaError_t launch_quant(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
-    if (p.M >= 2 * kFpTokens) {
+    const int nv = p.K / 8, row_blocks = (p.M + kWarps - 1) / kWarps;
+    if (p.M >= 256 && nv <= 32 * 8) {
+        quant_rows_kernel<8><<<row_blocks, kThreads, 0, stream>>>(p, x);
+    } else if (p.M >= 256 && nv <= 32 * 16) {
+        quant_rows_kernel<16><<<row_blocks, kThreads, 0, stream>>>(p, x);
+    } else if (p.M >= 2 * kFpTokens) {
         PrologueParams q = p;
         q.r = 0;
         return launch_gemm_prologue(q, x, stream);
+    } else {
+        quant_kernel<<<p.M, kThreads, 0, stream>>>(p, x);
     }
-    quant_kernel<<<p.M, kThreads, 0, stream>>>(p, x);
     count_launch();
     return cudaGetLastError();
 }
