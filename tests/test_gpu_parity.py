@@ -176,6 +176,24 @@ def test_act_quant_entry_point_and_crafted_ties(hgf):
     assert np.array_equal(xq.cpu().numpy(), ref_q) and np.array_equal(gx.cpu().numpy(), ref_g)
 
 
+@pytest.mark.parametrize("M,K", [(300, 2048), (260, 4096), (70, 5632), (257, 64)])
+def test_act_quant_many_rows_every_kernel(hgf, M, K):
+    """The many-row kernels (a warp per row; the GEMM path's prologue without its LoRA part), with
+    exact ties, an all-zero row and a ragged last block."""
+    x = syn.bf16_bits_to_f32(syn.make_x(M, K, config=7, layer=M))
+    for row in (0, M // 2, M - 1):
+        x[row, :3] = [1216.0, 608.0, -608.0]  # gamma = 1216: 63.5 -> 64, -63.5 -> -64
+        x[row, 3:] = np.clip(x[row, 3:], -1000.0, 1000.0)
+    x[1, :] = 0.0
+    xb = syn.f32_to_bf16_bits(x)
+    xq, gx, rs = hgf.act_quant(dev(xb, torch.bfloat16))
+    ref_q, ref_g = oracle.act_quant(xb)
+    assert np.array_equal(gx.cpu().numpy(), ref_g)
+    assert np.array_equal(xq.cpu().numpy(), ref_q)
+    assert xq[0, :3].tolist() == [127, 64, -64]
+    assert np.array_equal(rs.cpu().numpy(), ref_q.astype(np.int64).sum(axis=1).astype(np.int32))
+
+
 def test_pack_crafted_boundaries(hgf):
     W = syn.make_weights(16, 64, config=5)
     g = float(oracle.gamma_w(W))
