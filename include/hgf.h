@@ -174,6 +174,8 @@ hgf_status hgf_linear_forward_static(const void *x, int64_t M, const void *packe
  * same X; the MLP's two up-projections likewise), and each is small against the launch latency,
  * so a group streams all their packed weights in one pass.  Each problem is exactly one
  * hgf_linear_forward with M <= HGF_DECODE_MAX_M (same argument meaning, same requirements).
+ * Problems that name the same x (same pointer, M and d_in) are quantised once and share the
+ * result; their LoRA down-projections stay separate, since each has its own A.
  *
  * hgf_group_create records the problems (pointers are kept, not the data: x, y and the weights
  * stay owned by the caller and must stay valid) and allocates the group's descriptors and

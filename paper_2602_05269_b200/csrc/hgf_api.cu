@@ -3,6 +3,7 @@
 // fallback: without a CUDA device every forward call fails with HGF_ERR_CUDA.
 #include <atomic>
 #include <new>
+#include <unordered_map>
 #include <vector>
 
 #include "hgf_common.cuh"
@@ -271,7 +272,7 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     const int slice_k = prologue_slice_k(all_M);
     size_t n_quant = 0, n_lora = 0;
     for (int i = 0; i < n; ++i) {
-        n_quant += (size_t)problems[i].M;
+        n_quant += (size_t)problems[i].M;  // an upper bound: problems that share x share their items
         n_lora += ((size_t)ranks[i] / 16) * (size_t)((problems[i].d_in + slice_k - 1) / slice_k);
     }
     const size_t off_qit = align_up(off_pps + sizeof(PrologueParams) * (size_t)n, 256);
@@ -283,6 +284,7 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     if (cudaMalloc(&mem, off_ws + ws_total) != cudaSuccess) return HGF_ERR_CUDA;
     char *ws = (char *)mem + off_ws;
     float *hpart = (float *)((char *)mem + off_hpart);
+    std::unordered_map<const void *, int> first_with_x;
     for (int i = 0; i < n; ++i) {
         const hgf_problem &q = problems[i];
         fill_params(q.x, q.M, q.packed, q.gamma, q.d_in, q.d_out, q.At, q.Bt, ranks[i], q.gate, q.y, ws, lay[i], false,
@@ -290,11 +292,27 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         ws += lay[i].total;
         dps[i].tile_begin = tiles;
         dps[i].cost_begin = cost;
+        // problems on the same input (Q, K and V of an attention block; the two up-projections of its
+        // MLP) share one quantisation: a later one reads the first one's x~, scales and row sums
+        int first = i;
+        {
+            auto seen = first_with_x.find(q.x);
+            if (seen == first_with_x.end()) first_with_x.emplace(q.x, i);
+            else if (problems[seen->second].M == q.M && problems[seen->second].d_in == q.d_in) first = seen->second;
+        }
+        if (first != i) {
+            pps[i].xq = pps[first].xq;
+            pps[i].gamma_x = pps[first].gamma_x;
+            pps[i].row_sum = pps[first].row_sum;
+            dps[i].xq = dps[first].xq;
+            dps[i].gamma_x = dps[first].gamma_x;
+            dps[i].row_sum = dps[first].row_sum;
+        }
         {
             const int slices = (int)((q.d_in + slice_k - 1) / slice_k), jts = ranks[i] / 16;
             dps[i].hpart = jts ? hpart : nullptr;
             dps[i].nslices = jts ? slices : 0;
-            for (int m = 0; m < (int)q.M; ++m) {
+            for (int m = 0; first == i && m < (int)q.M; ++m) {
                 QuantItem qi = {pps[i].x + (size_t)m * q.d_in, pps[i].xq + (size_t)m * q.d_in, pps[i].gamma_x + m,
                                 pps[i].row_sum + m, (int)q.d_in, 0};
                 qitems.push_back(qi);

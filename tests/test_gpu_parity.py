@@ -283,6 +283,30 @@ def test_group_of_independent_layers_matches_oracle_and_single_calls(hgf, M):
     group.close()
 
 
+@pytest.mark.parametrize("M", [1, 5, 16])
+def test_group_problems_on_the_same_input_share_its_quantisation(hgf, M):
+    """Q, K, V on one x and two up-projections on another: the group quantises each input once;
+    results are those of the separate calls, bit for bit in the integer part."""
+    d = 1024
+    shapes = [syn.LayerShape("q", d, d, 32), syn.LayerShape("k", d, 256, 32), syn.LayerShape("v", d, 256, 16),
+              syn.LayerShape("up", d, 2816, 32), syn.LayerShape("gate", d, 2816, 32), syn.LayerShape("own", d, 512, 32)]
+    probs, hosts = zip(*[_group_problem(hgf, s, M, 14, i) for i, s in enumerate(shapes)])
+    probs, hosts = list(probs), list(hosts)
+    for i in (1, 2):          # k, v read q's x
+        probs[i]["x"], hosts[i]["x"] = probs[0]["x"], hosts[0]["x"]
+    probs[4]["x"], hosts[4]["x"] = probs[3]["x"], hosts[3]["x"]   # gate reads up's x
+    group = hgf.Group(probs)
+    group.forward()
+    hgf.check_status()
+    for q, h, s in zip(probs, hosts, shapes):
+        ref = oracle.forward(h["x"], h["T"], h["gamma"], h["At"], h["Bt"], h["gate"])
+        yg = q["y"].cpu().numpy().astype(np.float64)
+        assert np.abs(yg - ref["y"]).max() / np.abs(ref["y"]).max() <= TOL_DECODE, s
+        y_single = hgf.linear_forward(q["x"], q["packed"], q["gamma"], s.d_in, s.d_out, q["At"], q["Bt"], q["gate"])
+        assert (y_single - q["y"]).abs().max().item() <= 2e-6 * np.abs(ref["y"]).max(), s
+    group.close()
+
+
 def test_group_rejects_gemm_sized_problem(hgf):
     q, _ = _group_problem(hgf, syn.LayerShape("big", 256, 256, 16), 17, 12, 50)
     with pytest.raises(hgf.HgfError) as e:
