@@ -89,6 +89,7 @@ struct GemmPrologueExtra {
     const float *gate;       // [N]
     float gw_over_127;
     int N;
+    int tokens_per_block;    // set by the launcher of the GEMM path's prologue kernel
 };
 
 // Cost of one 16-row tile of a decode problem, the unit in which a launch is cut into equal shares:

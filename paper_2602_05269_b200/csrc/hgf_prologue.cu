@@ -489,7 +489,8 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
     __shared__ float s_amax[kFpWarps][kFpTokens];
     __shared__ float s_gamma[kFpTokens];
     constexpr int r = 8 * JT;
-    const int token_blocks = (p.M + kFpTokens - 1) / kFpTokens;
+    const int tpb = x.tokens_per_block;  // tokens this launch gives a block (at most kFpTokens)
+    const int token_blocks = (p.M + tpb - 1) / tpb;
     if ((int)blockIdx.x >= token_blocks) {
         // the remaining blocks prepare the up-projection's operand: row n of B^T times its channel's
         // gate, fp16, padded to 64 columns (one 16-byte piece per thread)
@@ -514,7 +515,7 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
     }
     const int K = p.K, M = p.M;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-    const int m0 = blockIdx.x * kFpTokens;
+    const int m0 = blockIdx.x * tpb;
     const uint32_t smem_u32 = (uint32_t)__cvta_generic_to_shared(fp_smem);
     constexpr int kStage = fp_stage_bytes(r);
     const int nchunks = (K + kFpChunk - 1) / kFpChunk;
@@ -528,7 +529,7 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
     for (int q = 0; q < kRowsPerThread; ++q) {
         const int row = warp + kFpWarps * q;
         if (row < kFpTokens) {
-            row_ok[q] = m0 + row < M;
+            row_ok[q] = row < tpb && m0 + row < M;
             src_row[q] = reinterpret_cast<const uint8_t *>(p.x + (size_t)(row_ok[q] ? m0 + row : 0) * K) + 16 * lane;
         } else {
             row_ok[q] = true;
@@ -570,6 +571,7 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
         const uint32_t st = smem_u32 + (c % kFpStages) * kStage + 64 * warp + 16 * t;
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
+            if (16 * mt >= tpb) break;  // a block of up to 16 tokens has no second tile
             const uint4 x0 = pg_lds_u4(st + (16 * mt + g) * kFpPitch), x1 = pg_lds_u4(st + (16 * mt + 8 + g) * kFpPitch);
             amax[mt][0] = absmax8_bits(amax[mt][0], x0);
             amax[mt][1] = absmax8_bits(amax[mt][1], x1);
@@ -634,7 +636,7 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
 #pragma unroll
             for (int w = 0; w < kFpWarps; ++w) z += s_acc[w * kFpTokens * r + e];
             const float h = (p.flags & HGF_FLAG_NO_SILU) ? z : silu_f(z);
-            if (m < M) {
+            if (ml < tpb && m < M) {
                 p.h[(size_t)m * r + j] = h;
                 if (p.dbg_h) p.dbg_h[(size_t)m * r + j] = h;
                 if (p.h16) p.h16[(size_t)m * 64 + j] = __float2half_rn(h);
@@ -644,17 +646,17 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
             if (p.h16)
                 for (int e = tid; e < kFpTokens * (64 - r); e += kFpThreads) {
                     const int ml = e / (64 - r), j = r + e % (64 - r), m = m0 + ml;
-                    if (m < M) p.h16[(size_t)m * 64 + j] = __float2half_rn(0.0f);
+                    if (ml < tpb && m < M) p.h16[(size_t)m * 64 + j] = __float2half_rn(0.0f);
                 }
         }
     }
 
-    // second pass: each warp rounds four of the block's rows
+    // second pass: the warps round the block's rows, warp w rows w, w + 8, ...
     const int nv = K / 8;
 #pragma unroll 1
     for (int rr = 0; rr < kFpTokens / kFpWarps; ++rr) {
-        const int ml = warp * (kFpTokens / kFpWarps) + rr, m = m0 + ml;
-        if (m >= M) break;
+        const int ml = warp + kFpWarps * rr, m = m0 + ml;
+        if (ml >= tpb || m >= M) break;
         const float gm = s_gamma[ml];
         const QuantScale qs = make_quant_scale(gm);
         const uint4 *xv = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K);
@@ -698,14 +700,27 @@ static cudaError_t launch_gemm_prologue_jt(const PrologueParams &p, const GemmPr
 
 // Quantisation and (r > 0) LoRA down-projection of the GEMM path, plus gate * B^T for its epilogue.
 cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
-    const int blocks = (p.M + kFpTokens - 1) / kFpTokens + ((p.r > 0 && x.gb16) ? (x.N * 8 + kFpThreads - 1) / kFpThreads : 0);
+    // Tokens per block: two blocks fit an SM, so up to twice the SM count of blocks share the rows
+    // evenly; beyond that a block takes its full 32.
+    static int sm_count = 0;
+    if (!sm_count) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return cudaErrorInvalidDevice;
+    }
+    int tpb = (p.M + 2 * sm_count - 1) / (2 * sm_count);
+    tpb = (tpb + 3) / 4 * 4;
+    tpb = tpb < 8 ? 8 : (tpb > kFpTokens ? kFpTokens : tpb);
+    GemmPrologueExtra xx = x;
+    xx.tokens_per_block = tpb;
+    const int blocks = (p.M + tpb - 1) / tpb + ((p.r > 0 && x.gb16) ? (x.N * 8 + kFpThreads - 1) / kFpThreads : 0);
     cudaError_t e;
     switch (p.r) {
-        case 0: e = launch_gemm_prologue_jt<0>(p, x, blocks, stream); break;
-        case 16: e = launch_gemm_prologue_jt<2>(p, x, blocks, stream); break;
-        case 32: e = launch_gemm_prologue_jt<4>(p, x, blocks, stream); break;
-        case 48: e = launch_gemm_prologue_jt<6>(p, x, blocks, stream); break;
-        case 64: e = launch_gemm_prologue_jt<8>(p, x, blocks, stream); break;
+        case 0: e = launch_gemm_prologue_jt<0>(p, xx, blocks, stream); break;
+        case 16: e = launch_gemm_prologue_jt<2>(p, xx, blocks, stream); break;
+        case 32: e = launch_gemm_prologue_jt<4>(p, xx, blocks, stream); break;
+        case 48: e = launch_gemm_prologue_jt<6>(p, xx, blocks, stream); break;
+        case 64: e = launch_gemm_prologue_jt<8>(p, xx, blocks, stream); break;
         default: return cudaErrorInvalidValue;
     }
     count_launch();
