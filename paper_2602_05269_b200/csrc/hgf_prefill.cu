@@ -292,6 +292,9 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Everything above touches only this CTA's own shared and tensor memory; what follows reads what
+    // the prologue launch wrote (a no-op unless the launch carries the programmatic-dependency attribute).
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -634,8 +637,18 @@ static cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &mh, 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    prefill_gemm_kernel<OUT_BF16, NS, OPSB><<<grid, GEMM_THREADS, smem, stream>>>(mx, mh, mgb, my, p, status);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (p.flags & HGF_FLAG_NO_PDL) ? 0 : 1;  // set-up (barriers, tensor memory) may overlap the prologue's tail
+    cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_gemm_kernel<OUT_BF16, NS, OPSB>, mx, mh, mgb, my, p, status);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {

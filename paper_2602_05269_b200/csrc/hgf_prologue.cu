@@ -259,6 +259,7 @@ __device__ __forceinline__ void lora_down_block(const PrologueParams &p, int jt)
 // synchronisation, and the per-row overhead (scale, reductions) is spread over 8 U elements per lane.
 template <int U>
 __global__ void __launch_bounds__(kThreads) quant_rows_kernel(const PrologueParams p, const GemmPrologueExtra x) {
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");  // see gemm_prologue_kernel
     const int lane = threadIdx.x & 31, m = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (m >= p.M) return;
     const int K = p.K, nv = K / 8;
@@ -489,6 +490,7 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
     __shared__ float s_amax[kFpWarps][kFpTokens];
     __shared__ float s_gamma[kFpTokens];
     constexpr int r = 8 * JT;
+    pdl_launch_dependents();  // the GEMM that follows may set itself up; it waits for this grid before it reads
     const int tpb = x.tokens_per_block;  // tokens this launch gives a block (at most kFpTokens)
     const int token_blocks = (p.M + tpb - 1) / tpb;
     if ((int)blockIdx.x >= token_blocks) {
