@@ -247,6 +247,9 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_BAR + C::BAR_COUNT * 8 + 4);
     static_assert(TILE_T == 128, "the epilogue's staging loops are written for 128-token tiles");
 
+    // the next launch in the stream, if it asks for it, may be set up while this one runs (it waits
+    // for this grid's completion before it touches memory)
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int tiles_t = (p.M + TILE_T - 1) / TILE_T, tiles_c = (p.N + TILE_C - 1) / TILE_C;
     const int num_tiles = tiles_t * tiles_c;

@@ -259,7 +259,7 @@ __device__ __forceinline__ void lora_down_block(const PrologueParams &p, int jt)
 // synchronisation, and the per-row overhead (scale, reductions) is spread over 8 U elements per lane.
 template <int U>
 __global__ void __launch_bounds__(kThreads) quant_rows_kernel(const PrologueParams p, const GemmPrologueExtra x) {
-    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");  // see gemm_prologue_kernel
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");  // see gemm_prologue_kernel
     const int lane = threadIdx.x & 31, m = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (m >= p.M) return;
     const int K = p.K, nv = K / 8;
@@ -272,6 +272,7 @@ __global__ void __launch_bounds__(kThreads) quant_rows_kernel(const ProloguePara
     for (int u = 0; u < U; ++u) abits = absmax8_bits(abits, v[u]);
     const float g = fmaxf(warp_max(absmax_bits_to_float(abits)), 1e-5f);
     const QuantScale qs = make_quant_scale(g);
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");  // the row is in registers: the next launch may be set up
     int sum = 0;
     uint2 *qv = reinterpret_cast<uint2 *>(p.xq + (size_t)m * K);
     uint2 *dq = p.dbg_xq ? reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * K) : nullptr;
@@ -463,6 +464,8 @@ decode_prologue_group_kernel(const QuantItem *quant_items, int n_quant, const Lo
     }
 }
 
+static cudaLaunchConfig_t prologue_cfg(int blocks, bool pdl, cudaStream_t stream, cudaLaunchAttribute *attr);
+
 // ---- GEMM-path prologue in one kernel -------------------------------------------------------------
 // Quantisation (Algorithm 1, steps 1-2) and the LoRA down-projection (steps 5-6) of a block of 32
 // tokens, reading x from HBM once.  First pass: x and the rows of A^T travel through a three-stage
@@ -490,7 +493,7 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
     __shared__ float s_amax[kFpWarps][kFpTokens];
     __shared__ float s_gamma[kFpTokens];
     constexpr int r = 8 * JT;
-    pdl_launch_dependents();  // the GEMM that follows may set itself up; it waits for this grid before it reads
+    pdl_wait();  // x, and the workspace this kernel overwrites, belong to earlier work
     const int tpb = x.tokens_per_block;  // tokens this launch gives a block (at most kFpTokens)
     const int token_blocks = (p.M + tpb - 1) / tpb;
     if ((int)blockIdx.x >= token_blocks) {
@@ -653,6 +656,11 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
         }
     }
 
+    // The launch that follows (the GEMM) may be set up from here on; it waits for this grid's completion
+    // before it reads.  (Not earlier: blocks of a dependent launch that sit waiting on an SM slow the
+    // blocks still working there.)
+    pdl_launch_dependents();
+
     // second pass: the warps round the block's rows, warp w rows w, w + 8, ...
     const int nv = K / 8;
 #pragma unroll 1
@@ -689,15 +697,22 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
 
 template <int JT>
 static cudaError_t launch_gemm_prologue_jt(const PrologueParams &p, const GemmPrologueExtra &x, int blocks, cudaStream_t stream) {
-    constexpr int smem = fp_smem_bytes(8 * JT);
+    // Never more than two blocks per SM (the launcher spreads the rows over twice the SM count of
+    // blocks): blocks that start as SMs come free at the tail of the preceding launch would otherwise
+    // pile up four to an SM on the first SMs free and leave the others idle.
+    constexpr int smem = fp_smem_bytes(8 * JT) > 80 * 1024 ? fp_smem_bytes(8 * JT) : 80 * 1024;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(gemm_prologue_kernel<JT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    gemm_prologue_kernel<JT><<<blocks, kFpThreads, smem, stream>>>(p, x);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = prologue_cfg(blocks, !(p.flags & HGF_FLAG_NO_PDL), stream, attr);
+    cfg.blockDim = dim3(kFpThreads);
+    cfg.dynamicSmemBytes = smem;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_prologue_kernel<JT>, p, x);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // Quantisation and (r > 0) LoRA down-projection of the GEMM path, plus gate * B^T for its epilogue.
@@ -734,9 +749,15 @@ cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtr
 cudaError_t launch_quant(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
     const int nv = p.K / 8, row_blocks = (p.M + kWarps - 1) / kWarps;
     if (p.M >= 256 && nv <= 32 * 8) {
-        quant_rows_kernel<8><<<row_blocks, kThreads, 0, stream>>>(p, x);
+        cudaLaunchAttribute attr[1];
+        cudaLaunchConfig_t cfg = prologue_cfg(row_blocks, !(p.flags & HGF_FLAG_NO_PDL), stream, attr);
+        cudaError_t e = cudaLaunchKernelEx(&cfg, quant_rows_kernel<8>, p, x);
+        if (e != cudaSuccess) return e;
     } else if (p.M >= 256 && nv <= 32 * 16) {
-        quant_rows_kernel<16><<<row_blocks, kThreads, 0, stream>>>(p, x);
+        cudaLaunchAttribute attr[1];
+        cudaLaunchConfig_t cfg = prologue_cfg(row_blocks, !(p.flags & HGF_FLAG_NO_PDL), stream, attr);
+        cudaError_t e = cudaLaunchKernelEx(&cfg, quant_rows_kernel<16>, p, x);
+        if (e != cudaSuccess) return e;
     } else if (p.M >= 2 * kFpTokens) {
         PrologueParams q = p;
         q.r = 0;
@@ -748,7 +769,7 @@ cudaError_t launch_quant(const PrologueParams &p, const GemmPrologueExtra &x, cu
     return cudaGetLastError();
 }
 
-static cudaLaunchConfig_t prologue_cfg(int blocks, bool pdl, cudaStream_t stream, cudaLaunchAttribute *attr) {
+cudaLaunchConfig_t prologue_cfg(int blocks, bool pdl, cudaStream_t stream, cudaLaunchAttribute *attr) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks);
     cfg.blockDim = dim3(kThreads);
