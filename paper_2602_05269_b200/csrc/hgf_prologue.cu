@@ -717,15 +717,16 @@ static cudaError_t launch_gemm_prologue_jt(const PrologueParams &p, const GemmPr
 
 // Quantisation and (r > 0) LoRA down-projection of the GEMM path, plus gate * B^T for its epilogue.
 cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
-    // Tokens per block: two blocks fit an SM, so up to twice the SM count of blocks share the rows
-    // evenly; beyond that a block takes its full 32.
+    // Tokens per block: as many blocks as are resident at once share the rows evenly; beyond that a
+    // block takes its full 32.
     static int sm_count = 0;
     if (!sm_count) {
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return cudaErrorInvalidDevice;
     }
-    int tpb = (p.M + 2 * sm_count - 1) / (2 * sm_count);
+    const int per_sm = p.r >= 48 ? 1 : 2;  // blocks that fit an SM (shared memory: 138 KB and more from rank 48 on)
+    int tpb = (p.M + per_sm * sm_count - 1) / (per_sm * sm_count);
     tpb = (tpb + 3) / 4 * 4;
     tpb = tpb < 8 ? 8 : (tpb > kFpTokens ? kFpTokens : tpb);
     GemmPrologueExtra xx = x;
