@@ -101,6 +101,12 @@ static void fill_params(const void *x, int64_t M, const void *packed, float gamm
     pp->dbg_xq = dbg ? dbg->xq : nullptr;
     pp->dbg_gamma_x = dbg ? dbg->gamma_x : nullptr;
     pp->dbg_h = (dbg && r) ? dbg->h : nullptr;
+    // decode path: unless H itself is asked for, x A is computed in K slices by more blocks and the
+    // GEMV adds the slices
+    if (!gemm && r && !pp->dbg_h) {
+        pp->hpart = (float *)(ws + L.hpart);
+        pp->nslices = (int)((d_in + prologue_slice_k((int)M) - 1) / prologue_slice_k((int)M));
+    }
     pp->M = (int)M;
     pp->K = (int)d_in;
     pp->r = r;
@@ -113,6 +119,8 @@ static void fill_params(const void *x, int64_t M, const void *packed, float gamm
         dp->row_sum = pp->row_sum;
         dp->h_hi = pp->h_hi;
         dp->h_lo = pp->h_lo;
+        dp->hpart = pp->hpart;
+        dp->nslices = pp->hpart ? pp->nslices : 0;
         dp->Bt = (const __half *)Bt;
         dp->gate = gate;
         dp->y = y;

@@ -34,13 +34,14 @@ static inline int64_t row_tiles(int64_t d_out) { return (d_out + 15) / 16; }
 //   h        [M][r]      float    SiLU(x A)
 //   h_hi     [M][r]      half     fp16 rounding of h          (decode path only)
 //   h_lo     [M][r]      half     fp16 rounding of h - h_hi   (decode path only)
+//   hpart    [r/16][slices][8][32] float  partial sums of x A per K slice (decode path only; see LoraItem)
 //   h16      [M][64]     half     h in fp16, zero-padded to 64 columns (GEMM path only)
 //   tok_sc   [M]         float    gamma_x[m] * gamma_W / 127 (GEMM path only)
 //   gb16     [N][64]     half     gate[n] * B[j][n], zero-padded to 64 columns (GEMM path only)
 // On the GEMM path the per-token arrays have room for M rounded up to 128: the kernel fetches them
 // 128 tokens at a time (what lies past M is never used).
 struct WsLayout {
-    size_t xq, gamma_x, row_sum, h, h_hi, h_lo, h16, tok_sc, gb16, total;
+    size_t xq, gamma_x, row_sum, h, h_hi, h_lo, hpart, h16, tok_sc, gb16, total;
 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -56,6 +57,7 @@ static inline WsLayout ws_layout(int64_t M, int64_t d_in, int64_t d_out, int32_t
     L.h = off;       off += align_up((size_t)M * rr * 4, 256);
     L.h_hi = off;    off += gemm_path ? 0 : align_up((size_t)M * rr * 2, 256);
     L.h_lo = off;    off += gemm_path ? 0 : align_up((size_t)M * rr * 2, 256);
+    L.hpart = off;   off += (gemm_path || r <= 0) ? 0 : (size_t)(r / 16) * (size_t)((d_in + 255) / 256) * 1024;
     L.h16 = off;     off += gemm_path ? align_up((size_t)M * 64 * 2, 256) : 0;
     L.tok_sc = off;  off += gemm_path ? align_up(Mp * 4, 256) : 0;
     L.gb16 = off;    off += (gemm_path && r > 0) ? align_up((size_t)d_out * 64 * 2, 256) : 0;
@@ -71,6 +73,7 @@ struct PrologueParams {
     float *gamma_x;          // [M]
     int32_t *row_sum;        // [M], nullable
     float *h;                // [M][r]
+    float *hpart;            // decode path, optional: per (16 columns of H, K slice) the 8 x 32 partial sums of x A
     __half *h_hi, *h_lo;     // [M][r] each (decode path) or null
     __half *h16;             // [M][64] (GEMM path) or null
     int8_t *dbg_xq;          // nullable debug copies
@@ -78,7 +81,9 @@ struct PrologueParams {
     float *dbg_h;
     int M, K, r;
     uint32_t flags;
+    int nslices;             // K slices behind hpart
 };
+static_assert(sizeof(PrologueParams) <= 128, "the decode prologue's parameter block: see GemmPrologueExtra");
 
 // What the GEMM path's prologue kernels produce beyond PrologueParams (kept apart so that the decode
 // kernels' parameter block stays as small as it was).
@@ -153,7 +158,7 @@ struct QuantItem {
     int32_t *row_sum;          // its sum of quantised values
     int K, pad;
 };
-static inline int prologue_slice_k(int max_M) { return max_M <= 8 ? 512 : 256; }
+__host__ __device__ inline int prologue_slice_k(int max_M) { return max_M <= 8 ? 512 : 256; }
 cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_quant,
                                          const LoraItem *d_lora_items, int n_lora, int max_M, bool pdl,
                                          cudaStream_t stream);

@@ -169,8 +169,10 @@ __device__ __forceinline__ uint4 ldg_nc_u4(const void *ptr) {
 // exact inputs and accumulated in fp32.  The rows of A^T are the 16-row operand, the tokens the
 // 8-column operand; the warps split K in 32-element chunks and their partial sums are added in a
 // fixed order through shared memory.  NT = number of 8-token tiles.
+// With `hpart` the block covers only the 32-column chunks [cbeg, cend) of K and parks its raw sums
+// there (MMA accumulator layout: [register][lane]); the GEMV adds the slices and applies the SiLU.
 template <int NT>
-__device__ __forceinline__ void lora_down_tile(const PrologueParams &p, int jt) {
+__device__ __forceinline__ void lora_down_tile(const PrologueParams &p, int jt, int cbeg, int cend, float *hpart) {
     __shared__ float s_red[kWarps][NT * 4][32];
     const int K = p.K, M = p.M, r = p.r, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const __half *rowA = p.At + (size_t)(16 * jt + g) * K + 8 * t;
@@ -188,9 +190,9 @@ __device__ __forceinline__ void lora_down_tile(const PrologueParams &p, int jt) 
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[nt][c] = 0.0f;
 
-    const int nchunks = K / 32;
+    const int nchunks = cend;
     constexpr int U = 4;  // chunks in flight per warp
-    for (int c0 = warp; c0 < nchunks; c0 += U * kWarps) {
+    for (int c0 = cbeg + warp; c0 < nchunks; c0 += U * kWarps) {
         uint4 av[U], bv[U], xv[U][NT];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -236,7 +238,9 @@ __device__ __forceinline__ void lora_down_tile(const PrologueParams &p, int jt) 
         for (int w = 0; w < kWarps; ++w) z += s_red[w][idx][ln];
         // accumulator register c of lane (g, t): row g + 8 (c >> 1), token 8 nt + 2 t + (c & 1)
         const int j = 16 * jt + (ln >> 2) + 8 * (c >> 1), m = 8 * nt + 2 * (ln & 3) + (c & 1);
-        if (m < M) {
+        if (hpart) {
+            hpart[idx * 32 + ln] = z;
+        } else if (m < M) {
             const float h = (p.flags & HGF_FLAG_NO_SILU) ? z : silu_f(z);
             const size_t o = (size_t)m * r + j;
             p.h[o] = h;
@@ -250,8 +254,8 @@ __device__ __forceinline__ void lora_down_tile(const PrologueParams &p, int jt) 
     }
 }
 
-__device__ __forceinline__ void lora_down_block(const PrologueParams &p, int jt) {
-    if (p.M <= 8) lora_down_tile<1>(p, jt); else lora_down_tile<2>(p, jt);
+__device__ __forceinline__ void lora_down_block(const PrologueParams &p, int jt, int cbeg, int cend, float *hpart) {
+    if (p.M <= 8) lora_down_tile<1>(p, jt, cbeg, cend, hpart); else lora_down_tile<2>(p, jt, cbeg, cend, hpart);
 }
 
 // Many rows of up to 4096 elements (quantisation alone): one warp per token row, the row held in registers between the maximum and
@@ -301,14 +305,21 @@ __global__ void __launch_bounds__(kThreads) quant_kernel(const PrologueParams p,
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 
-// Decode prologue: blocks [0, M) quantise one token each, blocks [M, M + r / 16) compute 16 columns of H.
+// Decode prologue: blocks [0, M) quantise one token each; the others compute 16 columns of H each,
+// over all of K, or - with a scratch for partial sums - over one K slice each (slice-major), which
+// shortens the chain of dependent loads from K / 1024 rounds to one or two.
 __global__ void __launch_bounds__(kThreads) decode_prologue_kernel(const PrologueParams p) {
     pdl_launch_dependents();  // the GEMV that follows may start streaming its weights
     pdl_wait();               // x, and the workspace this kernel overwrites, belong to earlier work
     if ((int)blockIdx.x < p.M)
         quant_row(p, blockIdx.x);
-    else
-        lora_down_block(p, blockIdx.x - p.M);
+    else if (p.hpart) {
+        const int lb = blockIdx.x - p.M, jts = p.r / 16, sl = lb / jts, jt = lb - sl * jts;
+        const int per = prologue_slice_k(p.M) / 32, cbeg = sl * per, cend = cbeg + per < p.K / 32 ? cbeg + per : p.K / 32;
+        lora_down_block(p, jt, cbeg, cend, p.hpart + ((size_t)jt * p.nslices + sl) * 256);
+    } else {
+        lora_down_block(p, blockIdx.x - p.M, 0, p.K / 32, nullptr);
+    }
 }
 
 // ---- group prologue: persistent CTAs, one warp per work item ------------------------------------
@@ -784,7 +795,7 @@ cudaLaunchConfig_t prologue_cfg(int blocks, bool pdl, cudaStream_t stream, cudaL
 
 cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream_t stream) {
     cudaLaunchAttribute attr[1];
-    cudaLaunchConfig_t cfg = prologue_cfg(p.M + p.r / 16, pdl, stream, attr);
+    cudaLaunchConfig_t cfg = prologue_cfg(p.M + (p.r / 16) * (p.hpart ? p.nslices : 1), pdl, stream, attr);
     cudaError_t e = cudaLaunchKernelEx(&cfg, decode_prologue_kernel, p);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();

@@ -136,6 +136,24 @@ def test_decode_every_token_count_and_ragged_shapes(hgf, M):
     check_layer(hgf, syn.LayerShape("tiny", 64, 8, 48), M, config=9, layer=100 + M, tol2=TOL_DECODE)
 
 
+@pytest.mark.parametrize("M,K,N,r", [(1, 2048, 512, 32), (3, 5632, 256, 32), (8, 448, 72, 16), (9, 1088, 264, 48),
+                                     (16, 3200, 328, 64), (2, 11008, 128, 64)])
+def test_decode_without_debug_outputs(hgf, M, K, N, r):
+    """The plain call (no debug outputs) computes x A in K slices spread over more blocks; its y must
+    meet the same bar as the call that also reports H."""
+    shape = syn.LayerShape("nd", K, N, r)
+    _, y_dbg, ref = check_layer(hgf, shape, M, config=15, layer=M, tol2=TOL_DECODE)
+    packed, gamma, _ = packed_layer(hgf, shape, 15, M)
+    x = syn.make_x(M, K, config=15, layer=M)
+    At, Bt, gate = syn.make_lora(K, N, r, config=15, layer=M)
+    y = hgf.linear_forward(dev(x, torch.bfloat16), packed, float(gamma), K, N, dev(At, torch.float16),
+                           dev(Bt, torch.float16), dev(gate))
+    hgf.check_status()
+    scale = np.abs(ref["y"]).max()
+    assert np.abs(y.cpu().numpy().astype(np.float64) - ref["y"]).max() / scale <= TOL_DECODE
+    assert (y - y_dbg).abs().max().item() <= 2e-6 * scale
+
+
 def test_decode_pure_bitlinear_and_gate_zero(hgf):
     shape = syn.LayerShape("p", 1024, 512, 32)
     _, y_pure, ref = check_layer(hgf, shape, 4, config=8, lora=False, tol2=TOL_DECODE)
