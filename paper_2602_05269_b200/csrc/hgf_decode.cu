@@ -5,7 +5,8 @@
 // The kernel is bound by the packed-weight stream from HBM, so it is built around keeping that
 // stream busy.  One persistent CTA of 16 warps per SM.  The weights of all problems of the launch
 // form one long sequence of 1 KiB tiles (16 output rows x 256 input columns); it is cut into
-// contiguous shares of equal cost (weight tiles plus a fixed charge per row tile), one per CTA.  Every warp owns a private ring of 1 KiB shared-memory slots
+// contiguous shares of equal cost (weight tiles plus a fixed charge per row tile), one per CTA.
+// Every warp owns a private ring of shared-memory slots (two of 4 KiB, or three to four of 2 KiB)
 // that one of its lanes keeps filled with bulk asynchronous copies (cp.async.bulk, completion on an
 // mbarrier), several tiles ahead of their use and across row-tile, layer and (under programmatic
 // dependent launch) kernel boundaries, so the number of bytes in flight does not depend on what
@@ -26,10 +27,12 @@ namespace hgf {
 constexpr int kDecWarps = 16;
 constexpr int kDecThreads = kDecWarps * 32;
 constexpr int kTileBytes = 1024;     // one 16 x 256 weight tile
-constexpr int kSlotTiles = 2;        // tiles per ring slot (the consumer loop is written for 2)
-constexpr int kSlotBytes = kSlotTiles * kTileBytes;
-constexpr int kMaxSlots = 4;         // slots per warp ring (fewer when the activations need the room)
-constexpr int kMinSlots = 3;
+// A warp's ring is either two slots of four tiles (fewer, larger copies and hand-overs: measured
+// 6 % faster) or, when the activations leave no room for that, three to four slots of two tiles.
+constexpr int kBigSlotTiles = 4, kBigSlots = 2;
+constexpr int kSmallSlotTiles = 2;
+constexpr int kMaxSlots = 4;         // slots per warp ring at most (barriers are laid out for that many)
+constexpr int kMinSlots = 3;         // small slots at least: what bounds the activations' share of shared memory
 constexpr int kXqPad = 64;           // row padding of the activations in shared memory (bank spread)
 constexpr int kHPitch = 72;          // halves per row of H in shared memory (r <= 64, + 8 bank spread)
 
@@ -52,7 +55,7 @@ constexpr int kRedBytes = kDecWarps * 8 * 32 * 4;  // per warp: up to 8 accumula
 constexpr int kOffFlags = kOffRed + kRedBytes;
 constexpr int kOffXq = (kOffFlags + 64 + 127) / 128 * 128;
 constexpr int kSmemLimit = 227 * 1024;
-constexpr int kXqLimit = (kSmemLimit - kOffXq - kMinSlots * kDecWarps * kSlotBytes) / 128 * 128;
+constexpr int kXqLimit = (kSmemLimit - kOffXq - kMinSlots * kDecWarps * kSmallSlotTiles * kTileBytes) / 128 * 128;
 
 constexpr unsigned long long kDecWaitLimitNs = 2000000000ull;  // bounded waits give up after two seconds
 
@@ -219,10 +222,11 @@ struct Producer {
     bool done;
 };
 
-// NT = number of 8-token tiles (1: M <= 8, 2: M <= 16).
-template <int NT>
+// NT = number of 8-token tiles (1: M <= 8, 2: M <= 16); ST = tiles per ring slot.
+template <int NT, int ST>
 __global__ void __launch_bounds__(kDecThreads, 1)
 decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned int *status) {
+    constexpr int kSlotTiles = ST, kSlotBytes = ST * kTileBytes;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int slots = L.ring_slots;  // slots of this warp's ring, kSlotBytes each
@@ -524,22 +528,20 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) xt[nt] = xrow[nt] + it.ks0 * 256;
             const int ntiles = it.ks1 - it.ks0;
-            for (int i = ntiles >> 1; i > 0 && ok; --i) {  // full slots
+            for (int left = ntiles; left > 0 && ok;) {  // slot by slot; the last may hold fewer tiles
                 if (!(ok = wait_slot())) break;  // stop computing and copying; requested slots stay outstanding
                 const uint8_t *sl = ring + cslot * kSlotBytes + 16 * lane;
-                compute_tile(sl, xt);
+                const int n = left < kSlotTiles ? left : kSlotTiles;
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) xt[nt] += 256;
-                compute_tile(sl + kTileBytes, xt);
+                for (int q = 0; q < kSlotTiles; ++q) {
+                    if (q < n) {
+                        compute_tile(sl + q * kTileBytes, xt);
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) xt[nt] += 256;
-                release_slot();
-            }
-            if ((ntiles & 1) && ok) {  // a last slot with one tile
-                if ((ok = wait_slot())) {
-                    compute_tile(ring + cslot * kSlotBytes + 16 * lane, xt);
-                    release_slot();
+                        for (int nt = 0; nt < NT; ++nt) xt[nt] += 256;
+                    }
                 }
+                release_slot();
+                left -= n;
             }
 
             // exact rescale of the four accumulators
@@ -599,24 +601,31 @@ int decode_grid(int total_tiles) {
     return total_tiles < g_sm_count ? total_tiles : g_sm_count;
 }
 
-cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *single, bool pdl, cudaStream_t stream) {
+template <int NT, int ST>
+static cudaError_t launch_decode_variant(cudaLaunchConfig_t &cfg, const DecodeLaunch &L, const DecodeProblem &sp, unsigned int *status) {
     static bool attr_set = false;
-    const int grid = decode_grid(L_in.total_tiles);
-    if (grid <= 0) return cudaErrorInvalidDevice;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(decode_gemv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(decode_gemv_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        cudaError_t e = cudaFuncSetAttribute(decode_gemv_kernel<NT, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
+    return cudaLaunchKernelEx(&cfg, decode_gemv_kernel<NT, ST>, L, sp, status);
+}
+
+cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *single, bool pdl, cudaStream_t stream) {
+    const int grid = decode_grid(L_in.total_tiles);
+    if (grid <= 0) return cudaErrorInvalidDevice;
     if (L_in.xq_smem_bytes > kXqLimit) return cudaErrorInvalidValue;
     unsigned int *status = device_status_word();
     if (!status) return cudaErrorMemoryAllocation;
     DecodeLaunch L = L_in;
-    // as many ring slots as shared memory allows beside the activations
+    // the ring beside the activations: two slots of four tiles if they fit, else as many slots of two
+    // tiles as shared memory allows
     const int xq_bytes = (L.xq_smem_bytes + 127) & ~127;
-    int slots = (kSmemLimit - kOffXq - xq_bytes) / (kDecWarps * kSlotBytes);
+    const int room = kSmemLimit - kOffXq - xq_bytes;
+    const bool big = room >= kDecWarps * kBigSlots * kBigSlotTiles * kTileBytes;
+    const int slot_bytes = (big ? kBigSlotTiles : kSmallSlotTiles) * kTileBytes;
+    int slots = big ? kBigSlots : room / (kDecWarps * slot_bytes);
     slots = slots > kMaxSlots ? kMaxSlots : slots;
     L.ring_slots = slots;
     DecodeProblem dummy = {};
@@ -625,15 +634,18 @@ cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *si
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kDecThreads);
-    cfg.dynamicSmemBytes = (size_t)(kOffXq + xq_bytes + kDecWarps * slots * kSlotBytes);
+    cfg.dynamicSmemBytes = (size_t)(kOffXq + xq_bytes + kDecWarps * slots * slot_bytes);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    cudaError_t e = L.max_M <= 8 ? cudaLaunchKernelEx(&cfg, decode_gemv_kernel<1>, L, sp, status)
-                                 : cudaLaunchKernelEx(&cfg, decode_gemv_kernel<2>, L, sp, status);
+    cudaError_t e;
+    if (L.max_M <= 8)
+        e = big ? launch_decode_variant<1, kBigSlotTiles>(cfg, L, sp, status) : launch_decode_variant<1, kSmallSlotTiles>(cfg, L, sp, status);
+    else
+        e = big ? launch_decode_variant<2, kBigSlotTiles>(cfg, L, sp, status) : launch_decode_variant<2, kSmallSlotTiles>(cfg, L, sp, status);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }
