@@ -380,8 +380,8 @@ def run_ours(args):
 # DRAM traffic of the decode GEMV launch from the committed ncu capture (profiles/): bytes moved
 # per algorithmic byte on the captured case.  It is only reported while the kernel source is the one
 # that was profiled.
-DECODE_TRAFFIC = {"source_sha1": "7d8e5a601f48bb095f7b23d6e93e0864017a71eb",
-                  "dram_bytes_per_algorithmic_byte": (517.347840e6 + 6.013952e6) / 518805504.0,
+DECODE_TRAFFIC = {"source_sha1": "6a7ec3df9f3fb531d0b7c707a2f325a9ca75d120",
+                  "dram_bytes_per_algorithmic_byte": (517.358848e6 + 6.933248e6) / 518805504.0,
                   "profile": "profiles/decode_gemv_config1_m1.md"}
 
 
