@@ -246,6 +246,16 @@ def test_gemm_pure_bitlinear_gate_zero_and_flags(hgf):
     check_layer(hgf, shape, 4, config=11, flags=hgf.FLAG_FORCE_GEMM, tol2=TOL_GEMM)
 
 
+def test_gemm_long_rows_without_correction_and_without_dependent_launch(hgf):
+    """Rows too long for the warp-per-row quantisation (the prologue kernel without its LoRA part feeds
+    the GEMM), and the GEMM path with programmatic dependent launch switched off: same results."""
+    shape = syn.LayerShape("long", 4352, 264, 32)
+    check_layer(hgf, shape, 300, config=16, lora=False, tol2=TOL_DECODE)
+    _, y1, _ = check_layer(hgf, shape, 300, config=16, tol2=TOL_GEMM)
+    _, y2, _ = check_layer(hgf, shape, 300, config=16, flags=hgf.FLAG_NO_PDL, tol2=TOL_GEMM)
+    assert torch.equal(y1, y2)
+
+
 def test_config3_prefill_m512_full(hgf):
     for i, shape in enumerate(syn.distinct_shapes(3)):
         check_layer(hgf, shape, 512, config=3, layer=i, tol2=TOL_GEMM)
