@@ -45,7 +45,9 @@ typedef enum {
 /* flags of hgf_linear_forward / hgf_workspace_bytes */
 #define HGF_FLAG_OUT_BF16 0x1u /* y is bfloat16 instead of fp32 */
 #define HGF_FLAG_NO_SILU 0x2u  /* correction is (x A) B, without the SiLU the paper defines */
-#define HGF_FLAG_FORCE_GEMM 0x4u /* route to the tensor-core GEMM path even when M <= 16 (testing) */
+#define HGF_FLAG_FORCE_GEMM 0x4u /* route to the tensor-core GEMM path even when M <= 16 (a small batch whose
+                                    consumer wants the GEMM path's bf16 tiles; also how the tests reach that
+                                    path on decode-sized inputs) */
 
 #define HGF_FLAG_NO_PDL 0x8u     /* do not use programmatic dependent launch (see hgf_linear_forward) */
 
@@ -131,6 +133,22 @@ hgf_status hgf_linear_forward(const void *x, int64_t M, const void *packed, floa
                               void *stream);
 
 /*
+ * The two launches of hgf_linear_forward separately (both bits together are hgf_linear_forward):
+ * HGF_PHASE_PROLOGUE runs Algorithm 1 steps 1-2 and 5-6 (activation quantisation, H = SiLU(x A))
+ * into the workspace; HGF_PHASE_GEMV runs steps 3-4 and 7-8 (the ternary contraction - GEMV or
+ * tensor-core GEMM, whichever path the problem takes - with dequantisation, up-projection and gated
+ * fusion) from what the last prologue call with the same arguments left in the workspace.  For
+ * timing the two kernels apart, and for callers that re-run the contraction of an unchanged input.
+ */
+#define HGF_PHASE_PROLOGUE 0x1u
+#define HGF_PHASE_GEMV 0x2u
+hgf_status hgf_linear_forward_phases(const void *x, int64_t M, const void *packed, float gamma,
+                                     int64_t d_in, int64_t d_out, const void *At, const void *Bt,
+                                     int32_t r, const float *gate, void *y, void *workspace,
+                                     size_t workspace_bytes, const hgf_debug_out *dbg, uint32_t flags,
+                                     uint32_t phases, void *stream);
+
+/*
  * hgf_linear_forward for callers that cannot hand over a workspace.  (The paper has no counterpart:
  * this is a convenience of the library, not a step of the method.)
  *
@@ -147,10 +165,12 @@ hgf_status hgf_linear_forward(const void *x, int64_t M, const void *packed, floa
  * without workspace and debug outputs; results are the same.
  *
  * Limits: only decode-sized problems (those hgf_linear_forward serves with its GEMV path, M <=
- * HGF_DECODE_MAX_M) whose hgf_workspace_bytes(M, d_in, d_out, r, flags) is at most
- * HGF_STATIC_SCRATCH_BYTES; e.g. M = 16 with d_in <= 6656, or M = 1 with any supported d_in.
- * A problem that needs more scratch returns HGF_ERR_TOO_LARGE, one that would take the GEMM path
- * HGF_ERR_UNSUPPORTED_SHAPE; nothing is launched in either case.
+ * HGF_DECODE_MAX_M) with hgf_workspace_bytes(M, d_in, d_out, r, flags) <= HGF_STATIC_SCRATCH_BYTES.
+ * The scratch holds M * d_in bytes of quantised activations plus (r / 16) * ceil(d_in / 256) KiB of
+ * partial sums of x A and a few KiB of per-token values: with r = 64 that is every model shape of
+ * the paper at M = 16 up to d_in = 6656 and at M = 1 up to d_in = 16384; M = 1, d_in = 32768, r = 64
+ * does not fit.  A problem that needs more returns HGF_ERR_TOO_LARGE; an unsupported rank, or a
+ * problem that would take the GEMM path, HGF_ERR_UNSUPPORTED_SHAPE; nothing is launched then.
  *
  * Sharing: all calls on a device use the same array, and it keeps what the last call left in it.
  * Nothing in it has to be cleared (each call writes every value before reading it), but two calls
@@ -209,9 +229,17 @@ hgf_status hgf_group_forward(hgf_group *group, void *stream);
  * workspace, HGF_PHASE_GEMV steps 3-4 and 7-8 from what the last prologue left there.  Both bits
  * together are hgf_group_forward.
  */
-#define HGF_PHASE_PROLOGUE 0x1u
-#define HGF_PHASE_GEMV 0x2u
 hgf_status hgf_group_forward_phases(hgf_group *group, uint32_t phases, void *stream);
+/*
+ * Parity-check access to problem `index` of a group (Algorithm 1, steps 1-3 as the group's own
+ * kernels compute them).  y_int: nullable device buffer [M][d_out] owned by the caller; from the
+ * next forward on, the GEMV also writes the problem's integer accumulators there (null switches
+ * that off again).  views: nullable host struct that receives device pointers INTO the group's
+ * workspace - xq [M][d_in] and gamma_x [M] as the last forward left them (problems that share an
+ * input share these) - plus y_int as passed; h is set to null (the group keeps x A in K slices).
+ * A set-up call: it synchronises the device; no forward of the group may be running.
+ */
+hgf_status hgf_group_debug(hgf_group *group, int32_t index, int32_t *y_int, hgf_debug_out *views);
 void hgf_group_destroy(hgf_group *group);
 
 /*

@@ -31,6 +31,23 @@ unsigned int *device_status_word() {
     return cached_ptr;
 }
 
+int current_device() {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
+
+int device_sm_count() {
+    static std::atomic<int> cache[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0 || dev >= kMaxDevices) return 0;
+    int n = cache[dev].load(std::memory_order_acquire);
+    if (!n) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 0;
+        cache[dev].store(n, std::memory_order_release);
+    }
+    return n;
+}
+
 static bool misaligned(const void *p) { return p && (((uintptr_t)p) & 15u); }
 
 // The decode path keeps a problem's quantised activations in shared memory; problems too large
@@ -142,6 +159,16 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
                                          int64_t d_out, const void *At, const void *Bt, int32_t r,
                                          const float *gate, void *y, void *workspace, size_t workspace_bytes,
                                          const hgf_debug_out *dbg, uint32_t flags, void *stream_) {
+    return hgf_linear_forward_phases(x, M, packed, gamma, d_in, d_out, At, Bt, r, gate, y, workspace, workspace_bytes, dbg,
+                                     flags, HGF_PHASE_PROLOGUE | HGF_PHASE_GEMV, stream_);
+}
+
+extern "C" hgf_status hgf_linear_forward_phases(const void *x, int64_t M, const void *packed, float gamma, int64_t d_in,
+                                                int64_t d_out, const void *At, const void *Bt, int32_t r,
+                                                const float *gate, void *y, void *workspace, size_t workspace_bytes,
+                                                const hgf_debug_out *dbg, uint32_t flags, uint32_t phases, void *stream_) {
+    if (!phases || (phases & ~(HGF_PHASE_PROLOGUE | HGF_PHASE_GEMV))) return HGF_ERR_INVALID_ARG;
+    const bool do_prologue = (phases & HGF_PHASE_PROLOGUE) != 0, do_main = (phases & HGF_PHASE_GEMV) != 0;
     bool gemm = false;
     hgf_status st = validate_problem(x, M, packed, d_in, d_out, At, Bt, r, gate, y, flags, &r, &gemm);
     if (st != HGF_OK) return st;
@@ -158,7 +185,8 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
     fill_params(x, M, packed, gamma, d_in, d_out, At, Bt, r, gate, y, (char *)workspace, L, gemm, dbg, flags, &pp, &dp);
 
     if (!gemm) {
-        if (launch_decode_prologue(pp, pdl, stream) != cudaSuccess) return HGF_ERR_CUDA;
+        if (do_prologue && launch_decode_prologue(pp, pdl, stream) != cudaSuccess) return HGF_ERR_CUDA;
+        if (!do_main) return HGF_OK;
         DecodeLaunch dl = {};
         dl.probs = nullptr;
         dl.n_probs = 1;
@@ -176,7 +204,9 @@ extern "C" hgf_status hgf_linear_forward(const void *x, int64_t M, const void *p
     gx.gate = gate;
     gx.gw_over_127 = dp.gw_over_127;
     gx.N = (int)d_out;
-    if ((r ? launch_gemm_prologue(pp, gx, stream) : launch_quant(pp, gx, stream)) != cudaSuccess) return HGF_ERR_CUDA;
+    if (do_prologue && (r ? launch_gemm_prologue(pp, gx, stream) : launch_quant(pp, gx, stream)) != cudaSuccess)
+        return HGF_ERR_CUDA;
+    if (!do_main) return HGF_OK;
     GemmParams gp = {};
     gp.xq = pp.xq;
     gp.packed = (const uint8_t *)packed;
@@ -224,6 +254,7 @@ extern "C" hgf_status hgf_linear_forward_static(const void *x, int64_t M, const 
     if (flags & HGF_FLAG_FORCE_GEMM) return HGF_ERR_INVALID_ARG;
     if (d_in % 64 != 0 || d_in > 65536 || M > HGF_DECODE_MAX_M) return HGF_ERR_UNSUPPORTED_SHAPE;
     const int32_t r_eff = (At && Bt && gate) ? r : 0;
+    if (r_eff != 0 && r_eff != 16 && r_eff != 32 && r_eff != 48 && r_eff != 64) return HGF_ERR_UNSUPPORTED_SHAPE;
     if (ws_layout(M, d_in, d_out, r_eff, false).total > (size_t)HGF_STATIC_SCRATCH_BYTES) return HGF_ERR_TOO_LARGE;
     if (takes_gemm_path(M, d_in, flags)) return HGF_ERR_UNSUPPORTED_SHAPE;
     void *scratch = static_scratch_address();
@@ -234,7 +265,8 @@ extern "C" hgf_status hgf_linear_forward_static(const void *x, int64_t M, const 
 
 // ---- groups of independent decode problems --------------------------------------------------------
 struct hgf_group {
-    int n, total_tiles, total_blocks, max_M, xq_smem_bytes, device;
+    int n, total_tiles, max_M, xq_smem_bytes, device;
+    std::vector<DecodeProblem> h_probs;  // host copy of the descriptors (hgf_group_debug edits one and re-uploads it)
     long long total_cost;
     uint32_t flags;
     void *d_mem;              // one allocation: descriptors, block offsets, workspaces
@@ -258,8 +290,9 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     std::vector<WsLayout> lay((size_t)n);
     std::vector<int32_t> ranks((size_t)n);
     size_t ws_total = 0;
-    int tiles = 0, blocks = 0, max_M = 0, xq_smem = 0;
+    int tiles = 0, max_M = 0, xq_smem = 0;
     long long cost = 0;
+    int64_t tiles64 = 0;
     for (int i = 0; i < n; ++i) {
         const hgf_problem &q = problems[i];
         bool gemm = false;
@@ -270,7 +303,9 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         ranks[i] = r;
         lay[i] = ws_layout(q.M, q.d_in, q.d_out, r, false);
         ws_total += lay[i].total;
-        if (tiles > (1 << 30) - (1 << 21)) return HGF_ERR_UNSUPPORTED_SHAPE;
+        // the kernels number the launch's row tiles (and the items of the prologue) with 32-bit integers
+        tiles64 += row_tiles(q.d_out);
+        if (tiles64 > (int64_t)1 << 30) return HGF_ERR_UNSUPPORTED_SHAPE;
     }
     const size_t off_probs = 0;
     const size_t off_pps = align_up(off_probs + sizeof(DecodeProblem) * (size_t)n, 256);
@@ -283,6 +318,7 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         n_quant += (size_t)problems[i].M;  // an upper bound: problems that share x share their items
         n_lora += ((size_t)ranks[i] / 16) * (size_t)((problems[i].d_in + slice_k - 1) / slice_k);
     }
+    if (n_quant > ((size_t)1 << 30) || n_lora > ((size_t)1 << 30)) return HGF_ERR_UNSUPPORTED_SHAPE;
     const size_t off_qit = align_up(off_pps + sizeof(PrologueParams) * (size_t)n, 256);
     const size_t off_lit = align_up(off_qit + sizeof(QuantItem) * n_quant, 256);
     const size_t off_cta = align_up(off_lit + sizeof(LoraItem) * n_lora, 256);
@@ -340,14 +376,13 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         }
         tiles += (int)row_tiles(q.d_out);
         cost += (long long)row_tiles(q.d_out) * row_tile_cost((int)q.d_in);
-        blocks += (int)q.M + ranks[i] / 16;
         max_M = q.M > max_M ? (int)q.M : max_M;
         const int xb = decode_xq_smem_bytes((int)q.M, (int)q.d_in);
         xq_smem = xb > xq_smem ? xb : xq_smem;
     }
     hgf_group *g = new (std::nothrow) hgf_group();
     if (!g) { cudaFree(mem); return HGF_ERR_CUDA; }
-    g->n = n; g->total_tiles = tiles; g->total_blocks = blocks; g->max_M = max_M; g->xq_smem_bytes = xq_smem;
+    g->n = n; g->total_tiles = tiles; g->max_M = max_M; g->xq_smem_bytes = xq_smem;
     g->total_cost = cost;
     g->flags = flags; g->d_mem = mem;
     g->d_probs = (DecodeProblem *)((char *)mem + off_probs);
@@ -392,7 +427,25 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
               (ranges.empty() ||
                cudaMemcpy(g->d_cta_range, ranges.data(), sizeof(int4) * ranges.size(), cudaMemcpyHostToDevice) == cudaSuccess);
     if (!ok) { cudaFree(mem); delete g; return HGF_ERR_CUDA; }
+    g->h_probs = std::move(dps);
     *out = g;
+    return HGF_OK;
+}
+
+extern "C" hgf_status hgf_group_debug(hgf_group *g, int32_t index, int32_t *y_int, hgf_debug_out *views) {
+    if (!g || index < 0 || index >= g->n) return HGF_ERR_INVALID_ARG;
+    if (misaligned(y_int)) return HGF_ERR_MISALIGNED;
+    DecodeProblem &P = g->h_probs[(size_t)index];
+    if (P.dbg_y_int != y_int) {
+        P.dbg_y_int = y_int;
+        if (cudaMemcpy(g->d_probs + index, &P, sizeof(DecodeProblem), cudaMemcpyHostToDevice) != cudaSuccess) return HGF_ERR_CUDA;
+    }
+    if (views) {
+        views->xq = const_cast<int8_t *>(P.xq);
+        views->gamma_x = const_cast<float *>(P.gamma_x);
+        views->y_int = y_int;
+        views->h = nullptr;
+    }
     return HGF_OK;
 }
 

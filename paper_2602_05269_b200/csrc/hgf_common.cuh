@@ -7,6 +7,8 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <atomic>
+
 #include "../../include/hgf.h"
 
 #if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ < 1000)
@@ -18,6 +20,26 @@ namespace hgf {
 // ---- launch accounting and the device-side status word ------------------------------------
 void count_launch(int n = 1);
 unsigned int *device_status_word();  // per-device word in global memory; nonzero = a wait gave up
+
+// ---- per-device launch set-up -----------------------------------------------------------------
+// A process may drive several GPUs: the SM count and the opt-in to large dynamic shared memory
+// (an attribute of the kernel on ONE device) are looked up for the device that is current.
+constexpr int kMaxDevices = 64;
+int current_device();      // ordinal of the current device, or -1
+int device_sm_count();     // SM count of the current device (cached per device), 0 if it cannot be queried
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per device; `done` is a per-kernel bit mask
+// of the devices already set up (one static instance beside each kernel's launcher).
+template <typename Kernel>
+static inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, std::atomic<unsigned long long> &done) {
+    const int dev = current_device();
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    const unsigned long long bit = 1ull << dev;
+    if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return e;
+    done.fetch_or(bit, std::memory_order_release);
+    return cudaSuccess;
+}
 
 // ---- packed weight layout ---------------------------------------------------------------------
 // Tiles of 16 output rows x 256 input columns, 1 KiB each, row-major inside the tile (64 bytes per

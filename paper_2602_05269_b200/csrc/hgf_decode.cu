@@ -590,25 +590,16 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
     }
 }
 
-static int g_sm_count = 0;
 int decode_grid(int total_tiles) {
-    if (!g_sm_count) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        g_sm_count = n;
-    }
-    return total_tiles < g_sm_count ? total_tiles : g_sm_count;
+    const int sms = device_sm_count();
+    return total_tiles < sms ? total_tiles : sms;
 }
 
 template <int NT, int ST>
 static cudaError_t launch_decode_variant(cudaLaunchConfig_t &cfg, const DecodeLaunch &L, const DecodeProblem &sp, unsigned int *status) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(decode_gemv_kernel<NT, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> attr_done{0};
+    cudaError_t e = ensure_dynamic_smem(decode_gemv_kernel<NT, ST>, kSmemLimit, attr_done);
+    if (e != cudaSuccess) return e;
     return cudaLaunchKernelEx(&cfg, decode_gemv_kernel<NT, ST>, L, sp, status);
 }
 

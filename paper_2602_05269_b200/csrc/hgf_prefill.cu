@@ -633,12 +633,11 @@ static bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, const void *ba
 template <bool OUT_BF16, int NS, int OPSB>
 static cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &mh, const CUtensorMap &mgb, const CUtensorMap &my,
                                   const GemmParams &p, int grid, unsigned int *status, cudaStream_t stream) {
-    static bool attr_set = false;
+    static std::atomic<unsigned long long> attr_done{0};
     constexpr int smem = Cfg<NS, OPSB>::SMEM_BYTES;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_gemm_kernel<OUT_BF16, NS, OPSB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    {
+        cudaError_t e = ensure_dynamic_smem(prefill_gemm_kernel<OUT_BF16, NS, OPSB>, smem, attr_done);
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -655,14 +654,8 @@ static cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &mh, 
 }
 
 cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
-    static int sm_count = 0;
-    if (!sm_count) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-    }
+    const int sm_count = device_sm_count();
+    if (!sm_count) return cudaErrorInvalidDevice;
     const bool bf16 = (p.flags & HGF_FLAG_OUT_BF16) != 0;
     const bool narrow = p.r <= 32;  // 64-byte operand rows for the correction, and room for a fourth stage
     CUtensorMap mx, mh, mgb, my;

@@ -712,11 +712,10 @@ static cudaError_t launch_gemm_prologue_jt(const PrologueParams &p, const GemmPr
     // blocks): blocks that start as SMs come free at the tail of the preceding launch would otherwise
     // pile up four to an SM on the first SMs free and leave the others idle.
     constexpr int smem = fp_smem_bytes(8 * JT) > 80 * 1024 ? fp_smem_bytes(8 * JT) : 80 * 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_prologue_kernel<JT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    static std::atomic<unsigned long long> attr_done{0};
+    {
+        cudaError_t e = ensure_dynamic_smem(gemm_prologue_kernel<JT>, smem, attr_done);
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     cudaLaunchAttribute attr[1];
     cudaLaunchConfig_t cfg = prologue_cfg(blocks, !(p.flags & HGF_FLAG_NO_PDL), stream, attr);
@@ -730,12 +729,8 @@ static cudaError_t launch_gemm_prologue_jt(const PrologueParams &p, const GemmPr
 cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream) {
     // Tokens per block: as many blocks as are resident at once share the rows evenly; beyond that a
     // block takes its full 32.
-    static int sm_count = 0;
-    if (!sm_count) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return cudaErrorInvalidDevice;
-    }
+    const int sm_count = device_sm_count();
+    if (!sm_count) return cudaErrorInvalidDevice;
     const int per_sm = p.r >= 48 ? 1 : 2;  // blocks that fit an SM (shared memory: 138 KB and more from rank 48 on)
     int tpb = (p.M + per_sm * sm_count - 1) / (per_sm * sm_count);
     tpb = (tpb + 3) / 4 * 4;
@@ -803,22 +798,15 @@ cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream
 
 cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_quant, const LoraItem *d_lora_items, int n_lora, int max_M, bool pdl,
                                          cudaStream_t stream) {
-    static int sm_count = 0;
-    static bool attr_set = false;
-    if (!sm_count) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-    }
+    static std::atomic<unsigned long long> attr_done1{0}, attr_done2{0};
+    const int sm_count = device_sm_count();
+    if (!sm_count) return cudaErrorInvalidDevice;
     const int smem1 = kPgWarps * 16 * (1024 + 512), smem2 = kPgWarps * 8 * (1024 + 1024);
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(decode_prologue_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1);
+    {
+        cudaError_t e = ensure_dynamic_smem(decode_prologue_group_kernel<1>, smem1, attr_done1);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(decode_prologue_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2);
+        e = ensure_dynamic_smem(decode_prologue_group_kernel<2>, smem2, attr_done2);
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     const int most = n_lora > n_quant ? n_lora : n_quant;
     int blocks = (most + kPgWarps - 1) / kPgWarps;

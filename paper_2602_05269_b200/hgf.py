@@ -26,7 +26,8 @@ PHASE_GEMV = 0x2
 EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_workspace_bytes",
            "hgf_linear_forward", "hgf_act_quant", "hgf_check_status", "hgf_tmax_tokens_per_s",
            "hgf_launch_count", "hgf_status_string", "hgf_group_create", "hgf_group_forward",
-           "hgf_group_destroy", "hgf_group_forward_phases", "hgf_linear_forward_static"]
+           "hgf_group_destroy", "hgf_group_forward_phases", "hgf_linear_forward_static", "hgf_group_debug",
+           "hgf_linear_forward_phases"]
 
 
 class HgfError(RuntimeError):
@@ -71,6 +72,9 @@ def lib() -> ctypes.CDLL:
         L.hgf_linear_forward.restype = c.c_int
         L.hgf_linear_forward.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, vp, sz,
                                          c.POINTER(DebugOut), u32, vp]
+        L.hgf_linear_forward_phases.restype = c.c_int
+        L.hgf_linear_forward_phases.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, vp, sz,
+                                                c.POINTER(DebugOut), u32, u32, vp]
         L.hgf_linear_forward_static.restype = c.c_int
         L.hgf_linear_forward_static.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, u32, vp]
         L.hgf_act_quant.restype = c.c_int
@@ -87,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.hgf_group_forward.argtypes = [vp, vp]
         L.hgf_group_forward_phases.restype = c.c_int
         L.hgf_group_forward_phases.argtypes = [vp, u32, vp]
+        L.hgf_group_debug.restype = c.c_int
+        L.hgf_group_debug.argtypes = [vp, i32, vp, c.POINTER(DebugOut)]
         L.hgf_group_destroy.restype = None
         L.hgf_group_destroy.argtypes = [vp]
         L.hgf_status_string.restype = c.c_char_p
@@ -153,7 +159,7 @@ def act_quant(x: torch.Tensor, stream=None):
 
 
 def linear_forward(x, packed, gamma, d_in, d_out, At=None, Bt=None, gate=None, *, y=None, workspace=None,
-                   debug=False, flags=0, stream=None):
+                   debug=False, flags=0, stream=None, phases=None):
     """Enqueue one layer forward.  Returns y, or (y, dbg dict of device tensors) with debug=True.
 
     x bf16 [M][d_in]; packed uint8 from pack_ternary; At fp16 [r][d_in]; Bt fp16 [d_out][r];
@@ -175,10 +181,15 @@ def linear_forward(x, packed, gamma, d_in, d_out, At=None, Bt=None, gate=None, *
                "h": torch.empty((M, max(r, 1)), dtype=torch.float32, device=x.device)}
         dbg_struct = DebugOut(dbg["xq"].data_ptr(), dbg["gamma_x"].data_ptr(), dbg["y_int"].data_ptr(),
                               dbg["h"].data_ptr())
-    st = lib().hgf_linear_forward(_ptr(x), M, _ptr(packed), ctypes.c_float(gamma), d_in, d_out, _ptr(At), _ptr(Bt),
-                                  r, _ptr(gate), _ptr(y), _ptr(workspace), workspace.numel(),
-                                  ctypes.byref(dbg_struct) if dbg_struct is not None else None, flags,
-                                  _stream(stream))
+    dbg_arg = ctypes.byref(dbg_struct) if dbg_struct is not None else None
+    if phases is None:
+        st = lib().hgf_linear_forward(_ptr(x), M, _ptr(packed), ctypes.c_float(gamma), d_in, d_out, _ptr(At), _ptr(Bt),
+                                      r, _ptr(gate), _ptr(y), _ptr(workspace), workspace.numel(), dbg_arg, flags,
+                                      _stream(stream))
+    else:   # hgf_linear_forward_phases: the prologue launch and the contraction launch separately
+        st = lib().hgf_linear_forward_phases(_ptr(x), M, _ptr(packed), ctypes.c_float(gamma), d_in, d_out, _ptr(At),
+                                             _ptr(Bt), r, _ptr(gate), _ptr(y), _ptr(workspace), workspace.numel(),
+                                             dbg_arg, flags, phases, _stream(stream))
     _check("hgf_linear_forward", st)
     if debug:
         dbg["h"] = dbg["h"][:, :r]
@@ -227,6 +238,23 @@ class Group:
 
     def forward_phases(self, phases: int, stream=None) -> None:
         _check("hgf_group_forward_phases", lib().hgf_group_forward_phases(self._handle, phases, _stream(stream)))
+
+    def debug(self, index: int, y_int=None):
+        """hgf_group_debug: route problem `index`'s int32 accumulators to `y_int` (a device int32
+        tensor [M][d_out], or None) from the next forward on, and return views (xq int8 [M][d_in],
+        gamma_x fp32 [M]) of the group's own workspace for that problem."""
+        q = self._keep[index]
+        M, K = q["x"].shape[0], q["d_in"]
+        views = DebugOut()
+        _check("hgf_group_debug", lib().hgf_group_debug(self._handle, index, _ptr(y_int), ctypes.byref(views)))
+        c = ctypes
+
+        def view(ptr, nbytes, dtype, shape):
+            class _Mem:  # exposes the device range through the CUDA array interface
+                __cuda_array_interface__ = {"shape": (nbytes,), "typestr": "|u1", "data": (int(ptr), False), "version": 2}
+            return torch.as_tensor(_Mem(), device=q["x"].device).view(dtype).view(shape)
+
+        return {"xq": view(views.xq, M * K, torch.int8, (M, K)), "gamma_x": view(views.gamma_x, M * 4, torch.float32, (M,))}
 
     def close(self) -> None:
         if self._handle:

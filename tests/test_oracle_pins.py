@@ -281,24 +281,33 @@ def test_no_silu_flag_is_plain_gated_lora():
     assert np.abs(with_silu["y"] - out["y"]).max() > 1e-3
 
 
-def test_float_fake_quant_restatement_agrees():
-    # The float formulation: dequantise x~ and the ternary weights first, then one float matmul,
-    # plus gate * (silu(x A) B).  Must agree with the integer path to float64 rounding.
+def test_dequantise_first_float_formulation_agrees():
+    # Definitions "Absmax Quantization" and "Dynamic Activation Quantization" read as real-valued
+    # maps: each token is replaced by its dequantised code vector  codes * gamma_x / 127  (codes from
+    # the true quotient 127 x / gamma_x, rounded to nearest), each weight by  t * gamma_W  (t from the
+    # +-gamma_W / 2 thresholds of the true quotient W / gamma_W).  One real matrix product of those two
+    # plus the gated correction of Definitions "Low-Rank Correction" / "Gated Fusion" must equal
+    # Algorithm 1's integer route (integer product first, scales applied afterwards) to float64 rounding.
     L, T, g = _layer(M=6, K=256, N=72, r=16, seed=13)
     out = oracle.forward(L["x"], T, g, L["At"], L["Bt"], L["gate"])
-    xd = syn.bf16_bits_to_f32(L["x"]).astype(np.float64)
-    gx = np.maximum(np.abs(xd).max(axis=1, keepdims=True), 1e-5)
-    scale_x = 127.0 / gx
-    x_fake = np.clip(np.rint(xd * scale_x), -127, 127) / scale_x
-    Wd = L["W"].astype(np.float64)
-    scale_w = 1.0 / np.mean(np.abs(Wd))
-    w_fake = np.clip(np.rint(Wd * scale_w), -1, 1) / scale_w
-    A = syn.fp16_bits_to_f32(L["At"]).astype(np.float64).T
-    B = syn.fp16_bits_to_f32(L["Bt"]).astype(np.float64).T
-    z = xd @ A
-    ref = x_fake @ w_fake.T + L["gate"].astype(np.float64)[None, :] * ((z / (1 + np.exp(-z))) @ B)
-    # the oracle's gamma is the fp32-rounded mean: allow that 6e-8 relative difference
-    np.testing.assert_allclose(out["y"], ref, rtol=2e-7, atol=2e-7 * np.abs(ref).max())
+    tokens = syn.bf16_bits_to_f32(L["x"]).astype(np.float64)
+    token_scale = np.maximum(np.abs(tokens).max(axis=1), 1e-5)
+    codes = np.clip(np.rint(127.0 * tokens / token_scale[:, None]), -127, 127)
+    tokens_deq = codes * token_scale[:, None] / 127.0
+    weights = L["W"].astype(np.float64)
+    weight_scale = np.abs(weights).mean()
+    quotient = weights / weight_scale
+    trits = np.where(quotient > 0.5, 1.0, np.where(quotient < -0.5, -1.0, 0.0))
+    backbone = tokens_deq @ (trits * weight_scale).T
+    down = syn.fp16_bits_to_f32(L["At"]).astype(np.float64)     # [r][K]
+    up = syn.fp16_bits_to_f32(L["Bt"]).astype(np.float64)       # [N][r]
+    pre = tokens @ down.T
+    hidden = pre * (1.0 / (1.0 + np.exp(-pre)))
+    expected = backbone + (hidden @ up.T) * L["gate"].astype(np.float64)[None, :]
+    # the oracle's gamma_W is the fp32-rounded mean: allow that 6e-8 relative difference
+    np.testing.assert_allclose(out["y"], expected, rtol=2e-7, atol=2e-7 * np.abs(expected).max())
+    # the float64 trits are the oracle's codes (no weight of this layer sits within 1e-7 of a threshold)
+    assert np.array_equal(trits.astype(np.int8), T)
 
 
 def test_transposed_operand_would_be_caught():

@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2602_05269_b200 import inputs as syn
 
 pytestmark = pytest.mark.gpu
@@ -37,7 +38,7 @@ def _dev(a, dtype=None):
 def _layer(hgf, shape, M, layer):
     L = syn.make_layer(shape, M, config=14, layer=layer)
     packed, gamma = hgf.pack_ternary(_dev(L["W"]))
-    return {"x": _dev(L["x"], torch.bfloat16), "packed": packed, "gamma": gamma,
+    return {"host": L, "x": _dev(L["x"], torch.bfloat16), "packed": packed, "gamma": gamma,
             "At": _dev(L["At"], torch.float16), "Bt": _dev(L["Bt"], torch.float16), "gate": _dev(L["gate"]),
             "shape": shape, "M": M}
 
@@ -52,6 +53,19 @@ def _both(hgf, q, flags=0):
     scale = want.float().abs().max().item()
     err = (got.float() - want.float()).abs().max().item() / scale
     assert err <= TOL_DECODE, f"{s.d_in}->{s.d_out} M={q['M']}: normalised difference {err:.3e}"
+    return got
+
+
+def test_static_scratch_call_matches_the_oracle(hgf):
+    """The same comparison the parity tests make for the ordinary call: the output of the call that
+    uses the built-in scratch against the CPU oracle's, on the same seeded inputs."""
+    for q in (_layer(hgf, syn.LayerShape("c", 1024, 264, 32), 3, 2), _layer(hgf, syn.LayerShape("d", 2048, 512, 64), 16, 3)):
+        got = _both(hgf, q)
+        L, s = q["host"], q["shape"]
+        T = oracle.ternarise(L["W"], np.float32(q["gamma"]))
+        ref = oracle.forward(L["x"], T, np.float32(q["gamma"]), L["At"], L["Bt"], L["gate"])
+        err = np.abs(got.cpu().numpy().astype(np.float64) - ref["y"]).max() / np.abs(ref["y"]).max()
+        assert err <= TOL_DECODE, f"{s.d_in}->{s.d_out}: normalised error against the oracle {err:.3e}"
 
 
 def test_static_scratch_call_matches_the_workspace_call_twice_in_a_row(hgf):
@@ -70,6 +84,17 @@ def test_static_scratch_call_refuses_what_does_not_fit(hgf):
     with pytest.raises(hgf.HgfError) as e:         # 8 x 65536 quantised activations alone exceed the array
         hgf.linear_forward_static(x, packed, 1.0, 65536, 64, y)
     assert e.value.status == 7
+    # one token, but rank 64 on a 32768-wide input: the partial sums of x A alone are 512 KiB
+    x1 = torch.zeros((1, 32768), dtype=torch.bfloat16, device="cuda")
+    At = torch.zeros((64, 32768), dtype=torch.float16, device="cuda")
+    Bt = torch.zeros((64, 64), dtype=torch.float16, device="cuda")
+    gate = torch.zeros(64, dtype=torch.float32, device="cuda")
+    with pytest.raises(hgf.HgfError) as e:
+        hgf.linear_forward_static(x1, packed, 1.0, 32768, 64, torch.empty((1, 64), device="cuda"), At, Bt, gate)
+    assert e.value.status == 7
+    with pytest.raises(hgf.HgfError) as e:         # a rank the layer does not support is reported as such
+        hgf.linear_forward_static(x1, packed, 1.0, 32768, 64, torch.empty((1, 64), device="cuda"), At[:24], Bt, gate)
+    assert e.value.status == 2
     x17 = torch.zeros((17, 256), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(hgf.HgfError) as e:         # more tokens than the decode path takes
         hgf.linear_forward_static(x17, packed, 1.0, 256, 64, torch.empty((17, 64), device="cuda"))
