@@ -8,8 +8,11 @@ from .hgf_oracle import (  # noqa: F401
     build,
     effective_bits,
     forward,
+    forward_ln,
     gamma_w,
     int_gemm,
+    ln_quant,
+    ln_stats,
     pack,
     packed_bytes,
     ternarise,

@@ -16,7 +16,11 @@
  * +-gamma/2 ties; pack/unpack round trips; int8 invariants, crafted rounding ties; brute-force
  * integer matmul on tiny shapes and numpy int64 matmul; gate = 0 reduces to the pure ternary
  * layer; hand-worked 2x2 correction; SiLU-off equals (x A) B; the fake-quant float restatement;
- * the paper's T_max worked example (7B, FP16, 500 GB/s -> 35.7 tokens/s).
+ * the paper's T_max worked example (7B, FP16, 500 GB/s -> 35.7 tokens/s); for the LayerNorm
+ * front end: numpy float64 statistics, a constant row, rows that are already normalised (the
+ * front end then reduces to the plain quantiser), sign and power-of-two invariances, the listing's
+ * rounding of the tie 76/152 (-> 63), the library layer_norm routine, and the equivalence of a
+ * grouped gate with its expanded per-channel vector.
  * No function here is "parity unpinned".
  */
 #include <math.h>
@@ -228,6 +232,113 @@ int oracle_forward(const uint16_t *x_bf16, int64_t M, const int8_t *T, float gam
                 for (int32_t j = 0; j < r; ++j)
                     y_corr += H[m * r + j] * fp16_to_double(Bt_fp16[n * r + j]);
                 y_corr *= (double)gate[n];
+            }
+            y[m * d_out + n] = y_tern + y_corr;
+        }
+    return overflow;
+}
+
+/* ---- Appendix E, ScientificBitLinear.forward: the LayerNorm in front of the quantiser -------- */
+/* The listing normalises each token before it is quantised (LayerNorm over d_in with a learned
+ * weight and bias, biased variance, eps inside the square root), while the correction path of
+ * AdaptiveDualPathLinear.forward reads the raw x.
+ *
+ * Statistics of each token, in double: mean = sum x / d_in, var = sum (x - mean)^2 / d_in,
+ * rstd = 1 / sqrt(var + eps). */
+void oracle_ln_stats(const uint16_t *x_bf16, int64_t M, int64_t d_in, double eps, double *mean, double *rstd) {
+    for (int64_t m = 0; m < M; ++m) {
+        double sum = 0.0;
+        for (int64_t k = 0; k < d_in; ++k) sum += bf16_to_double(x_bf16[m * d_in + k]);
+        double mu = sum / (double)d_in;
+        double ss = 0.0;
+        for (int64_t k = 0; k < d_in; ++k) {
+            double d = bf16_to_double(x_bf16[m * d_in + k]) - mu;
+            ss += d * d;
+        }
+        mean[m] = mu;
+        rstd[m] = 1.0 / sqrt(ss / (double)d_in + eps);
+    }
+}
+
+/* Normalisation and quantisation of the normalised token.  The listing does both in binary32
+ * (x.float(), autocast disabled), so the precision is the paper's: every operation below is one
+ * correctly rounded binary32 operation, in this order (the reading this library fixes, since the
+ * rounded value decides the int8 code):
+ *     d = x - mean;  n = d * rstd;  s = n * w[k];  xn = s + b[k];
+ *     gamma_x = max(max_k |xn|, 1e-5);  scale = 127 / gamma_x;  q = rint(xn * scale), clipped to
+ *     [-127, 127] (Algorithm 1's range; the product never reaches -127.5).
+ * mean and rstd are given as binary32 values (per token).  Compiled with -ffp-contract=off, so no
+ * operation is fused. */
+void oracle_ln_quant(const uint16_t *x_bf16, int64_t M, int64_t d_in, const float *mean, const float *rstd,
+                     const float *ln_w, const float *ln_b, float *xn_out, int8_t *xq, float *gamma_x) {
+    for (int64_t m = 0; m < M; ++m) {
+        float amax = 0.0f;
+        for (int64_t k = 0; k < d_in; ++k) {
+            float xf = (float)bf16_to_double(x_bf16[m * d_in + k]); /* exact */
+            float d = xf - mean[m];
+            float n = d * rstd[m];
+            float s = n * ln_w[k];
+            float xn = s + ln_b[k];
+            if (xn_out) xn_out[m * d_in + k] = xn;
+            float a = fabsf(xn);
+            if (a > amax) amax = a;
+        }
+        float g = amax < 1e-5f ? 1e-5f : amax;
+        gamma_x[m] = g;
+        float scale = 127.0f / g;
+        for (int64_t k = 0; k < d_in; ++k) {
+            float xf = (float)bf16_to_double(x_bf16[m * d_in + k]);
+            float d = xf - mean[m];
+            float n = d * rstd[m];
+            float s = n * ln_w[k];
+            float xn = s + ln_b[k];
+            float p = xn * scale;
+            float q = rintf(p);
+            if (q > 127.0f) q = 127.0f;
+            if (q < -127.0f) q = -127.0f;
+            xq[m * d_in + k] = (int8_t)q;
+        }
+    }
+}
+
+/* The layer with the LayerNorm front end and a grouped gate:
+ *   y[m][n] = Y_int[m][n] * gamma_x[m] * gamma_W / 127 + g[n / gate_group] * sum_j SiLU(sum_k x[m][k] A[k][j]) B[j][n]
+ * with X~, gamma_x from the NORMALISED token (above) and the correction from the RAW token.
+ * gate holds ceil(d_out / gate_group) values: gate_group = 1 is one value per channel, d_out / n_heads
+ * the listing's per-head gate (HeadAdaptiveDiffAttention), d_out the scalar gate.
+ * mean_in / rstd_in (nullable): binary32 statistics to use instead of the double ones rounded to
+ * binary32 (the tests pass the CUDA library's own, as they do for gamma_W). */
+int oracle_forward_ln(const uint16_t *x_bf16, int64_t M, const int8_t *T, float gamma_w, int64_t d_in, int64_t d_out,
+                      const float *ln_w, const float *ln_b, double eps, const float *mean_in, const float *rstd_in,
+                      const uint16_t *At_fp16, const uint16_t *Bt_fp16, int32_t r, const float *gate, int64_t gate_group,
+                      uint32_t flags, double *y, int8_t *xq, float *gamma_x, int32_t *y_int, double *H,
+                      float *mean_out, float *rstd_out, double *stat_scratch /* 2 M doubles */) {
+    int have_corr = (r > 0 && At_fp16 && Bt_fp16 && gate);
+    oracle_ln_stats(x_bf16, M, d_in, eps, stat_scratch, stat_scratch + M);
+    for (int64_t m = 0; m < M; ++m) {
+        mean_out[m] = mean_in ? mean_in[m] : (float)stat_scratch[m];
+        rstd_out[m] = rstd_in ? rstd_in[m] : (float)stat_scratch[M + m];
+    }
+    oracle_ln_quant(x_bf16, M, d_in, mean_out, rstd_out, ln_w, ln_b, NULL, xq, gamma_x);
+    int overflow = oracle_int_gemm(xq, T, M, d_out, d_in, y_int);
+    if (have_corr) {
+#pragma omp parallel for schedule(static)
+        for (int64_t m = 0; m < M; ++m)
+            for (int32_t j = 0; j < r; ++j) {
+                double z = 0.0;
+                for (int64_t k = 0; k < d_in; ++k)
+                    z += bf16_to_double(x_bf16[m * d_in + k]) * fp16_to_double(At_fp16[(int64_t)j * d_in + k]);
+                H[m * r + j] = (flags & ORACLE_FLAG_NO_SILU) ? z : silu(z);
+            }
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < d_out; ++n)
+        for (int64_t m = 0; m < M; ++m) {
+            double y_tern = (double)y_int[m * d_out + n] * ((double)gamma_x[m] * (double)gamma_w / 127.0);
+            double y_corr = 0.0;
+            if (have_corr) {
+                for (int32_t j = 0; j < r; ++j) y_corr += H[m * r + j] * fp16_to_double(Bt_fp16[n * r + j]);
+                y_corr *= (double)gate[n / gate_group];
             }
             y[m * d_out + n] = y_tern + y_corr;
         }

@@ -58,6 +58,13 @@ def _load():
         lib.oracle_forward.restype = c.c_int
         lib.oracle_forward.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, u32, vp,
                                        vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_ln_stats.restype = None
+        lib.oracle_ln_stats.argtypes = [vp, i64, i64, c.c_double, vp, vp]
+        lib.oracle_ln_quant.restype = None
+        lib.oracle_ln_quant.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_forward_ln.restype = c.c_int
+        lib.oracle_forward_ln.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, c.c_double, vp, vp, vp, vp, i32, vp,
+                                          i64, u32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_tmax.restype = c.c_double
         lib.oracle_tmax.argtypes = [c.c_double] * 3
         lib.oracle_effective_bits.restype = c.c_double
@@ -159,6 +166,68 @@ def forward(x_bf16_bits, T, gamma, At_fp16_bits=None, Bt_fp16_bits=None, gate=No
     if ovf:
         raise OverflowError("integer accumulator left the int32 range")
     return {"y": y, "xq": xq, "gamma_x": gx, "y_int": yi, "h": h[:, :r]}
+
+
+def ln_stats(x_bf16_bits, eps: float = 1e-5):
+    """Per-token LayerNorm statistics in float64: (mean [M], rstd [M])."""
+    x = _arr(x_bf16_bits, np.uint16)
+    M, K = x.shape
+    mean = np.empty(M, np.float64)
+    rstd = np.empty(M, np.float64)
+    _load().oracle_ln_stats(_p(x), M, K, float(eps), _p(mean), _p(rstd))
+    return mean, rstd
+
+
+def ln_quant(x_bf16_bits, mean_f32, rstd_f32, ln_w, ln_b):
+    """Normalise (binary32, fixed operation order) and quantise.  Returns (xn fp32, xq int8, gamma_x fp32)."""
+    x = _arr(x_bf16_bits, np.uint16)
+    M, K = x.shape
+    mean = _arr(mean_f32, np.float32, (M,))
+    rstd = _arr(rstd_f32, np.float32, (M,))
+    w = _arr(ln_w, np.float32, (K,))
+    b = _arr(ln_b, np.float32, (K,))
+    xn = np.empty((M, K), np.float32)
+    xq = np.empty((M, K), np.int8)
+    gx = np.empty(M, np.float32)
+    _load().oracle_ln_quant(_p(x), M, K, _p(mean), _p(rstd), _p(w), _p(b), _p(xn), _p(xq), _p(gx))
+    return xn, xq, gx
+
+
+def forward_ln(x_bf16_bits, T, gamma, ln_w, ln_b, eps=1e-5, At_fp16_bits=None, Bt_fp16_bits=None, gate=None,
+               gate_group: int = 1, flags: int = 0, mean=None, rstd=None):
+    """The layer with the LayerNorm front end and a grouped gate.  Returns a dict: y (float64), xq,
+    gamma_x, y_int, h, mean, rstd (the binary32 statistics used)."""
+    x = _arr(x_bf16_bits, np.uint16)
+    T = _arr(T, np.int8)
+    M, K = x.shape
+    N = T.shape[0]
+    assert T.shape[1] == K and gate_group >= 1
+    w = _arr(ln_w, np.float32, (K,))
+    b = _arr(ln_b, np.float32, (K,))
+    r = 0
+    At = Bt = g = None
+    if At_fp16_bits is not None and Bt_fp16_bits is not None and gate is not None:
+        At = _arr(At_fp16_bits, np.uint16)
+        r = At.shape[0]
+        At = _arr(At, np.uint16, (r, K))
+        Bt = _arr(Bt_fp16_bits, np.uint16, (N, r))
+        g = _arr(gate, np.float32, ((N + gate_group - 1) // gate_group,))
+    mean_in = None if mean is None else _arr(mean, np.float32, (M,))
+    rstd_in = None if rstd is None else _arr(rstd, np.float32, (M,))
+    y = np.empty((M, N), np.float64)
+    xq = np.empty((M, K), np.int8)
+    gx = np.empty(M, np.float32)
+    yi = np.empty((M, N), np.int32)
+    h = np.zeros((M, max(r, 1)), np.float64)
+    mo = np.empty(M, np.float32)
+    ro = np.empty(M, np.float32)
+    scratch = np.empty(2 * M, np.float64)
+    ovf = _load().oracle_forward_ln(_p(x), M, _p(T), float(np.float32(gamma)), K, N, _p(w), _p(b), float(eps),
+                                    _p(mean_in), _p(rstd_in), _p(At), _p(Bt), r, _p(g), gate_group, flags,
+                                    _p(y), _p(xq), _p(gx), _p(yi), _p(h), _p(mo), _p(ro), _p(scratch))
+    if ovf:
+        raise OverflowError("integer accumulator left the int32 range")
+    return {"y": y, "xq": xq, "gamma_x": gx, "y_int": yi, "h": h[:, :r], "mean": mo, "rstd": ro}
 
 
 def tmax(bmem_bytes_per_s: float, params: float, bits: float) -> float:
