@@ -149,6 +149,40 @@ hgf_status hgf_linear_forward_phases(const void *x, int64_t M, const void *packe
                                      uint32_t phases, void *stream);
 
 /*
+ * The layer with the front end and the gate granularity of the paper's reference module
+ * (Appendix E): ScientificBitLinear.forward normalises each token with a LayerNorm over d_in before
+ * it quantises it, AdaptiveDualPathLinear.forward feeds the RAW token to the correction path, and
+ * HeadAdaptiveDiffAttention gates per attention head.
+ *
+ *     xn[m][k]   = ((x[m][k] - mean[m]) * rstd[m]) * ln_weight[k] + ln_bias[k]
+ *                  mean, rstd = 1 / sqrt(var + eps) of token m (biased variance); every operation one
+ *                  binary32 operation, in this order (the rounded value decides the int8 code)
+ *     gamma_x[m] = max(max_k |xn[m][k]|, 1e-5);  xq = Clip(Round(xn * (127 / gamma_x)), -127, 127),
+ *                  binary32 as in the listing (a product, not a quotient)
+ *     y          = Y_int * gamma_x * gamma_W / 127 + gate[n / gate_group] * (SiLU(x A) B)[m][n]
+ *
+ * ln_weight, ln_bias: device fp32 [d_in]; both null = no LayerNorm (the call then is
+ * hgf_linear_forward with a grouped gate).  gate holds ceil(d_out / gate_group) values: gate_group
+ * 0 or 1 = one per channel, d_out / n_heads = one per head, >= d_out = the paper's scalar gate;
+ * it must be 1, a multiple of 16, or >= d_out.  mean_out / rstd_out: nullable device fp32 [M], receive
+ * the statistics the kernels used (for parity checks).  Everything else as hgf_linear_forward, same
+ * workspace size.  With a LayerNorm the GEMM path takes one more launch (normalise + quantise).
+ */
+typedef struct {
+    const float *ln_weight;
+    const float *ln_bias;
+    float eps;
+    int64_t gate_group;
+    float *mean_out;
+    float *rstd_out;
+} hgf_front_end;
+hgf_status hgf_linear_forward_ln(const void *x, int64_t M, const void *packed, float gamma,
+                                 int64_t d_in, int64_t d_out, const void *At, const void *Bt,
+                                 int32_t r, const float *gate, void *y, void *workspace,
+                                 size_t workspace_bytes, const hgf_debug_out *dbg,
+                                 const hgf_front_end *front_end, uint32_t flags, void *stream);
+
+/*
  * hgf_linear_forward for callers that cannot hand over a workspace.  (The paper has no counterpart:
  * this is a convenience of the library, not a step of the method.)
  *

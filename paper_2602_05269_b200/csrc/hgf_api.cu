@@ -150,8 +150,14 @@ static void fill_params(const void *x, int64_t M, const void *packed, float gamm
         dp->flags = flags;
         dp->tile_begin = 0;
         dp->cost_begin = 0;
+        dp->gate_group = 1;
     }
 }
+
+static hgf_status forward_impl(const void *x, int64_t M, const void *packed, float gamma, int64_t d_in, int64_t d_out,
+                               const void *At, const void *Bt, int32_t r, const float *gate, void *y, void *workspace,
+                               size_t workspace_bytes, const hgf_debug_out *dbg, const hgf_front_end *fe_in, uint32_t flags,
+                               uint32_t phases, void *stream_);
 
 }  // namespace hgf
 
@@ -167,6 +173,23 @@ extern "C" hgf_status hgf_linear_forward_phases(const void *x, int64_t M, const 
                                                 int64_t d_out, const void *At, const void *Bt, int32_t r,
                                                 const float *gate, void *y, void *workspace, size_t workspace_bytes,
                                                 const hgf_debug_out *dbg, uint32_t flags, uint32_t phases, void *stream_) {
+    return forward_impl(x, M, packed, gamma, d_in, d_out, At, Bt, r, gate, y, workspace, workspace_bytes, dbg, nullptr, flags,
+                        phases, stream_);
+}
+
+extern "C" hgf_status hgf_linear_forward_ln(const void *x, int64_t M, const void *packed, float gamma, int64_t d_in,
+                                            int64_t d_out, const void *At, const void *Bt, int32_t r, const float *gate,
+                                            void *y, void *workspace, size_t workspace_bytes, const hgf_debug_out *dbg,
+                                            const hgf_front_end *front_end, uint32_t flags, void *stream_) {
+    if (!front_end) return HGF_ERR_INVALID_ARG;
+    return forward_impl(x, M, packed, gamma, d_in, d_out, At, Bt, r, gate, y, workspace, workspace_bytes, dbg, front_end, flags,
+                        HGF_PHASE_PROLOGUE | HGF_PHASE_GEMV, stream_);
+}
+
+hgf_status hgf::forward_impl(const void *x, int64_t M, const void *packed, float gamma, int64_t d_in, int64_t d_out,
+                                    const void *At, const void *Bt, int32_t r, const float *gate, void *y, void *workspace,
+                                    size_t workspace_bytes, const hgf_debug_out *dbg, const hgf_front_end *fe_in, uint32_t flags,
+                                    uint32_t phases, void *stream_) {
     if (!phases || (phases & ~(HGF_PHASE_PROLOGUE | HGF_PHASE_GEMV))) return HGF_ERR_INVALID_ARG;
     const bool do_prologue = (phases & HGF_PHASE_PROLOGUE) != 0, do_main = (phases & HGF_PHASE_GEMV) != 0;
     bool gemm = false;
@@ -180,12 +203,35 @@ extern "C" hgf_status hgf_linear_forward_phases(const void *x, int64_t M, const 
     cudaStream_t stream = (cudaStream_t)stream_;
     const bool pdl = !(flags & HGF_FLAG_NO_PDL);
 
+    // front end (Appendix E): LayerNorm before the quantiser, grouped gate
+    bool ln = false;
+    int gate_group = 1;
+    FrontEnd fe = {};
+    if (fe_in) {
+        if ((fe_in->ln_weight == nullptr) != (fe_in->ln_bias == nullptr) || !(fe_in->eps >= 0.0f)) return HGF_ERR_INVALID_ARG;
+        if (misaligned(fe_in->ln_weight) || misaligned(fe_in->ln_bias)) return HGF_ERR_MISALIGNED;
+        if (fe_in->gate_group < 0) return HGF_ERR_INVALID_ARG;
+        if (fe_in->gate_group > 1) {
+            if (fe_in->gate_group >= d_out) gate_group = (int)((d_out + 15) / 16 * 16);  // scalar gate: one group holds every row tile
+            else if (fe_in->gate_group % 16 == 0) gate_group = (int)fe_in->gate_group;
+            else return HGF_ERR_UNSUPPORTED_SHAPE;
+        }
+        ln = fe_in->ln_weight != nullptr;
+        fe.ln_w = fe_in->ln_weight;
+        fe.ln_b = fe_in->ln_bias;
+        fe.dbg_mean = fe_in->mean_out;
+        fe.dbg_rstd = fe_in->rstd_out;
+        fe.eps = fe_in->eps;
+    }
+
     PrologueParams pp;
     DecodeProblem dp;
     fill_params(x, M, packed, gamma, d_in, d_out, At, Bt, r, gate, y, (char *)workspace, L, gemm, dbg, flags, &pp, &dp);
+    dp.gate_group = gate_group;
 
     if (!gemm) {
-        if (do_prologue && launch_decode_prologue(pp, pdl, stream) != cudaSuccess) return HGF_ERR_CUDA;
+        if (do_prologue && (ln ? launch_decode_prologue_ln(pp, fe, pdl, stream) : launch_decode_prologue(pp, pdl, stream)) != cudaSuccess)
+            return HGF_ERR_CUDA;
         if (!do_main) return HGF_OK;
         DecodeLaunch dl = {};
         dl.probs = nullptr;
@@ -204,8 +250,19 @@ extern "C" hgf_status hgf_linear_forward_phases(const void *x, int64_t M, const 
     gx.gate = gate;
     gx.gw_over_127 = dp.gw_over_127;
     gx.N = (int)d_out;
-    if (do_prologue && (r ? launch_gemm_prologue(pp, gx, stream) : launch_quant(pp, gx, stream)) != cudaSuccess)
+    gx.gate_group = gate_group;
+    if (do_prologue && ln) {
+        // the correction path's part of the prologue on the raw tokens (its own quantisation switched off),
+        // then one launch that normalises and quantises
+        if (r) {
+            PrologueParams lora_only = pp;
+            lora_only.xq = nullptr;
+            if (launch_gemm_prologue(lora_only, gx, stream) != cudaSuccess) return HGF_ERR_CUDA;
+        }
+        if (launch_ln_quant(pp, gx, fe, stream) != cudaSuccess) return HGF_ERR_CUDA;
+    } else if (do_prologue && (r ? launch_gemm_prologue(pp, gx, stream) : launch_quant(pp, gx, stream)) != cudaSuccess) {
         return HGF_ERR_CUDA;
+    }
     if (!do_main) return HGF_OK;
     GemmParams gp = {};
     gp.xq = pp.xq;

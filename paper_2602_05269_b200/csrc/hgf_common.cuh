@@ -117,6 +117,16 @@ struct GemmPrologueExtra {
     float gw_over_127;
     int N;
     int tokens_per_block;    // set by the launcher of the GEMM path's prologue kernel
+    int gate_group;          // channels per gate value (1 = one per channel)
+};
+
+// LayerNorm front end (Appendix E of the paper): parameters and where the statistics go.
+struct FrontEnd {
+    const float *ln_w;       // [K]
+    const float *ln_b;       // [K]
+    float *dbg_mean;         // [M], nullable
+    float *dbg_rstd;         // [M], nullable
+    float eps;
 };
 
 // Cost of one 16-row tile of a decode problem, the unit in which a launch is cut into equal shares:
@@ -146,6 +156,7 @@ struct DecodeProblem {
     uint32_t flags;
     int tile_begin;
     long long cost_begin;
+    int gate_group;          // channels per gate value: 1, or a multiple of 16 (a row tile then has one gate)
 };
 
 struct DecodeLaunch {
@@ -162,6 +173,11 @@ struct DecodeLaunch {
 // host-side launchers (each enqueues on `stream` and returns the CUDA error of the launch)
 cudaError_t launch_quant(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream);
 cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream_t stream);
+// The same with the LayerNorm front end: the row blocks normalise before they quantise.
+cudaError_t launch_decode_prologue_ln(const PrologueParams &p, const FrontEnd &fe, bool pdl, cudaStream_t stream);
+// GEMM path with the front end: normalise + quantise every token (one block per row); the LoRA part
+// runs in launch_gemm_prologue with p.xq == nullptr (its quantisation switched off).
+cudaError_t launch_ln_quant(const PrologueParams &p, const GemmPrologueExtra &x, const FrontEnd &fe, cudaStream_t stream);
 // Group prologue.  A quantisation item is one token row.  A LoRA item is 16 columns of H (rows
 // 16 jt .. 16 jt + 15 of A^T) over one K slice of a problem; its 16 x 16 partial sums of x A go to
 // `hpart` as [8 accumulator registers][32 lanes] floats, and the GEMV adds the slices of a tile in

@@ -48,7 +48,7 @@ struct SegSmall {                    // per-problem values the epilogue needs
     int32_t *dbg_y_int;
     const float *gate;
     uint32_t flags;
-    int pad;
+    int gate_group;
 };
 constexpr int kOffRed = kOffSmall + 2 * (int)sizeof(SegSmall);
 constexpr int kRedBytes = kDecWarps * 8 * 32 * 4;  // per warp: up to 8 accumulator registers per lane
@@ -353,7 +353,7 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
                 sm.scale[tid] = tid < M ? Pg.gamma_x[tid] * Pg.gw_over_127 : 0.0f;
                 sm.row_sum[tid] = tid < M ? Pg.row_sum[tid] : 0;
             }
-            if (tid == 32) { sm.y = Pg.y; sm.dbg_y_int = Pg.dbg_y_int; sm.gate = Pg.gate; sm.flags = Pg.flags; }
+            if (tid == 32) { sm.y = Pg.y; sm.dbg_y_int = Pg.dbg_y_int; sm.gate = Pg.gate; sm.flags = Pg.flags; sm.gate_group = Pg.gate_group; }
             if (Pg.nslices > 0) {
                 // group launch: H = act(sum over K slices of the parked partial sums of x A), slices in
                 // order.  The partial sums sit in the tf32 MMA's accumulator layout: column j = 16 jt + jl
@@ -426,8 +426,12 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
             float gA = 0.0f, gB = 0.0f;
             if (r > 0) {
                 const float *gate = sm.gate;
-                gA = __ldg(gate + (n0 + g < N ? n0 + g : N - 1));
-                gB = __ldg(gate + (n0 + g + 8 < N ? n0 + g + 8 : N - 1));
+                if (sm.gate_group > 1) {  // grouped gate (per head, or scalar): groups are whole row tiles
+                    gA = gB = __ldg(gate + n0 / sm.gate_group);
+                } else {
+                    gA = __ldg(gate + (n0 + g < N ? n0 + g : N - 1));
+                    gB = __ldg(gate + (n0 + g + 8 < N ? n0 + g + 8 : N - 1));
+                }
                 if (!wait_slot()) return false;
                 const int rows = N - n0 < 16 ? N - n0 : 16;
                 const uint32_t *bA = reinterpret_cast<const uint32_t *>(ring + cslot * kSlotBytes) + (g < rows ? g : rows - 1) * (r >> 1) + t;

@@ -147,6 +147,117 @@ __device__ __forceinline__ void quant_row(const PrologueParams &p, int m, float 
     }
 }
 
+// ---- LayerNorm front end (Appendix E, ScientificBitLinear.forward) -----------------------------------
+// One binary32 operation each, in this order: the rounded value decides the int8 code.
+__device__ __forceinline__ float ln_value(float x, float mean, float rstd, float w, float b) {
+    return __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(x, mean), rstd), w), b);
+}
+__device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f[e] = (e & 1) ? bf16hi_to_float(w[e >> 1]) : bf16lo_to_float(w[e >> 1]);
+}
+__device__ __forceinline__ double block_sum_d(double v, double *s_red, int lane, int warp) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();  // the previous use of s_red is over
+    if (lane == 0) s_red[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) t += s_red[w];
+    return t;
+}
+// One block normalises and quantises one token row: mean and variance (two passes, summed in double),
+// the row's largest |xn|, then the codes - the listing's binary32 arithmetic: scale = 127 / gamma_x,
+// code = rint(xn * scale).  The row is read from L1/L2 in every pass.
+__device__ __forceinline__ void quant_row_ln(const PrologueParams &p, const FrontEnd &fe, int m, float *tok_sc, float gw_over_127) {
+    __shared__ double s_red_d[kWarps];
+    __shared__ float s_red_f[kWarps];
+    __shared__ int s_red_i[kWarps];
+    const int K = p.K, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint4 *xv = reinterpret_cast<const uint4 *>(p.x + (size_t)m * K);
+    const int nv = K / 8;
+    float f[8];
+
+    double sum = 0.0;
+    for (int i = tid; i < nv; i += kThreads) {
+        unpack8(xv[i], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sum += (double)f[e];
+    }
+    const double mean_d = block_sum_d(sum, s_red_d, lane, warp) / (double)K;
+    double ss = 0.0;
+    for (int i = tid; i < nv; i += kThreads) {
+        unpack8(xv[i], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const double d = (double)f[e] - mean_d;
+            ss += d * d;
+        }
+    }
+    const double var = block_sum_d(ss, s_red_d, lane, warp) / (double)K;
+    const float mean = (float)mean_d, rstd = (float)(1.0 / sqrt(var + (double)fe.eps));
+
+    float amax = 0.0f;
+    for (int i = tid; i < nv; i += kThreads) {
+        unpack8(xv[i], f);
+        const float4 w0 = *reinterpret_cast<const float4 *>(fe.ln_w + 8 * i), w1 = *reinterpret_cast<const float4 *>(fe.ln_w + 8 * i + 4);
+        const float4 b0 = *reinterpret_cast<const float4 *>(fe.ln_b + 8 * i), b1 = *reinterpret_cast<const float4 *>(fe.ln_b + 8 * i + 4);
+        const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w}, b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(ln_value(f[e], mean, rstd, w[e], b[e])));
+    }
+    amax = warp_max(amax);
+    if (lane == 0) s_red_f[warp] = amax;
+    __syncthreads();
+    float g = s_red_f[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) g = fmaxf(g, s_red_f[w]);
+    g = fmaxf(g, 1e-5f);
+    const float scale = __fdiv_rn(127.0f, g);
+
+    int sum_q = 0;
+    uint2 *qv = reinterpret_cast<uint2 *>(p.xq + (size_t)m * K);
+    uint2 *dq = p.dbg_xq ? reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * K) : nullptr;
+    for (int i = tid; i < nv; i += kThreads) {
+        unpack8(xv[i], f);
+        const float4 w0 = *reinterpret_cast<const float4 *>(fe.ln_w + 8 * i), w1 = *reinterpret_cast<const float4 *>(fe.ln_w + 8 * i + 4);
+        const float4 b0 = *reinterpret_cast<const float4 *>(fe.ln_b + 8 * i), b1 = *reinterpret_cast<const float4 *>(fe.ln_b + 8 * i + 4);
+        const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w}, b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+        uint32_t c[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            float q = rintf(__fmul_rn(ln_value(f[e], mean, rstd, w[e], b[e]), scale));
+            q = fminf(fmaxf(q, -127.0f), 127.0f);
+            c[e] = (uint32_t)__float2int_rn(q);
+        }
+        uint32_t o[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t p01 = __byte_perm(c[4 * h], c[4 * h + 1], 0x0040), p23 = __byte_perm(c[4 * h + 2], c[4 * h + 3], 0x0040);
+            o[h] = __byte_perm(p01, p23, 0x5410);
+            sum_q = __dp4a((int)o[h], 0x01010101, sum_q);
+        }
+        qv[i] = make_uint2(o[0], o[1]);
+        if (dq) dq[i] = make_uint2(o[0], o[1]);
+    }
+    sum_q = warp_sum_i(sum_q);
+    if (lane == 0) s_red_i[warp] = sum_q;
+    __syncthreads();
+    if (tid == 0) {
+        int tot = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) tot += s_red_i[w];
+        if (p.row_sum) p.row_sum[m] = tot;
+        if (tok_sc) tok_sc[m] = g * gw_over_127;
+        p.gamma_x[m] = g;
+        if (p.dbg_gamma_x) p.dbg_gamma_x[m] = g;
+        if (fe.dbg_mean) fe.dbg_mean[m] = mean;
+        if (fe.dbg_rstd) fe.dbg_rstd[m] = rstd;
+    }
+}
+
 __device__ __forceinline__ void mma_tf32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
                                          uint32_t a3, uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -320,6 +431,28 @@ __global__ void __launch_bounds__(kThreads) decode_prologue_kernel(const Prologu
     } else {
         lora_down_block(p, blockIdx.x - p.M, 0, p.K / 32, nullptr);
     }
+}
+
+// The same with the LayerNorm front end: the row blocks normalise before they quantise; the
+// correction path's blocks read the raw x as before.
+__global__ void __launch_bounds__(kThreads) decode_prologue_ln_kernel(const PrologueParams p, const FrontEnd fe) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if ((int)blockIdx.x < p.M)
+        quant_row_ln(p, fe, blockIdx.x, nullptr, 0.0f);
+    else if (p.hpart) {
+        const int lb = blockIdx.x - p.M, jts = p.r / 16, sl = lb / jts, jt = lb - sl * jts;
+        const int per = prologue_slice_k(p.M) / 32, cbeg = sl * per, cend = cbeg + per < p.K / 32 ? cbeg + per : p.K / 32;
+        lora_down_block(p, jt, cbeg, cend, p.hpart + ((size_t)jt * p.nslices + sl) * 256);
+    } else {
+        lora_down_block(p, blockIdx.x - p.M, 0, p.K / 32, nullptr);
+    }
+}
+
+// GEMM path with the front end: one block per token row.
+__global__ void __launch_bounds__(kThreads) ln_quant_kernel(const PrologueParams p, const GemmPrologueExtra x, const FrontEnd fe) {
+    pdl_wait();
+    quant_row_ln(p, fe, blockIdx.x, x.tok_sc, x.gw_over_127);
 }
 
 // ---- group prologue: persistent CTAs, one warp per work item ------------------------------------
@@ -516,7 +649,7 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
                 uint4 v = make_uint4(0u, 0u, 0u, 0u);
                 if (c * 8 < r) {
                     v = *reinterpret_cast<const uint4 *>(x.Bt + (size_t)n * r + c * 8);
-                    const float g = x.gate[n];
+                    const float g = x.gate[x.gate_group > 1 ? n / x.gate_group : n];
                     __half2 *h2 = reinterpret_cast<__half2 *>(&v);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
@@ -672,6 +805,8 @@ __global__ void __launch_bounds__(kFpThreads) gemm_prologue_kernel(const Prologu
     // blocks still working there.)
     pdl_launch_dependents();
 
+    if (!p.xq) return;  // the LayerNorm front end quantises in a kernel of its own
+
     // second pass: the warps round the block's rows, warp w rows w, w + 8, ...
     const int nv = K / 8;
 #pragma unroll 1
@@ -792,6 +927,22 @@ cudaError_t launch_decode_prologue(const PrologueParams &p, bool pdl, cudaStream
     cudaLaunchAttribute attr[1];
     cudaLaunchConfig_t cfg = prologue_cfg(p.M + (p.r / 16) * (p.hpart ? p.nslices : 1), pdl, stream, attr);
     cudaError_t e = cudaLaunchKernelEx(&cfg, decode_prologue_kernel, p);
+    count_launch();
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_decode_prologue_ln(const PrologueParams &p, const FrontEnd &fe, bool pdl, cudaStream_t stream) {
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = prologue_cfg(p.M + (p.r / 16) * (p.hpart ? p.nslices : 1), pdl, stream, attr);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_prologue_ln_kernel, p, fe);
+    count_launch();
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_ln_quant(const PrologueParams &p, const GemmPrologueExtra &x, const FrontEnd &fe, cudaStream_t stream) {
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = prologue_cfg(p.M, !(p.flags & HGF_FLAG_NO_PDL), stream, attr);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, ln_quant_kernel, p, x, fe);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -27,7 +27,7 @@ EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_wo
            "hgf_linear_forward", "hgf_act_quant", "hgf_check_status", "hgf_tmax_tokens_per_s",
            "hgf_launch_count", "hgf_status_string", "hgf_group_create", "hgf_group_forward",
            "hgf_group_destroy", "hgf_group_forward_phases", "hgf_linear_forward_static", "hgf_group_debug",
-           "hgf_linear_forward_phases"]
+           "hgf_linear_forward_phases", "hgf_linear_forward_ln"]
 
 
 class HgfError(RuntimeError):
@@ -46,6 +46,11 @@ class Problem(ctypes.Structure):
 class DebugOut(ctypes.Structure):
     _fields_ = [("xq", ctypes.c_void_p), ("gamma_x", ctypes.c_void_p), ("y_int", ctypes.c_void_p),
                 ("h", ctypes.c_void_p)]
+
+
+class FrontEnd(ctypes.Structure):
+    _fields_ = [("ln_weight", ctypes.c_void_p), ("ln_bias", ctypes.c_void_p), ("eps", ctypes.c_float),
+                ("gate_group", ctypes.c_int64), ("mean_out", ctypes.c_void_p), ("rstd_out", ctypes.c_void_p)]
 
 
 _lib = None
@@ -75,6 +80,9 @@ def lib() -> ctypes.CDLL:
         L.hgf_linear_forward_phases.restype = c.c_int
         L.hgf_linear_forward_phases.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, vp, sz,
                                                 c.POINTER(DebugOut), u32, u32, vp]
+        L.hgf_linear_forward_ln.restype = c.c_int
+        L.hgf_linear_forward_ln.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, vp, sz,
+                                            c.POINTER(DebugOut), c.POINTER(FrontEnd), u32, vp]
         L.hgf_linear_forward_static.restype = c.c_int
         L.hgf_linear_forward_static.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, u32, vp]
         L.hgf_act_quant.restype = c.c_int
@@ -159,11 +167,14 @@ def act_quant(x: torch.Tensor, stream=None):
 
 
 def linear_forward(x, packed, gamma, d_in, d_out, At=None, Bt=None, gate=None, *, y=None, workspace=None,
-                   debug=False, flags=0, stream=None, phases=None):
+                   debug=False, flags=0, stream=None, phases=None, ln_weight=None, ln_bias=None, eps=1e-5,
+                   gate_group=None):
     """Enqueue one layer forward.  Returns y, or (y, dbg dict of device tensors) with debug=True.
 
     x bf16 [M][d_in]; packed uint8 from pack_ternary; At fp16 [r][d_in]; Bt fp16 [d_out][r];
     gate fp32 [d_out]; y fp32 (or bf16 with FLAG_OUT_BF16) [M][d_out].
+    With ln_weight / ln_bias (fp32 [d_in]) and/or gate_group the call is hgf_linear_forward_ln: LayerNorm
+    in front of the quantiser, gate fp32 [ceil(d_out / gate_group)]; debug then also returns mean and rstd.
     """
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
     M = x.shape[0]
@@ -182,7 +193,18 @@ def linear_forward(x, packed, gamma, d_in, d_out, At=None, Bt=None, gate=None, *
         dbg_struct = DebugOut(dbg["xq"].data_ptr(), dbg["gamma_x"].data_ptr(), dbg["y_int"].data_ptr(),
                               dbg["h"].data_ptr())
     dbg_arg = ctypes.byref(dbg_struct) if dbg_struct is not None else None
-    if phases is None:
+    if ln_weight is not None or gate_group is not None:
+        assert phases is None
+        fe = FrontEnd(None if ln_weight is None else ln_weight.data_ptr(), None if ln_bias is None else ln_bias.data_ptr(),
+                      float(eps), int(gate_group or 1), None, None)
+        if debug:
+            dbg["mean"] = torch.empty(M, dtype=torch.float32, device=x.device)
+            dbg["rstd"] = torch.empty(M, dtype=torch.float32, device=x.device)
+            fe.mean_out, fe.rstd_out = dbg["mean"].data_ptr(), dbg["rstd"].data_ptr()
+        st = lib().hgf_linear_forward_ln(_ptr(x), M, _ptr(packed), ctypes.c_float(gamma), d_in, d_out, _ptr(At), _ptr(Bt),
+                                         r, _ptr(gate), _ptr(y), _ptr(workspace), workspace.numel(), dbg_arg,
+                                         ctypes.byref(fe), flags, _stream(stream))
+    elif phases is None:
         st = lib().hgf_linear_forward(_ptr(x), M, _ptr(packed), ctypes.c_float(gamma), d_in, d_out, _ptr(At), _ptr(Bt),
                                       r, _ptr(gate), _ptr(y), _ptr(workspace), workspace.numel(), dbg_arg, flags,
                                       _stream(stream))
