@@ -14,9 +14,12 @@ from .hgf_oracle import (  # noqa: F401
     ln_quant,
     ln_stats,
     pack,
+    pack_b3,
     packed_bytes,
+    packed_bytes_b3,
     ternarise,
     threads,
     tmax,
     unpack,
+    unpack_b3,
 )

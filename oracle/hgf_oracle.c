@@ -142,6 +142,67 @@ int64_t oracle_unpack(const uint8_t *packed, int64_t d_out, int64_t d_in, int8_t
     return bad;
 }
 
+/* ---- base-3 packed layout: five ternary codes per byte, 1.6 bits per weight ------------------- */
+/* The paper counts log2(3) = 1.58 bits per weight; five codes c = t + 1 in {0,1,2} fit one byte as
+ * the base-3 number c0 + 3 c1 + 9 c2 + 27 c3 + 81 c4 (0..242).  The matrix is cut into tiles of 16
+ * output rows by 320 input columns (d_out padded to 16, d_in to 320, with zero weights); a tile is
+ * 1024 bytes, its 16 rows one after the other, 64 bytes per row; tiles are stored with the column
+ * tile running fastest: tile (R, C) starts at byte (R * (d_in_padded / 320) + C) * 1024.
+ * Which five columns of its row a byte holds: write the byte's index in the row as q = 16 t + j
+ * (t in 0..3, j in 0..15) and let col(p, t) = 32 (p / 2) + 16 (p % 2) + 4 t for p in 0..19.  Then
+ * digit e < 4 of the byte is the code of tile column col(j, t) + e, and digit 4 is the code of tile
+ * column col(16 + j / 4, t) + j % 4. */
+static int64_t padded_cols_b3(int64_t d_in) { return (d_in + 319) / 320 * 320; }
+
+int64_t oracle_packed_bytes_b3(int64_t d_out, int64_t d_in) { return padded_rows(d_out) * padded_cols_b3(d_in) / 5; }
+
+/* Byte offset of the byte that holds weight (n, k), and the power of three its code is scaled by. */
+static int64_t byte_offset_b3(int64_t n, int64_t k, int64_t d_in, int *power) {
+    static const int pow3[5] = {1, 3, 9, 27, 81};
+    int64_t col_tiles = padded_cols_b3(d_in) / 320;
+    int64_t R = n / 16, row = n % 16, C = k / 320, col = k % 320;
+    int64_t p = 2 * (col / 32) + (col % 32) / 16, t = (col % 16) / 4, e = col % 4;
+    int64_t j;
+    if (p < 16) {
+        j = p;
+        *power = pow3[e];
+    } else {
+        j = 4 * (p - 16) + e;
+        *power = pow3[4];
+    }
+    return (R * col_tiles + C) * 1024 + row * 64 + 16 * t + j;
+}
+
+void oracle_pack_b3(const int8_t *T, int64_t d_out, int64_t d_in, uint8_t *packed) {
+    int64_t rows = padded_rows(d_out), cols = padded_cols_b3(d_in);
+    memset(packed, 0, (size_t)(rows * cols / 5));
+    for (int64_t n = 0; n < rows; ++n)
+        for (int64_t k = 0; k < cols; ++k) {
+            int t = (n < d_out && k < d_in) ? T[n * d_in + k] : 0; /* padding is weight 0 */
+            int power;
+            int64_t off = byte_offset_b3(n, k, d_in, &power);
+            packed[off] = (uint8_t)(packed[off] + (t + 1) * power);
+        }
+}
+
+/* Returns the number of invalid bytes (value above 242) met; their codes decode to 0. */
+int64_t oracle_unpack_b3(const uint8_t *packed, int64_t d_out, int64_t d_in, int8_t *T) {
+    int64_t bad = 0;
+    for (int64_t n = 0; n < d_out; ++n)
+        for (int64_t k = 0; k < d_in; ++k) {
+            int power;
+            int64_t off = byte_offset_b3(n, k, d_in, &power);
+            int v = packed[off];
+            if (v > 242) {
+                bad += (power == 1); /* count each bad byte once per column group that starts in it */
+                T[n * d_in + k] = 0;
+                continue;
+            }
+            T[n * d_in + k] = (int8_t)((v / power) % 3 - 1);
+        }
+    return bad;
+}
+
 /* ---- Section 2.2.1 / Algorithm 1 steps 1-2: per-token absmax int8 quantisation --------------- */
 /* gamma_x = max_k |x_k| (floored at 1e-5 so that an all-zero token does not divide by zero; the
  * floored value is used for both quantisation and dequantisation);

@@ -51,6 +51,12 @@ def _load():
         lib.oracle_pack.argtypes = [vp, i64, i64, vp]
         lib.oracle_unpack.restype = i64
         lib.oracle_unpack.argtypes = [vp, i64, i64, vp]
+        lib.oracle_packed_bytes_b3.restype = i64
+        lib.oracle_packed_bytes_b3.argtypes = [i64, i64]
+        lib.oracle_pack_b3.restype = None
+        lib.oracle_pack_b3.argtypes = [vp, i64, i64, vp]
+        lib.oracle_unpack_b3.restype = i64
+        lib.oracle_unpack_b3.argtypes = [vp, i64, i64, vp]
         lib.oracle_act_quant.restype = None
         lib.oracle_act_quant.argtypes = [vp, i64, i64, vp, vp]
         lib.oracle_int_gemm.restype = c.c_int
@@ -116,6 +122,26 @@ def unpack(packed, d_out: int, d_in: int, return_bad: bool = False):
     packed = _arr(packed, np.uint8, (packed_bytes(d_out, d_in),))
     T = np.empty((d_out, d_in), np.int8)
     bad = int(_load().oracle_unpack(_p(packed), d_out, d_in, _p(T)))
+    return (T, bad) if return_bad else T
+
+
+def packed_bytes_b3(d_out: int, d_in: int) -> int:
+    return int(_load().oracle_packed_bytes_b3(d_out, d_in))
+
+
+def pack_b3(T) -> np.ndarray:
+    """Base-3 layout: five codes per byte (1.6 bits per weight)."""
+    T = _arr(T, np.int8)
+    d_out, d_in = T.shape
+    out = np.zeros(packed_bytes_b3(d_out, d_in), np.uint8)
+    _load().oracle_pack_b3(_p(T), d_out, d_in, _p(out))
+    return out
+
+
+def unpack_b3(packed, d_out: int, d_in: int, return_bad: bool = False):
+    packed = _arr(packed, np.uint8, (packed_bytes_b3(d_out, d_in),))
+    T = np.empty((d_out, d_in), np.int8)
+    bad = int(_load().oracle_unpack_b3(_p(packed), d_out, d_in, _p(T)))
     return (T, bad) if return_bad else T
 
 
