@@ -50,6 +50,7 @@ typedef enum {
                                     path on decode-sized inputs) */
 
 #define HGF_FLAG_NO_PDL 0x8u     /* do not use programmatic dependent launch (see hgf_linear_forward) */
+#define HGF_FLAG_BASE3 0x10u     /* `packed` is in the base-3 layout of hgf_pack_ternary_b3 (decode path only) */
 
 /* Largest token count the register-resident decode path handles; above it the GEMM path runs. */
 #define HGF_DECODE_MAX_M 16
@@ -94,6 +95,30 @@ hgf_status hgf_pack_ternary(const float *W, int64_t d_out, int64_t d_in, void *p
 /* Inverse of the packing: T[n][k] in {-1,0,1} as int8, device [d_out][d_in].  Enqueue only. */
 hgf_status hgf_unpack_ternary(const void *packed, int64_t d_out, int64_t d_in, int8_t *T,
                               void *stream);
+
+/*
+ * The same weights at 1.6 bits each: five codes per byte as the base-3 number
+ * c0 + 3 c1 + 9 c2 + 27 c3 + 81 c4 (0..242), the nearest byte-aligned packing to the log2(3) = 1.58
+ * bits the paper counts per ternary weight (Introduction, the T_max bound; Section 4.2, the
+ * effective bit-width).  It takes a fifth off the weight stream of the memory-bound decode path at
+ * the price of a table look-up per byte; forward calls take it with HGF_FLAG_BASE3, on the decode
+ * path only (M <= HGF_DECODE_MAX_M; the compute-bound GEMM path wants the two-bit layout and returns
+ * HGF_ERR_UNSUPPORTED_SHAPE).
+ * Layout: tiles of 16 output rows by 320 input columns (d_out padded to 16, d_in to 320, with zero
+ * weights); a tile is 1024 bytes, its 16 rows one after the other, 64 bytes per row; tile (R, C)
+ * starts at byte (R * (d_in_padded / 320) + C) * 1024.  Byte q = 16 t + j (t in 0..3, j in 0..15) of a
+ * row holds in digit e < 4 the code of tile column col(j, t) + e and in digit 4 the code of tile column
+ * col(16 + j / 4, t) + j % 4, with col(p, t) = 32 (p / 2) + 16 (p % 2) + 4 t.  Examples: column 0 is
+ * digit 0 of byte 0, column 5 digit 1 of byte 16, column 16 digit 0 of byte 1, column 47 digit 3 of
+ * byte 50, column 256 digit 4 of byte 0, column 319 digit 4 of byte 63.
+ * hgf_packed_bytes_b3 returns ceil(d_out / 16) * 16 * ceil(d_in / 320) * 320 / 5, or 0 for invalid
+ * sizes.  Arguments and behaviour of the other two calls are those of their two-bit counterparts.
+ */
+size_t hgf_packed_bytes_b3(int64_t d_out, int64_t d_in);
+hgf_status hgf_pack_ternary_b3(const float *W, int64_t d_out, int64_t d_in, void *packed,
+                               float *gamma_out, void *stream);
+hgf_status hgf_unpack_ternary_b3(const void *packed, int64_t d_out, int64_t d_in, int8_t *T,
+                                 void *stream);
 
 /* Bytes of caller-provided scratch hgf_linear_forward needs for this problem (never 0). */
 size_t hgf_workspace_bytes(int64_t M, int64_t d_in, int64_t d_out, int32_t r, uint32_t flags);

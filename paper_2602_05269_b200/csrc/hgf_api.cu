@@ -54,7 +54,7 @@ static bool misaligned(const void *p) { return p && (((uintptr_t)p) & 15u); }
 // for that (and every M > 16) take the GEMM path.
 static bool takes_gemm_path(int64_t M, int64_t d_in, uint32_t flags) {
     if (M > HGF_DECODE_MAX_M || (flags & HGF_FLAG_FORCE_GEMM)) return true;
-    return decode_xq_smem_bytes((int)M, (int)d_in) > decode_xq_smem_limit();
+    return decode_xq_smem_bytes((int)M, (int)d_in, flags) > decode_xq_smem_limit();
 }
 
 }  // namespace hgf
@@ -89,12 +89,13 @@ static hgf_status validate_problem(const void *x, int64_t M, const void *packed,
                                    const void *At, const void *Bt, int32_t r, const float *gate, const void *y,
                                    uint32_t flags, int32_t *r_eff, bool *gemm) {
     if (!x || !packed || !y || M <= 0 || d_in <= 0 || d_out <= 0 || r < 0) return HGF_ERR_INVALID_ARG;
-    if (flags & ~(HGF_FLAG_OUT_BF16 | HGF_FLAG_NO_SILU | HGF_FLAG_FORCE_GEMM | HGF_FLAG_NO_PDL)) return HGF_ERR_INVALID_ARG;
+    if (flags & ~(HGF_FLAG_OUT_BF16 | HGF_FLAG_NO_SILU | HGF_FLAG_FORCE_GEMM | HGF_FLAG_NO_PDL | HGF_FLAG_BASE3)) return HGF_ERR_INVALID_ARG;
     if (!At || !Bt || !gate) r = 0;  // pure ternary layer
     if (d_in % 64 != 0 || d_in > 65536 || d_out > (1 << 24) || M > (1 << 22)) return HGF_ERR_UNSUPPORTED_SHAPE;
     if (r != 0 && r != 16 && r != 32 && r != 48 && r != 64) return HGF_ERR_UNSUPPORTED_SHAPE;
     *gemm = takes_gemm_path(M, d_in, flags);
     if (*gemm && (d_out % 8 != 0)) return HGF_ERR_UNSUPPORTED_SHAPE;
+    if (*gemm && (flags & HGF_FLAG_BASE3)) return HGF_ERR_UNSUPPORTED_SHAPE;  // base-3 weights serve the byte-bound decode path
     if (misaligned(x) || misaligned(packed) || misaligned(y) || misaligned(At) || misaligned(Bt) || misaligned(gate))
         return HGF_ERR_MISALIGNED;
     *r_eff = r;
@@ -237,9 +238,9 @@ hgf_status hgf::forward_impl(const void *x, int64_t M, const void *packed, float
         dl.probs = nullptr;
         dl.n_probs = 1;
         dl.total_tiles = (int)row_tiles(d_out);
-        dl.total_cost = (long long)dl.total_tiles * row_tile_cost((int)d_in);
+        dl.total_cost = (long long)dl.total_tiles * row_tile_cost((int)d_in, flags);
         dl.max_M = (int)M;
-        dl.xq_smem_bytes = decode_xq_smem_bytes((int)M, (int)d_in);
+        dl.xq_smem_bytes = decode_xq_smem_bytes((int)M, (int)d_in, flags);
         return launch_decode_gemv(dl, &dp, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
     }
 
@@ -432,9 +433,9 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
             hpart += (size_t)jts * slices * 8 * 32;
         }
         tiles += (int)row_tiles(q.d_out);
-        cost += (long long)row_tiles(q.d_out) * row_tile_cost((int)q.d_in);
+        cost += (long long)row_tiles(q.d_out) * row_tile_cost((int)q.d_in, flags);
         max_M = q.M > max_M ? (int)q.M : max_M;
-        const int xb = decode_xq_smem_bytes((int)q.M, (int)q.d_in);
+        const int xb = decode_xq_smem_bytes((int)q.M, (int)q.d_in, flags);
         xq_smem = xb > xq_smem ? xb : xq_smem;
     }
     hgf_group *g = new (std::nothrow) hgf_group();
@@ -460,7 +461,7 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
                 const int mid = (lo + hi + 1) >> 1;
                 if (dps[mid].cost_begin <= c) lo = mid; else hi = mid - 1;
             }
-            const long long steps = row_tile_cost(dps[lo].K), tl = row_tiles(dps[lo].N);
+            const long long steps = row_tile_cost(dps[lo].K, flags), tl = row_tiles(dps[lo].N);
             long long local = (c - dps[lo].cost_begin + steps - 1) / steps;
             if (local > tl) local = tl;
             *prob = lo;
@@ -523,6 +524,7 @@ extern "C" hgf_status hgf_group_forward_phases(hgf_group *g, uint32_t phases, vo
     dl.max_M = g->max_M;
     dl.xq_smem_bytes = g->xq_smem_bytes;
     dl.cta_range = g->grid == decode_grid(g->total_tiles) ? g->d_cta_range : nullptr;
+    dl.flags = g->flags;
     return launch_decode_gemv(dl, nullptr, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
 }
 

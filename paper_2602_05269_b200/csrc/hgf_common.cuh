@@ -47,6 +47,8 @@ static inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, std::ato
 // d_out to a multiple of 16 with code 1 (weight 0).
 static inline int64_t padded_k(int64_t d_in) { return (d_in + 255) / 256 * 256; }
 static inline int64_t row_tiles(int64_t d_out) { return (d_out + 15) / 16; }
+// Base-3 layout (five codes per byte): tiles of 16 output rows x 320 input columns, also 1 KiB each.
+static inline int64_t padded_k_b3(int64_t d_in) { return (d_in + 319) / 320 * 320; }
 
 // ---- workspace layout (all sections 256-byte aligned) --------------------------------------
 //   xq       [M][d_in]   int8     quantised activations
@@ -134,7 +136,9 @@ struct FrontEnd {
 // weight tiles (measured: a layer with short rows runs slower per byte than one with long rows by
 // about this much per row tile).
 constexpr int kRowTileOverhead = 6;
-__host__ __device__ inline long long row_tile_cost(int K) { return (long long)((K + 255) >> 8) + kRowTileOverhead; }
+// 1 KiB weight tiles per 16-row tile: 256 columns each at two bits per weight, 320 in the base-3 layout.
+__host__ __device__ inline int weight_steps(int K, uint32_t flags) { return (flags & HGF_FLAG_BASE3) ? (K + 319) / 320 : (K + 255) >> 8; }
+__host__ __device__ inline long long row_tile_cost(int K, uint32_t flags) { return (long long)weight_steps(K, flags) + kRowTileOverhead; }
 
 // One layer problem of a decode launch (M <= 16).  tile_begin = index of its first 16-row tile in
 // the launch-wide tile numbering; cost_begin = sum of the costs of all row tiles of earlier problems.
@@ -167,6 +171,7 @@ struct DecodeLaunch {
     int max_M;                   // largest token count of any problem
     int xq_smem_bytes;           // shared memory for the largest problem's activations
     int ring_slots;              // weight-ring slots per warp (set by the launcher)
+    uint32_t flags;              // the launch's layout flag (HGF_FLAG_BASE3) for a group; a single problem carries its own
     const int4 *cta_range;       // per CTA: first tile, end tile, first problem (device array), or null
 };
 
@@ -203,7 +208,7 @@ cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_q
 cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream);
 cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream);
 // Shared memory the decode kernel needs for one problem's activations, and the largest it accepts.
-int decode_xq_smem_bytes(int M, int K);
+int decode_xq_smem_bytes(int M, int K, uint32_t flags);
 int decode_xq_smem_limit();
 // Grid of the decode GEMV for a launch with that many row tiles (0 if the device cannot be queried).
 int decode_grid(int total_tiles);

@@ -55,13 +55,20 @@ constexpr int kRedBytes = kDecWarps * 8 * 32 * 4;  // per warp: up to 8 accumula
 constexpr int kOffFlags = kOffRed + kRedBytes;
 constexpr int kOffXq = (kOffFlags + 64 + 127) / 128 * 128;
 constexpr int kSmemLimit = 227 * 1024;
-constexpr int kXqLimit = (kSmemLimit - kOffXq - kMinSlots * kDecWarps * kSmallSlotTiles * kTileBytes) / 128 * 128;
+// Base-3 weights: the decode table sits in front of the activations (four copies of 256 entries of
+// 8 bytes: the first four codes of a byte as four bytes of one word, and its fifth code already
+// moved to the byte position the entry's copy stands for).
+constexpr int kLutBytes = 4 * 256 * 8;
+constexpr int kXqLimit = (kSmemLimit - kOffXq - kLutBytes - kMinSlots * kDecWarps * kSmallSlotTiles * kTileBytes) / 128 * 128;
 
 constexpr unsigned long long kDecWaitLimitNs = 2000000000ull;  // bounded waits give up after two seconds
 
 // Rows of activations kept in shared memory: the M tokens, plus one row of zeros that stands in for
 // the absent tokens of the 8-token tiles.
-int decode_xq_smem_bytes(int M, int K) { return (M + (M < 16 ? 1 : 0)) * ((int)padded_k(K) + kXqPad); }
+int decode_xq_smem_bytes(int M, int K, uint32_t flags) {
+    const int Kp = (flags & HGF_FLAG_BASE3) ? (int)padded_k_b3(K) : (int)padded_k(K);
+    return (M + (M < 16 ? 1 : 0)) * (Kp + kXqPad);
+}
 int decode_xq_smem_limit() { return kXqLimit; }
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -142,7 +149,7 @@ struct Item {
 __device__ __forceinline__ const DecodeProblem &problem_of(const DecodeLaunch &L, const DecodeProblem &single, int p) {
     return L.probs ? L.probs[p] : single;
 }
-__device__ __forceinline__ int steps_of(int K) { return (K + 255) >> 8; }
+__device__ __forceinline__ int b3_col(int p, int t) { return 32 * (p >> 1) + 16 * (p & 1) + 4 * t; }
 __device__ __forceinline__ int tiles_of(int N) { return (N + 15) >> 4; }
 
 // Smallest launch-wide tile index at which the cost of all earlier row tiles is >= cost.
@@ -153,7 +160,7 @@ __device__ int tile_of_cost(const DecodeLaunch &L, const DecodeProblem &single, 
         if (problem_of(L, single, mid).cost_begin <= cost) lo = mid; else hi = mid - 1;
     }
     const DecodeProblem &P = problem_of(L, single, lo);
-    const long long steps = row_tile_cost(P.K);
+    const long long steps = row_tile_cost(P.K, P.flags);
     const int tiles = tiles_of(P.N);
     long long local = (cost - P.cost_begin + steps - 1) / steps;
     if (local > tiles) local = tiles;
@@ -184,7 +191,7 @@ __device__ bool next_segment(const DecodeLaunch &L, const DecodeProblem &single,
         if (tb >= t1) return false;
         const int lo = t0 > tb ? t0 : tb, hi = t1 < te ? t1 : te;
         if (lo < hi) {
-            s.p = p; s.lo = lo; s.hi = hi; s.tile_begin = tb; s.nsteps = steps_of(P.K); s.packed = P.packed;
+            s.p = p; s.lo = lo; s.hi = hi; s.tile_begin = tb; s.nsteps = weight_steps(P.K, P.flags); s.packed = P.packed;
             return true;
         }
     }
@@ -222,24 +229,39 @@ struct Producer {
     bool done;
 };
 
-// NT = number of 8-token tiles (1: M <= 8, 2: M <= 16); ST = tiles per ring slot.
-template <int NT, int ST>
+// NT = number of 8-token tiles (1: M <= 8, 2: M <= 16); ST = tiles per ring slot; B3 = the weights
+// are in the base-3 layout (tiles of 320 columns, decoded through a table in shared memory).
+template <int NT, int ST, bool B3>
 __global__ void __launch_bounds__(kDecThreads, 1)
 decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned int *status) {
     constexpr int kSlotTiles = ST, kSlotBytes = ST * kTileBytes;
+    constexpr int kTileCols = B3 ? 320 : 256, kLut = B3 ? kLutBytes : 0;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int slots = L.ring_slots;  // slots of this warp's ring, kSlotBytes each
-    uint8_t *ring = smem + kOffXq + ((L.xq_smem_bytes + 127) & ~127) + warp * slots * kSlotBytes;
+    uint8_t *ring = smem + kOffXq + kLut + ((L.xq_smem_bytes + 127) & ~127) + warp * slots * kSlotBytes;
     const uint32_t ring_u32 = dsmem_u32(ring);
     const uint32_t bars_u32 = dsmem_u32(smem + kOffBars) + warp * kMaxSlots * 8;
     SegSmall *small = reinterpret_cast<SegSmall *>(smem + kOffSmall);
     int *red = reinterpret_cast<int *>(smem + kOffRed);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffFlags);
-    int8_t *xq_s = reinterpret_cast<int8_t *>(smem + kOffXq);
+    int8_t *xq_s = reinterpret_cast<int8_t *>(smem + kOffXq + kLut);
+    const uint32_t lut_u32 = dsmem_u32(smem + kOffXq);
 
     pdl_launch_dependents();
     if (tid == 0) *abort_flag = 0;
+    if (B3) {
+        // copy e of the table, entry b: .x = codes 0..3 of byte value b, one per byte; .y = code 4 in byte e.
+        // Values above 242 never occur in a packed matrix; they decode as zero weights (code 1).
+        uint2 *lut = reinterpret_cast<uint2 *>(smem + kOffXq);
+        for (int i = tid; i < 4 * 256; i += kDecThreads) {
+            const int e = i >> 8, b = i & 255;
+            uint2 v = make_uint2(0x01010101u, 1u << (8 * e));
+            if (b <= 242) v = make_uint2((uint32_t)(b % 3) | ((uint32_t)(b / 3 % 3) << 8) | ((uint32_t)(b / 9 % 3) << 16) | ((uint32_t)(b / 27 % 3) << 24),
+                                         (uint32_t)(b / 81) << (8 * e));
+            lut[i] = v;
+        }
+    }
     if (lane == 0) {
         for (int s = 0; s < slots; ++s) dmbar_init(bars_u32 + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -320,7 +342,7 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
          more = next_segment(L, single, t0, t1, false, seg), ++seg_idx) {
         const DecodeProblem &Pg = problem_of(L, single, seg.p);
         const int K = Pg.K, M = Pg.M, N = Pg.N, r = Pg.r;
-        const int Kp = seg.nsteps * 256, pitch = Kp + kXqPad;
+        const int Kp = seg.nsteps * kTileCols, pitch = Kp + kXqPad;
         SegSmall &sm = small[seg_idx & 1];
 
         // stage the problem's activations and per-token values (all reads of the previous
@@ -337,7 +359,23 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
             if (M < 16)  // the row of zeros
                 for (int u = tid; u < (Kp >> 4); u += kDecThreads)
                     *reinterpret_cast<uint4 *>(xq_s + (size_t)M * pitch + 16 * u) = make_uint4(0u, 0u, 0u, 0u);
-            for (int u = tid; u < M * groups_per_row; u += kDecThreads) {
+            if (B3) {
+                // Base-3 tiles have 320 columns; lane t's five 16-byte units of a tile sit at bytes
+                // 64 u + 16 t of it and hold, four bytes each, the columns col(4 u + i, t) .. + 3, i = 0..3 -
+                // the second operands of the MMAs whose first operands come out of the lane's 16 weight bytes.
+                const int units_per_row = seg.nsteps * 20;
+                for (int v = tid; v < M * units_per_row; v += kDecThreads) {
+                    const int m = v / units_per_row, rem = v - m * units_per_row, c = rem / 20, ut = rem - c * 20, u = ut >> 2, tt = ut & 3;
+                    uint32_t r4[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int k = c * 320 + b3_col(4 * u + i, tt);
+                        r4[i] = k < K ? *reinterpret_cast<const uint32_t *>(xq_g + (size_t)m * K + k) : 0u;
+                    }
+                    *reinterpret_cast<uint4 *>(xq_s + (size_t)m * pitch + c * 320 + 64 * u + 16 * tt) = make_uint4(r4[0], r4[1], r4[2], r4[3]);
+                }
+            }
+            for (int u = tid; !B3 && u < M * groups_per_row; u += kDecThreads) {
                 const int m = u / groups_per_row, q = u - m * groups_per_row;
                 uint4 v0 = make_uint4(0u, 0u, 0u, 0u), v1 = v0;
                 if (32 * q < K) {
@@ -506,6 +544,39 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
                 const uint4 qq = *reinterpret_cast<const uint4 *>(wt + 512);
                 const uint32_t pw[4] = {pq.x, pq.y, pq.z, pq.w};
                 const uint32_t qw[4] = {qq.x, qq.y, qq.z, qq.w};
+                if constexpr (B3) {
+                    // The lane's 16 bytes of row g (pw) and of row g + 8 (qw): byte 4 w + e gives, through the
+                    // table, the first operand of one half of MMA 2 w + e / 2 (four codes), and the fifth codes
+                    // of a word's four bytes together make one operand register of MMAs 8 and 9.
+                    uint32_t f5g[4], f5h[4];
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        uint32_t ag[4], ah[4];
+                        f5g[w] = 0u; f5h[w] = 0u;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            uint2 vg, vh;
+                            const uint32_t a_g = lut_u32 + 2048 * e + (((pw[w] >> (8 * e)) & 0xffu) << 3);
+                            const uint32_t a_h = lut_u32 + 2048 * e + (((qw[w] >> (8 * e)) & 0xffu) << 3);
+                            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(vg.x), "=r"(vg.y) : "r"(a_g));
+                            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(vh.x), "=r"(vh.y) : "r"(a_h));
+                            ag[e] = vg.x; ah[e] = vh.x;
+                            f5g[w] |= vg.y; f5h[w] |= vh.y;
+                        }
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const uint4 xv = *reinterpret_cast<const uint4 *>(xt[nt] + 64 * w);
+                            mma_u8s8(acc[nt][0], ag[0], ah[0], ag[1], ah[1], xv.x, xv.y);
+                            mma_u8s8(acc[nt][0], ag[2], ah[2], ag[3], ah[3], xv.z, xv.w);
+                        }
+                    }
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const uint4 xv = *reinterpret_cast<const uint4 *>(xt[nt] + 64 * 4);
+                        mma_u8s8(acc[nt][0], f5g[0], f5h[0], f5g[1], f5h[1], xv.x, xv.y);
+                        mma_u8s8(acc[nt][0], f5g[2], f5h[2], f5g[3], f5h[3], xv.z, xv.w);
+                    }
+                } else {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     uint4 xa[NT], xb[NT];
@@ -527,10 +598,11 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
                         }
                     }
                 }
+                }
             };
             const int8_t *xt[NT];
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) xt[nt] = xrow[nt] + it.ks0 * 256;
+            for (int nt = 0; nt < NT; ++nt) xt[nt] = xrow[nt] + it.ks0 * kTileCols;
             const int ntiles = it.ks1 - it.ks0;
             for (int left = ntiles; left > 0 && ok;) {  // slot by slot; the last may hold fewer tiles
                 if (!(ok = wait_slot())) break;  // stop computing and copying; requested slots stay outstanding
@@ -541,7 +613,7 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
                     if (q < n) {
                         compute_tile(sl + q * kTileBytes, xt);
 #pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) xt[nt] += 256;
+                        for (int nt = 0; nt < NT; ++nt) xt[nt] += kTileCols;
                     }
                 }
                 release_slot();
@@ -599,12 +671,18 @@ int decode_grid(int total_tiles) {
     return total_tiles < sms ? total_tiles : sms;
 }
 
-template <int NT, int ST>
+template <int NT, int ST, bool B3>
 static cudaError_t launch_decode_variant(cudaLaunchConfig_t &cfg, const DecodeLaunch &L, const DecodeProblem &sp, unsigned int *status) {
     static std::atomic<unsigned long long> attr_done{0};
-    cudaError_t e = ensure_dynamic_smem(decode_gemv_kernel<NT, ST>, kSmemLimit, attr_done);
+    cudaError_t e = ensure_dynamic_smem(decode_gemv_kernel<NT, ST, B3>, kSmemLimit, attr_done);
     if (e != cudaSuccess) return e;
-    return cudaLaunchKernelEx(&cfg, decode_gemv_kernel<NT, ST>, L, sp, status);
+    return cudaLaunchKernelEx(&cfg, decode_gemv_kernel<NT, ST, B3>, L, sp, status);
+}
+template <bool B3>
+static cudaError_t launch_decode_layout(cudaLaunchConfig_t &cfg, const DecodeLaunch &L, const DecodeProblem &sp, unsigned int *status, bool big) {
+    if (L.max_M <= 8)
+        return big ? launch_decode_variant<1, kBigSlotTiles, B3>(cfg, L, sp, status) : launch_decode_variant<1, kSmallSlotTiles, B3>(cfg, L, sp, status);
+    return big ? launch_decode_variant<2, kBigSlotTiles, B3>(cfg, L, sp, status) : launch_decode_variant<2, kSmallSlotTiles, B3>(cfg, L, sp, status);
 }
 
 cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *single, bool pdl, cudaStream_t stream) {
@@ -616,8 +694,10 @@ cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *si
     DecodeLaunch L = L_in;
     // the ring beside the activations: two slots of four tiles if they fit, else as many slots of two
     // tiles as shared memory allows
+    const bool b3 = ((single ? single->flags : L_in.flags) & HGF_FLAG_BASE3) != 0;
+    const int lut = b3 ? kLutBytes : 0;
     const int xq_bytes = (L.xq_smem_bytes + 127) & ~127;
-    const int room = kSmemLimit - kOffXq - xq_bytes;
+    const int room = kSmemLimit - kOffXq - lut - xq_bytes;
     const bool big = room >= kDecWarps * kBigSlots * kBigSlotTiles * kTileBytes;
     const int slot_bytes = (big ? kBigSlotTiles : kSmallSlotTiles) * kTileBytes;
     int slots = big ? kBigSlots : room / (kDecWarps * slot_bytes);
@@ -629,18 +709,14 @@ cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *si
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kDecThreads);
-    cfg.dynamicSmemBytes = (size_t)(kOffXq + xq_bytes + kDecWarps * slots * slot_bytes);
+    cfg.dynamicSmemBytes = (size_t)(kOffXq + lut + xq_bytes + kDecWarps * slots * slot_bytes);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    cudaError_t e;
-    if (L.max_M <= 8)
-        e = big ? launch_decode_variant<1, kBigSlotTiles>(cfg, L, sp, status) : launch_decode_variant<1, kSmallSlotTiles>(cfg, L, sp, status);
-    else
-        e = big ? launch_decode_variant<2, kBigSlotTiles>(cfg, L, sp, status) : launch_decode_variant<2, kSmallSlotTiles>(cfg, L, sp, status);
+    cudaError_t e = b3 ? launch_decode_layout<true>(cfg, L, sp, status, big) : launch_decode_layout<false>(cfg, L, sp, status, big);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }

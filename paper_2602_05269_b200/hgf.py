@@ -18,6 +18,7 @@ FLAG_OUT_BF16 = 0x1
 FLAG_NO_SILU = 0x2
 FLAG_FORCE_GEMM = 0x4
 FLAG_NO_PDL = 0x8
+FLAG_BASE3 = 0x10
 DECODE_MAX_M = 16
 PHASE_PROLOGUE = 0x1
 PHASE_GEMV = 0x2
@@ -27,7 +28,8 @@ EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_wo
            "hgf_linear_forward", "hgf_act_quant", "hgf_check_status", "hgf_tmax_tokens_per_s",
            "hgf_launch_count", "hgf_status_string", "hgf_group_create", "hgf_group_forward",
            "hgf_group_destroy", "hgf_group_forward_phases", "hgf_linear_forward_static", "hgf_group_debug",
-           "hgf_linear_forward_phases", "hgf_linear_forward_ln"]
+           "hgf_linear_forward_phases", "hgf_linear_forward_ln",
+           "hgf_packed_bytes_b3", "hgf_pack_ternary_b3", "hgf_unpack_ternary_b3"]
 
 
 class HgfError(RuntimeError):
@@ -72,6 +74,12 @@ def lib() -> ctypes.CDLL:
         L.hgf_pack_ternary.argtypes = [vp, i64, i64, vp, c.POINTER(c.c_float), vp]
         L.hgf_unpack_ternary.restype = c.c_int
         L.hgf_unpack_ternary.argtypes = [vp, i64, i64, vp, vp]
+        L.hgf_packed_bytes_b3.restype = sz
+        L.hgf_packed_bytes_b3.argtypes = [i64, i64]
+        L.hgf_pack_ternary_b3.restype = c.c_int
+        L.hgf_pack_ternary_b3.argtypes = [vp, i64, i64, vp, c.POINTER(c.c_float), vp]
+        L.hgf_unpack_ternary_b3.restype = c.c_int
+        L.hgf_unpack_ternary_b3.argtypes = [vp, i64, i64, vp, vp]
         L.hgf_workspace_bytes.restype = sz
         L.hgf_workspace_bytes.argtypes = [i64, i64, i64, i32, u32]
         L.hgf_linear_forward.restype = c.c_int
@@ -127,27 +135,29 @@ def status_string(status: int) -> str:
     return lib().hgf_status_string(int(status)).decode()
 
 
-def packed_bytes(d_out: int, d_in: int) -> int:
-    return int(lib().hgf_packed_bytes(d_out, d_in))
+def packed_bytes(d_out: int, d_in: int, base3: bool = False) -> int:
+    return int(lib().hgf_packed_bytes_b3(d_out, d_in) if base3 else lib().hgf_packed_bytes(d_out, d_in))
 
 
-def pack_ternary(W: torch.Tensor, stream=None):
-    """W: CUDA fp32 [d_out][d_in] -> (packed uint8 [d_out*d_in/4] on the device, gamma_W as float)."""
+def pack_ternary(W: torch.Tensor, stream=None, base3: bool = False):
+    """W: CUDA fp32 [d_out][d_in] -> (packed uint8 on the device, gamma_W as float): two bits per weight, or
+    with base3 the 1.6-bit layout of hgf_pack_ternary_b3 (forward calls then take FLAG_BASE3)."""
     assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
     d_out, d_in = W.shape
-    nbytes = packed_bytes(d_out, d_in)
+    nbytes = packed_bytes(d_out, d_in, base3)
     if nbytes == 0:
         raise HgfError("hgf_packed_bytes", 2)
     packed = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
     gamma = ctypes.c_float(0.0)
-    _check("hgf_pack_ternary",
-           lib().hgf_pack_ternary(_ptr(W), d_out, d_in, _ptr(packed), ctypes.byref(gamma), _stream(stream)))
+    fn = lib().hgf_pack_ternary_b3 if base3 else lib().hgf_pack_ternary
+    _check("hgf_pack_ternary", fn(_ptr(W), d_out, d_in, _ptr(packed), ctypes.byref(gamma), _stream(stream)))
     return packed, float(gamma.value)
 
 
-def unpack_ternary(packed: torch.Tensor, d_out: int, d_in: int, stream=None) -> torch.Tensor:
+def unpack_ternary(packed: torch.Tensor, d_out: int, d_in: int, stream=None, base3: bool = False) -> torch.Tensor:
     T = torch.empty((d_out, d_in), dtype=torch.int8, device=packed.device)
-    _check("hgf_unpack_ternary", lib().hgf_unpack_ternary(_ptr(packed), d_out, d_in, _ptr(T), _stream(stream)))
+    fn = lib().hgf_unpack_ternary_b3 if base3 else lib().hgf_unpack_ternary
+    _check("hgf_unpack_ternary", fn(_ptr(packed), d_out, d_in, _ptr(T), _stream(stream)))
     return T
 
 
