@@ -36,9 +36,10 @@ UNIT = "GB/s"
 L2_BYTES = 126e6
 
 
-def layer_bytes(K, N, r, M, out_bytes=4):
-    """Algorithmic bytes one layer call must move: packed W, A, B, gate, x, y."""
-    return K * N // 4 + 2 * r * (K + N) + 4 * N + 2 * M * K + out_bytes * M * N
+def layer_bytes(K, N, r, M, out_bytes=4, base3=False):
+    """Algorithmic bytes one layer call must move: packed W (2 bits per weight, or 1.6 in the base-3
+    layout), A, B, gate, x, y."""
+    return (K * N // 5 if base3 else K * N // 4) + 2 * r * (K + N) + 4 * N + 2 * M * K + out_bytes * M * N
 
 
 def measured_peaks():
@@ -125,6 +126,8 @@ class Workload:
 
     def __init__(self, hgf, torch, shapes, M, copies, flags=0, seed=0, host_io=False, own_ws=False):
         self.hgf, self.torch, self.M, self.flags = hgf, torch, M, flags
+        base3 = bool(flags & hgf.FLAG_BASE3)
+        self.base3 = base3
         dev = torch.device("cuda")
         g = torch.Generator(device=dev)
         g.manual_seed(seed)
@@ -145,7 +148,7 @@ class Workload:
                 if own_ws:
                     self.ws_of.append(torch.empty(hgf.workspace_bytes(M, s.d_in, s.d_out, s.r, flags), dtype=torch.uint8, device=dev))
                 W = torch.randn((s.d_out, s.d_in), generator=g, device=dev, dtype=torch.float32) * 0.02
-                packed, gamma = hgf.pack_ternary(W)
+                packed, gamma = hgf.pack_ternary(W, base3=base3)
                 del W
                 At = (torch.randn((s.r, s.d_in), generator=g, device=dev) / s.d_in ** 0.5).to(torch.float16)
                 Bt = (torch.randn((s.d_out, s.r), generator=g, device=dev) / s.r ** 0.5).to(torch.float16)
@@ -159,7 +162,7 @@ class Workload:
                 xo += M * s.d_in
                 yo += M * s.d_out
                 self.layers.append((s, x, packed, gamma, At, Bt, gate, y))
-                self.bytes += layer_bytes(s.d_in, s.d_out, s.r, M, 2 if flags & hgf.FLAG_OUT_BF16 else 4)
+                self.bytes += layer_bytes(s.d_in, s.d_out, s.r, M, 2 if flags & hgf.FLAG_OUT_BF16 else 4, base3)
                 self.ops += 2 * M * s.d_in * s.d_out
         self.weight_bytes = sum(l[2].numel() + l[4].numel() * 2 + l[5].numel() * 2 for l in self.layers)
         self.graph = None
@@ -260,7 +263,8 @@ class Workload:
     def gemv_bytes(self):
         """Algorithmic bytes of the GEMV launch alone: packed W, B, gate, x~ (int8), y."""
         ob = 2 if self.flags & self.hgf.FLAG_OUT_BF16 else 4
-        return sum(s.d_in * s.d_out // 4 + 2 * s.r * s.d_out + 4 * s.d_out + self.M * s.d_in + ob * self.M * s.d_out
+        wdiv = 5 if self.base3 else 4
+        return sum(s.d_in * s.d_out // wdiv + 2 * s.r * s.d_out + 4 * s.d_out + self.M * s.d_in + ob * self.M * s.d_out
                    for (s, *_rest) in self.layers)
 
     def time_gemv_only(self, stream, steps, warmup):
@@ -542,17 +546,17 @@ def run_extra(hgf, torch, syn, stream, args, peaks, int8_peak_measured=None):
     extra = {"decode_group": [], "decode_per_call": [], "prefill": []}
     steps = max(args.steps // 4, 10)
 
-    def decode_case(cfg, shapes, M, label, min_copies=1, group=True):
-        block = sum(layer_bytes(s.d_in, s.d_out, s.r, M) for s in shapes)
+    def decode_case(cfg, shapes, M, label, min_copies=1, group=True, base3=False):
+        block = sum(layer_bytes(s.d_in, s.d_out, s.r, M, 4, base3) for s in shapes)
         copies = max(min_copies, int(np.ceil(4.4 * L2_BYTES / block)))
-        w = Workload(hgf, torch, shapes, M, copies)
+        w = Workload(hgf, torch, shapes, M, copies, flags=hgf.FLAG_BASE3 if base3 else 0)
         if group:
             w.make_group()
         else:
             w.capture(stream)
         ms = w.time_steps(stream, steps, args.warmup)
         gbs = w.bytes / (ms * 1e-3) / 1e9
-        row = {"workload": label, "M": M, "layers": len(w.layers), "ms_per_step": ms, "GB/s": gbs,
+        row = {"workload": label, "M": M, "bits_per_weight": 1.6 if base3 else 2.0, "layers": len(w.layers), "ms_per_step": ms, "GB/s": gbs,
                "frac_measured_peak": gbs / peaks["hbm_gbs"], "frac_nominal_8000": gbs / 8000.0,
                "launches_per_step": w.launches_per_step}
         if group:
@@ -568,14 +572,17 @@ def run_extra(hgf, torch, syn, stream, args, peaks, int8_peak_measured=None):
         extra["decode_group"].append(decode_case(1, syn.CONFIGS[1]["layers"], M, "config1 1.2B-class block"))
     for M in (1, 8):
         extra["decode_group"].append(decode_case(2, syn.CONFIGS[2]["layers"], M, "config2 3B-class block"))
+    extra["decode_group"].append(decode_case(2, syn.CONFIGS[2]["layers"], 1, "config2 3B-class block", base3=True))
+    extra["decode_group"].append(decode_case(1, syn.CONFIGS[1]["layers"], 1, "config1 1.2B-class block", base3=True))
     # config 4: the 7B-class stack, 32 blocks x 7 projections, decode M = 1 -> tokens/s
     params = 32 * sum(s.d_in * s.d_out for s in syn.CONFIGS[4]["layers"])
-    for group in (True, False):
-        row = decode_case(4, syn.CONFIGS[4]["layers"], 1, "config4 7B-class stack (32 blocks)", min_copies=32, group=group)
+    for group, base3 in ((True, False), (True, True), (False, False)):
+        row = decode_case(4, syn.CONFIGS[4]["layers"], 1, "config4 7B-class stack (32 blocks)", min_copies=32, group=group, base3=base3)
         tok_s = 1e3 / row["ms_per_step"] * (32 * 7 / row["layers"])
         row.update({"tokens_per_s": tok_s, "params": params,
                     "tmax_2bit_measured_bw": hgf.tmax_tokens_per_s(peaks["hbm_gbs"] * 1e9, params, 2.0),
                     "tmax_1p58bit_measured_bw": hgf.tmax_tokens_per_s(peaks["hbm_gbs"] * 1e9, params, 1.58),
+                    "tmax_1p6bit_measured_bw": hgf.tmax_tokens_per_s(peaks["hbm_gbs"] * 1e9, params, 1.6),
                     "tmax_2bit_8TBs": hgf.tmax_tokens_per_s(8e12, params, 2.0),
                     "tmax_1p58bit_8TBs": hgf.tmax_tokens_per_s(8e12, params, 1.58)})
         extra["decode_group" if group else "decode_per_call"].append(row)

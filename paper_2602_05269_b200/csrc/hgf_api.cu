@@ -54,7 +54,7 @@ static bool misaligned(const void *p) { return p && (((uintptr_t)p) & 15u); }
 // for that (and every M > 16) take the GEMM path.
 static bool takes_gemm_path(int64_t M, int64_t d_in, uint32_t flags) {
     if (M > HGF_DECODE_MAX_M || (flags & HGF_FLAG_FORCE_GEMM)) return true;
-    return decode_xq_smem_bytes((int)M, (int)d_in, flags) > decode_xq_smem_limit();
+    return decode_xq_smem_bytes((int)M, (int)d_in, flags) > decode_xq_smem_limit(flags);
 }
 
 }  // namespace hgf

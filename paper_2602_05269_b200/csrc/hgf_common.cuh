@@ -209,7 +209,7 @@ cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtr
 cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream);
 // Shared memory the decode kernel needs for one problem's activations, and the largest it accepts.
 int decode_xq_smem_bytes(int M, int K, uint32_t flags);
-int decode_xq_smem_limit();
+int decode_xq_smem_limit(uint32_t flags);
 // Grid of the decode GEMV for a launch with that many row tiles (0 if the device cannot be queried).
 int decode_grid(int total_tiles);
 

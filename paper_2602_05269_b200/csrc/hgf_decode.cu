@@ -55,11 +55,11 @@ constexpr int kRedBytes = kDecWarps * 8 * 32 * 4;  // per warp: up to 8 accumula
 constexpr int kOffFlags = kOffRed + kRedBytes;
 constexpr int kOffXq = (kOffFlags + 64 + 127) / 128 * 128;
 constexpr int kSmemLimit = 227 * 1024;
-// Base-3 weights: the decode table sits in front of the activations (four copies of 256 entries of
-// 8 bytes: the first four codes of a byte as four bytes of one word, and its fifth code already
-// moved to the byte position the entry's copy stands for).
-constexpr int kLutBytes = 4 * 256 * 8;
-constexpr int kXqLimit = (kSmemLimit - kOffXq - kLutBytes - kMinSlots * kDecWarps * kSmallSlotTiles * kTileBytes) / 128 * 128;
+// Base-3 weights: the decode table (byte value -> its first four codes, one per byte of a word) is
+// a static shared array with one copy per lane (entry b of lane l at word 32 b + l), so that a warp's
+// 32 look-ups of unrelated bytes never meet in a bank.  A byte's fifth code is found arithmetically.
+constexpr int kLutBytes = 256 * 32 * 4;
+constexpr int kXqLimit = (kSmemLimit - kOffXq - kMinSlots * kDecWarps * kSmallSlotTiles * kTileBytes) / 128 * 128;
 
 constexpr unsigned long long kDecWaitLimitNs = 2000000000ull;  // bounded waits give up after two seconds
 
@@ -69,7 +69,12 @@ int decode_xq_smem_bytes(int M, int K, uint32_t flags) {
     const int Kp = (flags & HGF_FLAG_BASE3) ? (int)padded_k_b3(K) : (int)padded_k(K);
     return (M + (M < 16 ? 1 : 0)) * (Kp + kXqPad);
 }
-int decode_xq_smem_limit() { return kXqLimit; }
+// (With the base-3 table in shared memory a ring of two small slots per warp is accepted, which gives
+// the same limit as three slots without the table.)
+int decode_xq_smem_limit(uint32_t flags) {
+    if (!(flags & HGF_FLAG_BASE3)) return kXqLimit;
+    return (kSmemLimit - kOffXq - kLutBytes - 2 * kDecWarps * kSmallSlotTiles * kTileBytes) / 128 * 128;
+}
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t dsmem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -235,32 +240,30 @@ template <int NT, int ST, bool B3>
 __global__ void __launch_bounds__(kDecThreads, 1)
 decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned int *status) {
     constexpr int kSlotTiles = ST, kSlotBytes = ST * kTileBytes;
-    constexpr int kTileCols = B3 ? 320 : 256, kLut = B3 ? kLutBytes : 0;
+    constexpr int kTileCols = B3 ? 320 : 256;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int slots = L.ring_slots;  // slots of this warp's ring, kSlotBytes each
-    uint8_t *ring = smem + kOffXq + kLut + ((L.xq_smem_bytes + 127) & ~127) + warp * slots * kSlotBytes;
+    uint8_t *ring = smem + kOffXq + ((L.xq_smem_bytes + 127) & ~127) + warp * slots * kSlotBytes;
     const uint32_t ring_u32 = dsmem_u32(ring);
     const uint32_t bars_u32 = dsmem_u32(smem + kOffBars) + warp * kMaxSlots * 8;
     SegSmall *small = reinterpret_cast<SegSmall *>(smem + kOffSmall);
     int *red = reinterpret_cast<int *>(smem + kOffRed);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffFlags);
-    int8_t *xq_s = reinterpret_cast<int8_t *>(smem + kOffXq + kLut);
-    const uint32_t lut_u32 = dsmem_u32(smem + kOffXq);
+    int8_t *xq_s = reinterpret_cast<int8_t *>(smem + kOffXq);
 
     pdl_launch_dependents();
     if (tid == 0) *abort_flag = 0;
-    if (B3) {
-        // copy e of the table, entry b: .x = codes 0..3 of byte value b, one per byte; .y = code 4 in byte e.
+    uint32_t lut_lane = 0;  // shared-window address of this lane's copy of the table
+    if constexpr (B3) {
         // Values above 242 never occur in a packed matrix; they decode as zero weights (code 1).
-        uint2 *lut = reinterpret_cast<uint2 *>(smem + kOffXq);
-        for (int i = tid; i < 4 * 256; i += kDecThreads) {
-            const int e = i >> 8, b = i & 255;
-            uint2 v = make_uint2(0x01010101u, 1u << (8 * e));
-            if (b <= 242) v = make_uint2((uint32_t)(b % 3) | ((uint32_t)(b / 3 % 3) << 8) | ((uint32_t)(b / 9 % 3) << 16) | ((uint32_t)(b / 27 % 3) << 24),
-                                         (uint32_t)(b / 81) << (8 * e));
-            lut[i] = v;
+        __shared__ __align__(128) uint32_t b3_lut[256 * 32];
+        for (int i = tid; i < 256 * 32; i += kDecThreads) {
+            const int b = i >> 5;
+            b3_lut[i] = b <= 242 ? ((uint32_t)(b % 3) | ((uint32_t)(b / 3 % 3) << 8) | ((uint32_t)(b / 9 % 3) << 16) | ((uint32_t)(b / 27 % 3) << 24))
+                                 : 0x01010101u;
         }
+        lut_lane = dsmem_u32(b3_lut) + 4 * lane;
     }
     if (lane == 0) {
         for (int s = 0; s < slots; ++s) dmbar_init(bars_u32 + 8 * s, 1);
@@ -549,19 +552,30 @@ decode_gemv_kernel(const DecodeLaunch L, const DecodeProblem single, unsigned in
                     // table, the first operand of one half of MMA 2 w + e / 2 (four codes), and the fifth codes
                     // of a word's four bytes together make one operand register of MMAs 8 and 9.
                     uint32_t f5g[4], f5h[4];
+                    // fifth codes of a word's four bytes, one per byte: [b >= 81] + [b >= 162], from carries
+                    // into bit 7 of the bytes' low seven bits (no carry crosses a byte: 127 + 94 < 256)
+                    auto fifth = [](uint32_t w) {
+                        const uint32_t u = w & 0x7f7f7f7fu;
+                        const uint32_t ge81 = ((u + 0x2f2f2f2fu) | w) & 0x80808080u;
+                        const uint32_t ge162 = (u + 0x5e5e5e5eu) & w & 0x80808080u;
+                        return (ge81 >> 7) + (ge162 >> 7);
+                    };
+                    auto look_up = [&](uint32_t w, int e) {
+                        // byte e of w, times 128 (the table's stride), plus the lane's base address
+                        const uint32_t idx = (e == 0 ? (w << 7) : (w >> (8 * e - 7))) & 0x7f80u;
+                        uint32_t v;
+                        asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(lut_lane + idx));
+                        return v;
+                    };
 #pragma unroll
                     for (int w = 0; w < 4; ++w) {
                         uint32_t ag[4], ah[4];
-                        f5g[w] = 0u; f5h[w] = 0u;
+                        f5g[w] = fifth(pw[w]);
+                        f5h[w] = fifth(qw[w]);
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            uint2 vg, vh;
-                            const uint32_t a_g = lut_u32 + 2048 * e + (((pw[w] >> (8 * e)) & 0xffu) << 3);
-                            const uint32_t a_h = lut_u32 + 2048 * e + (((qw[w] >> (8 * e)) & 0xffu) << 3);
-                            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(vg.x), "=r"(vg.y) : "r"(a_g));
-                            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(vh.x), "=r"(vh.y) : "r"(a_h));
-                            ag[e] = vg.x; ah[e] = vh.x;
-                            f5g[w] |= vg.y; f5h[w] |= vh.y;
+                            ag[e] = look_up(pw[w], e);
+                            ah[e] = look_up(qw[w], e);
                         }
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt) {
@@ -674,7 +688,7 @@ int decode_grid(int total_tiles) {
 template <int NT, int ST, bool B3>
 static cudaError_t launch_decode_variant(cudaLaunchConfig_t &cfg, const DecodeLaunch &L, const DecodeProblem &sp, unsigned int *status) {
     static std::atomic<unsigned long long> attr_done{0};
-    cudaError_t e = ensure_dynamic_smem(decode_gemv_kernel<NT, ST, B3>, kSmemLimit, attr_done);
+    cudaError_t e = ensure_dynamic_smem(decode_gemv_kernel<NT, ST, B3>, kSmemLimit - (B3 ? kLutBytes : 0), attr_done);
     if (e != cudaSuccess) return e;
     return cudaLaunchKernelEx(&cfg, decode_gemv_kernel<NT, ST, B3>, L, sp, status);
 }
@@ -688,7 +702,7 @@ static cudaError_t launch_decode_layout(cudaLaunchConfig_t &cfg, const DecodeLau
 cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *single, bool pdl, cudaStream_t stream) {
     const int grid = decode_grid(L_in.total_tiles);
     if (grid <= 0) return cudaErrorInvalidDevice;
-    if (L_in.xq_smem_bytes > kXqLimit) return cudaErrorInvalidValue;
+    if (L_in.xq_smem_bytes > decode_xq_smem_limit(single ? single->flags : L_in.flags)) return cudaErrorInvalidValue;
     unsigned int *status = device_status_word();
     if (!status) return cudaErrorMemoryAllocation;
     DecodeLaunch L = L_in;
@@ -709,7 +723,7 @@ cudaError_t launch_decode_gemv(const DecodeLaunch &L_in, const DecodeProblem *si
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kDecThreads);
-    cfg.dynamicSmemBytes = (size_t)(kOffXq + lut + xq_bytes + kDecWarps * slots * slot_bytes);
+    cfg.dynamicSmemBytes = (size_t)(kOffXq + xq_bytes + kDecWarps * slots * slot_bytes);  // (the table is static shared memory)
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
