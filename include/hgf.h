@@ -315,6 +315,15 @@ hgf_status hgf_act_quant(const void *x, int64_t M, int64_t d_in, int8_t *xq, flo
  */
 hgf_status hgf_check_status(void *stream);
 
+/*
+ * Exercises that error path without any fault: enqueues a one-warp kernel whose bounded wait (the
+ * one every role of the GEMM kernel uses, with a limit of `limit_us` microseconds, 1 .. 1000000,
+ * instead of two seconds) sits on a barrier that nothing ever completes.  The wait gives up, records
+ * it and the kernel returns normally; the next hgf_check_status reports HGF_ERR_TIMEOUT once and the
+ * device stays usable.  For tests of the callers' handling of HGF_ERR_TIMEOUT.
+ */
+hgf_status hgf_selftest_wait_timeout(uint32_t limit_us, void *stream);
+
 /* Memory-wall bound of the paper's introduction: T_max = B_mem / (P * b / 8) tokens/s. */
 double hgf_tmax_tokens_per_s(double bmem_bytes_per_s, double params, double bits_per_param);
 

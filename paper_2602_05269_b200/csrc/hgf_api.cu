@@ -552,6 +552,11 @@ extern "C" hgf_status hgf_check_status(void *stream) {
     return HGF_OK;
 }
 
+extern "C" hgf_status hgf_selftest_wait_timeout(uint32_t limit_us, void *stream) {
+    if (limit_us == 0 || limit_us > 1000000u) return HGF_ERR_INVALID_ARG;
+    return launch_wait_timeout_selftest((unsigned long long)limit_us * 1000ull, (cudaStream_t)stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
+}
+
 extern "C" double hgf_tmax_tokens_per_s(double bmem_bytes_per_s, double params, double bits_per_param) {
     return bmem_bytes_per_s / (params * bits_per_param / 8.0);
 }

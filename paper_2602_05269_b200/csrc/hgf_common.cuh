@@ -228,6 +228,7 @@ struct GemmParams {
     uint32_t flags;
 };
 cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream);
+cudaError_t launch_wait_timeout_selftest(unsigned long long limit_ns, cudaStream_t stream);
 
 // ---- small device helpers ---------------------------------------------------------------------
 __device__ __forceinline__ float bf16lo_to_float(uint32_t w) { return __uint_as_float(w << 16); }

@@ -114,7 +114,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 // this kernel share the SM's schedulers and its shared-memory pipe, and warps that poll without a
 // pause slow the ones that have work.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          unsigned int *status, unsigned int code) {
+                                          unsigned int *status, unsigned int code, unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;
     unsigned int ns = 20;
@@ -126,7 +126,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const unsigned long long now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) break;
+            else if (now - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;
@@ -597,6 +597,29 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
+}
+
+// The bounded wait on a barrier that nothing completes: it gives up after `limit_ns`, records that
+// in the status word and the kernel returns (the error path of every role above, exercised alone).
+__global__ void wait_timeout_selftest_kernel(unsigned long long limit_ns, unsigned int *status) {
+    __shared__ __align__(8) unsigned long long bar_mem;
+    __shared__ int abort_mem;
+    const uint32_t bar = smem_u32(&bar_mem);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        abort_mem = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_wait(bar, 0u, &abort_mem, status, 0x700u, limit_ns);
+}
+
+cudaError_t launch_wait_timeout_selftest(unsigned long long limit_ns, cudaStream_t stream) {
+    unsigned int *status = device_status_word();
+    if (!status) return cudaErrorMemoryAllocation;
+    wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(limit_ns, status);
+    count_launch();
+    return cudaGetLastError();
 }
 
 // ---- host side: tensor maps and launch -----------------------------------------------------------

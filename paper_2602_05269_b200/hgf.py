@@ -29,7 +29,8 @@ EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_wo
            "hgf_launch_count", "hgf_status_string", "hgf_group_create", "hgf_group_forward",
            "hgf_group_destroy", "hgf_group_forward_phases", "hgf_linear_forward_static", "hgf_group_debug",
            "hgf_linear_forward_phases", "hgf_linear_forward_ln",
-           "hgf_packed_bytes_b3", "hgf_pack_ternary_b3", "hgf_unpack_ternary_b3"]
+           "hgf_packed_bytes_b3", "hgf_pack_ternary_b3", "hgf_unpack_ternary_b3",
+           "hgf_selftest_wait_timeout"]
 
 
 class HgfError(RuntimeError):
@@ -95,6 +96,8 @@ def lib() -> ctypes.CDLL:
         L.hgf_linear_forward_static.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, u32, vp]
         L.hgf_act_quant.restype = c.c_int
         L.hgf_act_quant.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+        L.hgf_selftest_wait_timeout.restype = c.c_int
+        L.hgf_selftest_wait_timeout.argtypes = [u32, vp]
         L.hgf_check_status.restype = c.c_int
         L.hgf_check_status.argtypes = [vp]
         L.hgf_tmax_tokens_per_s.restype = c.c_double
@@ -303,6 +306,11 @@ class Group:
 def check_status(stream=None) -> None:
     """Synchronise and raise if a bounded device-side wait gave up since the last check."""
     _check("hgf_check_status", lib().hgf_check_status(_stream(stream)))
+
+
+def selftest_wait_timeout(limit_us: int = 200, stream=None) -> None:
+    """Enqueue the kernel whose bounded wait runs out (hgf_selftest_wait_timeout); the next check_status raises."""
+    _check("hgf_selftest_wait_timeout", lib().hgf_selftest_wait_timeout(int(limit_us), _stream(stream)))
 
 
 def tmax_tokens_per_s(bmem_bytes_per_s: float, params: float, bits: float) -> float:

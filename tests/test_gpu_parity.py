@@ -459,3 +459,16 @@ def test_the_two_launches_of_a_layer_call_separately(hgf, M, K, N, r):
         hgf.check_status()
         # the whole call above also asked for H, which changes the summation order of x A on the decode path
         assert (y - y_whole).abs().max().item() <= 2e-6 * y_whole.abs().max().item()
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_device_stays_usable(hgf):
+    """The error path of the device-side waits, without any fault: a kernel waits (bounded, 200 us) on a
+    barrier that nothing completes, gives up and returns; the status check reports it once; the
+    next layer call on the same context is correct."""
+    hgf.check_status()
+    hgf.selftest_wait_timeout(200)
+    with pytest.raises(hgf.HgfError) as e:
+        hgf.check_status()
+    assert e.value.status == 6
+    hgf.check_status()                      # reported once, then clear
+    check_layer(hgf, syn.LayerShape("after", 256, 256, 16), 40, config=22, tol2=TOL_GEMM)
