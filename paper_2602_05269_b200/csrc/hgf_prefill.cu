@@ -15,12 +15,14 @@
 // 256 input columns (eight MMAs): every hand-over between the roles costs a shared-memory round
 // trip, and the single MMA-issuing thread can only afford one per 512 tensor-core clocks.
 //
-// One persistent CTA per SM, 11 warps with fixed roles:
+// One persistent CTA per SM, 12 warps with fixed roles:
 //   warp 0      producer (all lanes): per stage the int8 activation tile as two 128 tokens x 128 B
 //               boxes (128-byte swizzle) and the packed weights of 128 channels (eight contiguous
 //               1 KiB tiles of the tiled weight layout, one bulk copy each); per tile what its
 //               epilogue needs: row sums, scales, the H tile and the (g B)^T tile
-//   warp 1      allocates tensor memory; one lane issues the MMAs and commits to mbarriers
+//   warp 1      allocates tensor memory; one lane issues the MMAs of every other pipeline stage (and the
+//               correction MMAs) and commits to mbarriers
+//   warp 11     one lane issues the MMAs of the stages in between
 //   warps 2-5   epilogue: dequantise the accumulator in place (tcgen05.ld / tcgen05.st), wait for
 //               the correction MMA, read the result, transpose it through shared memory and store
 //               y with TMA
@@ -47,7 +49,7 @@ constexpr int X_TILE_BYTES = 2 * X_HALF_BYTES;   // 32 KiB per stage
 constexpr int P_TILE_BYTES = TILE_C * KBLK / 4;  // 8 KiB: 8 weight tiles of 16 rows x 256 columns
 constexpr int TOKV_BYTES = TILE_T * 8;           // row sums and scales of the tile's tokens
 constexpr int STORE_BUF_BYTES = 32 * 32 * 4;     // per epilogue warp: 32 tokens x 32 channels
-constexpr int GEMM_THREADS = 352;  // 11 warps
+constexpr int GEMM_THREADS = 384;  // 12 warps
 // tensor memory: two accumulators of 128 columns, then one weight operand of 64 columns (= 256 int8 per lane) per stage
 constexpr int TMEM_COLS = 512, ACC_COLS = TILE_T, A_COL = 2 * ACC_COLS, A_STAGE_COLS = KBLK / 4;
 
@@ -72,7 +74,8 @@ struct Cfg {
     static constexpr int BAR_FULL = 0, BAR_EMPTY = BAR_FULL + NS, BAR_PFULL = BAR_EMPTY + NS, BAR_PEMPTY = BAR_PFULL + PSTAGES,
                          BAR_ACCFULL = BAR_PEMPTY + PSTAGES,
                          BAR_ACCEMPTY = BAR_ACCFULL + 2, BAR_LORAREADY = BAR_ACCEMPTY + 2, BAR_LORADONE = BAR_LORAREADY + 2,
-                         BAR_OPSFULL = BAR_LORADONE + 2, BAR_OPSEMPTY = BAR_OPSFULL + 2, BAR_COUNT = BAR_OPSEMPTY + 2;
+                         BAR_OPSFULL = BAR_LORADONE + 2, BAR_OPSEMPTY = BAR_OPSFULL + 2, BAR_TURN = BAR_OPSEMPTY + 2,
+                         BAR_COUNT = BAR_TURN + 2;
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
     static_assert(BAR_COUNT * 8 + 16 <= 512, "barrier block too small");
     static_assert(A_COL + NS * A_STAGE_COLS <= TMEM_COLS, "tensor memory budget");
@@ -274,7 +277,8 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             mbar_init(bar(C::BAR_PEMPTY + j), 4);
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(bar(C::BAR_ACCFULL + b), 1);
+            mbar_init(bar(C::BAR_ACCFULL + b), 2);  // one commit from each of the two MMA-issuing threads
+            mbar_init(bar(C::BAR_TURN + b), 1);
             mbar_init(bar(C::BAR_ACCEMPTY + b), 4);
             mbar_init(bar(C::BAR_LORAREADY + b), 4);
             mbar_init(bar(C::BAR_LORADONE + b), 1);
@@ -356,17 +360,28 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar(C::BAR_OPSFULL + q), par); ++i) {}
                 }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == 11) {
+        // ------------------------------------------------------------------ MMA issuers
         // Tile `it` accumulates into accumulator it % 2, so the epilogue of one tile runs under the main
         // loop of the next.  With a correction, the epilogue first rewrites the accumulator as fp32
-        // (dequantised), then this thread adds (g B) H^T onto it with one more MMA, slipped in between
+        // (dequantised), then the first issuer adds (g B) H^T onto it with one more MMA, slipped in between
         // the k blocks of the tile in progress as soon as the epilogue is ready for it.
+        //
+        // TWO threads issue the integer MMAs, in turns: the stages are numbered through the whole tile
+        // sequence and warp 1 takes the even ones, warp 11 the odd ones.  The tensor pipe holds hardly any
+        // MMA in reserve and takes a 128 x 128 x 32 one about as fast as it executes it (64 clocks), so with
+        // a single issuing thread it idles while that thread waits on barriers, commits and keeps its
+        // books - about as long per stage as the stage's eight MMAs run.  Here one thread does all that
+        // for its next stage while the other's MMAs run, and only the hand-over itself is exposed.  Order
+        // between the two threads' MMAs on the shared accumulator is established the documented way: after
+        // its stage a thread executes tcgen05.fence::before_thread_sync and arrives on the other's TURN
+        // barrier; the other waits there and executes tcgen05.fence::after_thread_sync before its first MMA.
+        // Each thread commits the stages it issued (EMPTY) and, at the end of a tile, ACCFULL (two arrivals).
+        const int half = warp == 1 ? 0 : 1;
         if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
             bool ok = true;
-            int it = 0, pend = -1;  // pend: tile whose correction MMA is still to be issued
+            int it = 0, pend = -1;  // pend: tile whose correction MMA is still to be issued (first issuer only)
+            int gs = 0;             // stage number, counted through all tiles of this CTA
             const uint64_t xdesc0 = make_sw128_desc(sbase + C::OFF_X);
             auto issue_lora = [&](int t) {
                 const int b = t & 1;
@@ -382,15 +397,24 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
                 const int b = it & 1;
                 const uint32_t acc = tmem_base + b * ACC_COLS;
-                if (it >= 2 && !(ok = mbar_wait(bar(C::BAR_ACCEMPTY + b), (uint32_t)((it >> 1) - 1) & 1u, abort_flag, status, 0x200u)))
-                    break;
-                tc_fence_after();
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (pend >= 0 && mbar_try_wait(bar(C::BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u)) {
+                bool acc_mine = false;  // this thread has waited for the accumulator's release
+                for (int kb = 0; kb < kblocks; ++kb, ++gs) {
+                    if ((gs & 1) != half) continue;
+                    if (!acc_mine) {
+                        if (it >= 2 && !(ok = mbar_wait(bar(C::BAR_ACCEMPTY + b), (uint32_t)((it >> 1) - 1) & 1u, abort_flag, status, 0x200u)))
+                            break;
+                        acc_mine = true;
+                    }
+                    if (half == 0 && pend >= 0 && mbar_try_wait(bar(C::BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u)) {
                         issue_lora(pend);
                         pend = -1;
                     }
+                    const int s = gs % C::STAGES;
+                    const uint32_t ph = (uint32_t)(gs / C::STAGES) & 1u;
                     if (!(ok = mbar_wait(bar(C::BAR_FULL + s), ph, abort_flag, status, 0x210u + s))) break;
+                    // the other thread has issued stage gs - 1
+                    if (gs > 0 && !(ok = mbar_wait(bar(C::BAR_TURN + half), (uint32_t)((gs - 1) >> 1) & 1u, abort_flag, status, 0x240u + half)))
+                        break;
                     tc_fence_after();
                     const uint64_t bdesc = xdesc0 + (uint64_t)(s * (X_TILE_BYTES >> 4));
                     const uint32_t a_tmem = tmem_base + A_COL + s * A_STAGE_COLS;
@@ -404,11 +428,13 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     mma_i8_ts(acc, a_tmem + 40u, bdesc + (X_HALF_BYTES >> 4) + 2u, IDESC_I8, 1u);
                     mma_i8_ts(acc, a_tmem + 48u, bdesc + (X_HALF_BYTES >> 4) + 4u, IDESC_I8, 1u);
                     mma_i8_ts(acc, a_tmem + 56u, bdesc + (X_HALF_BYTES >> 4) + 6u, IDESC_I8, 1u);
+                    tc_fence_before();
+                    mbar_arrive(bar(C::BAR_TURN + (half ^ 1)));  // the other thread's turn
                     tc_commit(bar(C::BAR_EMPTY + s));
-                    if (++s == C::STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
                 tc_commit(bar(C::BAR_ACCFULL + b));
+                if (half != 0) continue;
                 if (pend >= 0) {  // the previous tile's correction has to be out before its accumulator's next turn
                     if (!(ok = mbar_wait(bar(C::BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x230u)))
                         break;
@@ -417,7 +443,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
                 if (has_lora) pend = it;
             }
-            if (ok && pend >= 0 &&
+            if (half == 0 && ok && pend >= 0 &&
                 mbar_wait(bar(C::BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x231u))
                 issue_lora(pend);
         }
