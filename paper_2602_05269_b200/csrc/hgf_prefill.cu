@@ -15,7 +15,7 @@
 // 256 input columns (eight MMAs): every hand-over between the roles costs a shared-memory round
 // trip, and the single MMA-issuing thread can only afford one per 512 tensor-core clocks.
 //
-// One persistent CTA per SM, 12 warps with fixed roles:
+// One persistent CTA per SM, 16 warps with fixed roles:
 //   warp 0      producer (all lanes): per stage the int8 activation tile as two 128 tokens x 128 B
 //               boxes (128-byte swizzle) and the packed weights of 128 channels (eight contiguous
 //               1 KiB tiles of the tiled weight layout, one bulk copy each); per tile what its
@@ -23,9 +23,10 @@
 //   warp 1      allocates tensor memory; one lane issues the MMAs of every other pipeline stage (and the
 //               correction MMAs) and commits to mbarriers
 //   warp 11     one lane issues the MMAs of the stages in between
-//   warps 2-5   epilogue: dequantise the accumulator in place (tcgen05.ld / tcgen05.st), wait for
-//               the correction MMA, read the result, transpose it through shared memory and store
-//               y with TMA
+//   warps 2-5, 12-15  epilogue, two warps per tensor-memory lane quarter (32 channels), one for each
+//               half of the tile's tokens: dequantise the accumulator in place (tcgen05.ld /
+//               tcgen05.st), wait for the correction MMA, read the result, transpose it through shared
+//               memory and store y with TMA
 //   warps 6-9   expand the packed tile into tensor memory
 //   warp 10     producer of the packed codes (eight contiguous 1 KiB tiles of the tiled weight layout
 //               per stage, one bulk copy each), in a ring that runs ahead of the activations'
@@ -48,8 +49,8 @@ constexpr int X_HALF_BYTES = TILE_T * 128;       // 16 KiB: 128 tokens x 128 col
 constexpr int X_TILE_BYTES = 2 * X_HALF_BYTES;   // 32 KiB per stage
 constexpr int P_TILE_BYTES = TILE_C * KBLK / 4;  // 8 KiB: 8 weight tiles of 16 rows x 256 columns
 constexpr int TOKV_BYTES = TILE_T * 8;           // row sums and scales of the tile's tokens
-constexpr int STORE_BUF_BYTES = 32 * 32 * 4;     // per epilogue warp: 32 tokens x 32 channels
-constexpr int GEMM_THREADS = 384;  // 12 warps
+constexpr int STORE_BUF_BYTES = 2048;            // per epilogue warp: 32 channels x 32 tokens (bf16) or x 16 tokens (fp32)
+constexpr int GEMM_THREADS = 512;  // 16 warps
 // tensor memory: two accumulators of 128 columns, then one weight operand of 64 columns (= 256 int8 per lane) per stage
 constexpr int TMEM_COLS = 512, ACC_COLS = TILE_T, A_COL = 2 * ACC_COLS, A_STAGE_COLS = KBLK / 4;
 
@@ -68,7 +69,7 @@ struct Cfg {
     static constexpr int OFF_P = OFF_LB + 2 * LORA_B_BYTES;
     static constexpr int OFF_TOKV = OFF_P + PSTAGES * P_TILE_BYTES;
     static constexpr int OFF_ST = OFF_TOKV + 2 * TOKV_BYTES;
-    static constexpr int OFF_BAR = OFF_ST + 4 * STORE_BUF_BYTES;
+    static constexpr int OFF_BAR = OFF_ST + 8 * STORE_BUF_BYTES;
     static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;  // + slack for the 1024-byte alignment of the base
     // barrier slots (8 bytes each) inside the OFF_BAR block
     static constexpr int BAR_FULL = 0, BAR_EMPTY = BAR_FULL + NS, BAR_PFULL = BAR_EMPTY + NS, BAR_PEMPTY = BAR_PFULL + PSTAGES,
@@ -107,6 +108,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// The same test without the hardware's suspend interval: returns at once.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
@@ -130,6 +143,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             const unsigned long long now = global_timer_ns();
             if (t0 == 0) t0 = now;
             else if (now - t0 > limit_ns) break;
+        }
+    }
+    *abort_flag = 1;
+    atomicExch(status, code);
+    return false;
+}
+
+// The same bound, but polling without a pause: for the hand-over between the two MMA-issuing threads,
+// where every clock of wake-up delay is a clock the tensor pipe idles (one thread polls, briefly).
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                               unsigned int *status, unsigned int code) {
+    unsigned long long t0 = 0;
+    for (uint32_t i = 0; i < (kSpinLimit << 4); ++i) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
         }
     }
     *abort_flag = 1;
@@ -190,6 +222,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
 }
@@ -279,11 +320,11 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(C::BAR_ACCFULL + b), 2);  // one commit from each of the two MMA-issuing threads
             mbar_init(bar(C::BAR_TURN + b), 1);
-            mbar_init(bar(C::BAR_ACCEMPTY + b), 4);
-            mbar_init(bar(C::BAR_LORAREADY + b), 4);
+            mbar_init(bar(C::BAR_ACCEMPTY + b), 8);
+            mbar_init(bar(C::BAR_LORAREADY + b), 8);
             mbar_init(bar(C::BAR_LORADONE + b), 1);
             mbar_init(bar(C::BAR_OPSFULL + b), 1);
-            mbar_init(bar(C::BAR_OPSEMPTY + b), 4);
+            mbar_init(bar(C::BAR_OPSEMPTY + b), 8);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -413,7 +454,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint32_t ph = (uint32_t)(gs / C::STAGES) & 1u;
                     if (!(ok = mbar_wait(bar(C::BAR_FULL + s), ph, abort_flag, status, 0x210u + s))) break;
                     // the other thread has issued stage gs - 1
-                    if (gs > 0 && !(ok = mbar_wait(bar(C::BAR_TURN + half), (uint32_t)((gs - 1) >> 1) & 1u, abort_flag, status, 0x240u + half)))
+                    if (gs > 0 && !(ok = mbar_wait_spin(bar(C::BAR_TURN + half), (uint32_t)((gs - 1) >> 1) & 1u, abort_flag, status, 0x240u + half)))
                         break;
                     tc_fence_after();
                     const uint64_t bdesc = xdesc0 + (uint64_t)(s * (X_TILE_BYTES >> 4));
@@ -447,11 +488,16 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 mbar_wait(bar(C::BAR_LORAREADY + (pend & 1)), (uint32_t)(pend >> 1) & 1u, abort_flag, status, 0x231u))
                 issue_lora(pend);
         }
-    } else if (warp < 6) {
+    } else if (warp < 6 || warp >= 12) {
         // ------------------------------------------------------------------ epilogue warps
-        const int e = warp - 2;          // staging role index
-        const int q = warp & 3;          // tensor-memory lane quarter this warp may access
-        uint8_t *buf = smem + C::OFF_ST + e * STORE_BUF_BYTES;
+        // Eight of them: the warp pair of a tensor-memory lane quarter (32 output channels) shares the
+        // tile's 128 tokens, 64 each, so a tile's epilogue takes half as long as with one warp per
+        // quarter - with the two issuing threads the main loop of a short-K tile is over sooner than that.
+        const int e2 = warp < 6 ? 0 : 1;                  // which 64 tokens of the tile
+        const int q = warp & 3;                           // tensor-memory lane quarter this warp may access
+        constexpr int HALF_T = TILE_T / 2;
+        constexpr int W = OUT_BF16 ? 32 : 16;             // tokens per staging step (2 KiB of staging either way)
+        uint8_t *buf = smem + C::OFF_ST + (4 * e2 + q) * STORE_BUF_BYTES;
         bool ok = true;
         int it = 0;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
@@ -472,16 +518,18 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             tc_fence_after();
             const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16) + b * ACC_COLS;
 
+            // int32 sums -> fp32 (Y_int - row sum) * scale, for the WN tokens from cc on
             // (the per-token values are read as vectors ahead of the arithmetic: a shared-memory load per
             // element in the dependent chain costs its full latency every time)
-            auto dequant_chunk = [&](int cc, uint32_t (&ai)[32]) {  // int32 sums -> fp32 (Y_int - row sum) * scale
+            auto dequant_chunk = [&](int cc, auto &ai) {
+                constexpr int WN = (int)(sizeof(ai) / sizeof(uint32_t));
                 if (p.dbg_y_int && n_ok) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
+                    for (int j = 0; j < WN; ++j)
                         if (t0 + cc + j < p.M) p.dbg_y_int[(size_t)(t0 + cc + j) * p.N + n] = (int)ai[j] - tok_rs[cc + j];
                 }
 #pragma unroll
-                for (int v = 0; v < 8; ++v) {
+                for (int v = 0; v < WN / 4; ++v) {
                     const int4 rs4 = *reinterpret_cast<const int4 *>(tok_rs + cc + 4 * v);
                     const float4 sc4 = *reinterpret_cast<const float4 *>(tok_sc + cc + 4 * v);
                     ai[4 * v + 0] = __float_as_uint((float)((int)ai[4 * v + 0] - rs4.x) * sc4.x);
@@ -492,7 +540,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             };
             if (has_lora) {
                 // first pass: dequantise in place (int32 -> fp32), then let the MMA warp add the correction
-                for (int cc = 0; cc < TILE_T; cc += 32) {
+                for (int cc = HALF_T * e2; cc < HALF_T * (e2 + 1); cc += 32) {
                     uint32_t ai[32];
                     tmem_ld32(lane_base + cc, ai);
                     tmem_ld_wait();
@@ -508,11 +556,11 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 tc_fence_after();
             }
 
-            // read the result, transpose it through shared memory (a thread holds one channel of 32
+            // read the result, transpose it through shared memory (a thread holds one channel of W
             // tokens; y wants the channels of a token next to each other) and store with TMA
-            for (int cc = 0; cc < TILE_T; cc += 32) {
-                uint32_t ai[32];
-                tmem_ld32(lane_base + cc, ai);
+            for (int cc = HALF_T * e2; cc < HALF_T * (e2 + 1); cc += W) {
+                uint32_t ai[W];
+                if constexpr (W == 32) tmem_ld32(lane_base + cc, ai); else tmem_ld16(lane_base + cc, ai);
                 tmem_ld_wait();
                 if (!has_lora) dequant_chunk(cc, ai);
                 // the buffer was handed to a TMA store one chunk ago: wait until it was read
@@ -520,11 +568,11 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 __syncwarp();
                 if (OUT_BF16) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
+                    for (int j = 0; j < W; ++j)
                         reinterpret_cast<__nv_bfloat16 *>(buf)[j * 32 + lane] = __float2bfloat16_rn(__uint_as_float(ai[j]));
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) reinterpret_cast<uint32_t *>(buf)[j * 32 + lane] = ai[j];
+                    for (int j = 0; j < W; ++j) reinterpret_cast<uint32_t *>(buf)[j * 32 + lane] = ai[j];
                 }
                 fence_proxy_async();
                 __syncwarp();
@@ -533,7 +581,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     bulk_commit();
                 }
             }
-            // all tensor-memory reads of this tile are done: hand the accumulator back to the MMA warp
+            // all tensor-memory reads of this tile are done: hand the accumulator back to the MMA warps
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
@@ -721,7 +769,7 @@ cudaError_t launch_prefill_gemm(const GemmParams &p, cudaStream_t stream) {
         mgb = mx;
     }
     if (!make_map_2d(&my, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, p.y, (uint64_t)p.N,
-                     (uint64_t)p.M, (uint64_t)p.N * (bf16 ? 2 : 4), 32, 32, CU_TENSOR_MAP_SWIZZLE_NONE))
+                     (uint64_t)p.M, (uint64_t)p.N * (bf16 ? 2 : 4), 32, bf16 ? 32 : 16, CU_TENSOR_MAP_SWIZZLE_NONE))
         return cudaErrorInvalidValue;
     const int tiles = ((p.M + TILE_T - 1) / TILE_T) * ((p.N + TILE_C - 1) / TILE_C);
     const int grid = tiles < sm_count ? tiles : sm_count;
