@@ -281,6 +281,18 @@ typedef struct hgf_group hgf_group;
 
 hgf_status hgf_group_create(const hgf_problem *problems /* host array */, int32_t n, uint32_t flags,
                             hgf_group **out);
+/*
+ * The same with a front end per problem (front_ends: host array of n entries, or null for none):
+ * the LayerNorm in front of the quantiser and the gate granularity of hgf_linear_forward_ln.  This is
+ * the paper's attention block in one group (Appendix E, HeadAdaptiveDiffAttention): Q, K and V are
+ * three HGF layers of the same x, each behind a LayerNorm of its own, with one gate per head.
+ * Problems on the same x share a quantisation only if they also name the same LayerNorm parameters.
+ * The parameter arrays are kept by pointer, like the other tensors; mean_out / rstd_out, if given,
+ * are written by every forward.
+ */
+hgf_status hgf_group_create_ln(const hgf_problem *problems /* host array */,
+                               const hgf_front_end *front_ends /* host array, nullable */, int32_t n,
+                               uint32_t flags, hgf_group **out);
 hgf_status hgf_group_forward(hgf_group *group, void *stream);
 /*
  * The two launches of hgf_group_forward separately, for measurement: HGF_PHASE_PROLOGUE runs

@@ -187,6 +187,29 @@ extern "C" hgf_status hgf_linear_forward_ln(const void *x, int64_t M, const void
                         HGF_PHASE_PROLOGUE | HGF_PHASE_GEMV, stream_);
 }
 
+// Validates a front-end description (nullable) and turns it into the kernels' form.
+static hgf_status parse_front_end(const hgf_front_end *fe_in, int64_t d_out, bool *ln, int *gate_group, FrontEnd *fe) {
+    *ln = false;
+    *gate_group = 1;
+    *fe = FrontEnd{};
+    if (!fe_in) return HGF_OK;
+    if ((fe_in->ln_weight == nullptr) != (fe_in->ln_bias == nullptr) || !(fe_in->eps >= 0.0f)) return HGF_ERR_INVALID_ARG;
+    if ((((uintptr_t)fe_in->ln_weight) | ((uintptr_t)fe_in->ln_bias)) & 15u) return HGF_ERR_MISALIGNED;
+    if (fe_in->gate_group < 0) return HGF_ERR_INVALID_ARG;
+    if (fe_in->gate_group > 1) {
+        if (fe_in->gate_group >= d_out) *gate_group = (int)((d_out + 15) / 16 * 16);  // scalar gate: one group holds every row tile
+        else if (fe_in->gate_group % 16 == 0) *gate_group = (int)fe_in->gate_group;
+        else return HGF_ERR_UNSUPPORTED_SHAPE;
+    }
+    *ln = fe_in->ln_weight != nullptr;
+    fe->ln_w = fe_in->ln_weight;
+    fe->ln_b = fe_in->ln_bias;
+    fe->dbg_mean = fe_in->mean_out;
+    fe->dbg_rstd = fe_in->rstd_out;
+    fe->eps = fe_in->eps;
+    return HGF_OK;
+}
+
 hgf_status hgf::forward_impl(const void *x, int64_t M, const void *packed, float gamma, int64_t d_in, int64_t d_out,
                                     const void *At, const void *Bt, int32_t r, const float *gate, void *y, void *workspace,
                                     size_t workspace_bytes, const hgf_debug_out *dbg, const hgf_front_end *fe_in, uint32_t flags,
@@ -208,21 +231,9 @@ hgf_status hgf::forward_impl(const void *x, int64_t M, const void *packed, float
     bool ln = false;
     int gate_group = 1;
     FrontEnd fe = {};
-    if (fe_in) {
-        if ((fe_in->ln_weight == nullptr) != (fe_in->ln_bias == nullptr) || !(fe_in->eps >= 0.0f)) return HGF_ERR_INVALID_ARG;
-        if (misaligned(fe_in->ln_weight) || misaligned(fe_in->ln_bias)) return HGF_ERR_MISALIGNED;
-        if (fe_in->gate_group < 0) return HGF_ERR_INVALID_ARG;
-        if (fe_in->gate_group > 1) {
-            if (fe_in->gate_group >= d_out) gate_group = (int)((d_out + 15) / 16 * 16);  // scalar gate: one group holds every row tile
-            else if (fe_in->gate_group % 16 == 0) gate_group = (int)fe_in->gate_group;
-            else return HGF_ERR_UNSUPPORTED_SHAPE;
-        }
-        ln = fe_in->ln_weight != nullptr;
-        fe.ln_w = fe_in->ln_weight;
-        fe.ln_b = fe_in->ln_bias;
-        fe.dbg_mean = fe_in->mean_out;
-        fe.dbg_rstd = fe_in->rstd_out;
-        fe.eps = fe_in->eps;
+    {
+        hgf_status fst = parse_front_end(fe_in, d_out, &ln, &gate_group, &fe);
+        if (fst != HGF_OK) return fst;
     }
 
     PrologueParams pp;
@@ -338,6 +349,11 @@ struct hgf_group {
 };
 
 extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, uint32_t flags, hgf_group **out) {
+    return hgf_group_create_ln(problems, nullptr, n, flags, out);
+}
+
+extern "C" hgf_status hgf_group_create_ln(const hgf_problem *problems, const hgf_front_end *front_ends, int32_t n, uint32_t flags,
+                                          hgf_group **out) {
     if (!problems || !out || n <= 0 || n > 65536) return HGF_ERR_INVALID_ARG;
     if (flags & HGF_FLAG_FORCE_GEMM) return HGF_ERR_INVALID_ARG;
     *out = nullptr;
@@ -347,6 +363,9 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
     std::vector<LoraItem> litems;
     std::vector<WsLayout> lay((size_t)n);
     std::vector<int32_t> ranks((size_t)n);
+    std::vector<FrontEnd> fes((size_t)n);
+    std::vector<int> gate_groups((size_t)n, 1);
+    std::vector<char> lns((size_t)n, 0);
     size_t ws_total = 0;
     int tiles = 0, max_M = 0, xq_smem = 0;
     long long cost = 0;
@@ -358,6 +377,12 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         hgf_status st = validate_problem(q.x, q.M, q.packed, q.d_in, q.d_out, q.At, q.Bt, q.r, q.gate, q.y, flags, &r, &gemm);
         if (st != HGF_OK) return st;
         if (gemm) return HGF_ERR_UNSUPPORTED_SHAPE;  // groups hold decode-sized problems only
+        {
+            bool ln = false;
+            st = parse_front_end(front_ends ? front_ends + i : nullptr, q.d_out, &ln, &gate_groups[i], &fes[i]);
+            if (st != HGF_OK) return st;
+            lns[i] = ln ? 1 : 0;
+        }
         ranks[i] = r;
         lay[i] = ws_layout(q.M, q.d_in, q.d_out, r, false);
         ws_total += lay[i].total;
@@ -394,13 +419,19 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
         ws += lay[i].total;
         dps[i].tile_begin = tiles;
         dps[i].cost_begin = cost;
+        dps[i].gate_group = gate_groups[i];
         // problems on the same input (Q, K and V of an attention block; the two up-projections of its
         // MLP) share one quantisation: a later one reads the first one's x~, scales and row sums
         int first = i;
         {
             auto seen = first_with_x.find(q.x);
+            // (projections behind LayerNorms of their own - the paper's Q, K and V each have one - are
+            // quantised separately unless they name the same parameters)
             if (seen == first_with_x.end()) first_with_x.emplace(q.x, i);
-            else if (problems[seen->second].M == q.M && problems[seen->second].d_in == q.d_in) first = seen->second;
+            else if (problems[seen->second].M == q.M && problems[seen->second].d_in == q.d_in &&
+                     fes[seen->second].ln_w == fes[i].ln_w && fes[seen->second].ln_b == fes[i].ln_b &&
+                     (!lns[i] || fes[seen->second].eps == fes[i].eps))
+                first = seen->second;
         }
         if (first != i) {
             pps[i].xq = pps[first].xq;
@@ -415,8 +446,19 @@ extern "C" hgf_status hgf_group_create(const hgf_problem *problems, int32_t n, u
             dps[i].hpart = jts ? hpart : nullptr;
             dps[i].nslices = jts ? slices : 0;
             for (int m = 0; first == i && m < (int)q.M; ++m) {
-                QuantItem qi = {pps[i].x + (size_t)m * q.d_in, pps[i].xq + (size_t)m * q.d_in, pps[i].gamma_x + m,
-                                pps[i].row_sum + m, (int)q.d_in, 0};
+                QuantItem qi = {};
+                qi.x = pps[i].x + (size_t)m * q.d_in;
+                qi.xq = pps[i].xq + (size_t)m * q.d_in;
+                qi.gamma_x = pps[i].gamma_x + m;
+                qi.row_sum = pps[i].row_sum + m;
+                qi.K = (int)q.d_in;
+                if (lns[i]) {
+                    qi.eps = fes[i].eps;
+                    qi.ln_w = fes[i].ln_w;
+                    qi.ln_b = fes[i].ln_b;
+                    qi.mean_out = fes[i].dbg_mean ? fes[i].dbg_mean + m : nullptr;
+                    qi.rstd_out = fes[i].dbg_rstd ? fes[i].dbg_rstd + m : nullptr;
+                }
                 qitems.push_back(qi);
             }
             for (int sl = 0; sl < slices; ++sl)      // slice-major: neighbouring warps share x

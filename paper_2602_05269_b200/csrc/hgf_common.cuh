@@ -199,7 +199,10 @@ struct QuantItem {
     int8_t *xq;                // its quantised row
     float *gamma_x;            // its scale
     int32_t *row_sum;          // its sum of quantised values
-    int K, pad;
+    int K;
+    float eps;                 // LayerNorm front end (ln_w non-null): normalise the row before quantising it
+    const float *ln_w, *ln_b;  // [K] each, or null
+    float *mean_out, *rstd_out;  // nullable: where this row's statistics go
 };
 __host__ __device__ inline int prologue_slice_k(int max_M) { return max_M <= 8 ? 512 : 256; }
 cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_quant,

@@ -512,6 +512,79 @@ __device__ void warp_quant_row(const QuantItem &q, uint32_t buf_u32, const uint8
     }
 }
 
+// The same for a row behind the LayerNorm front end (Appendix E of the paper): statistics in two passes
+// summed in double, the largest |xn|, then the codes - the arithmetic of quant_row_ln, one warp per
+// row, each pass reading the row from L1 / L2.
+__device__ void warp_quant_row_ln(const QuantItem &q, int lane) {
+    const int K = q.K, nv = K / 8;
+    const uint4 *xv = reinterpret_cast<const uint4 *>(q.x);
+    float f[8];
+    double sum = 0.0;
+    for (int i = lane; i < nv; i += 32) {
+        unpack8(xv[i], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sum += (double)f[e];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const double mean_d = sum / (double)K;
+    double ss = 0.0;
+    for (int i = lane; i < nv; i += 32) {
+        unpack8(xv[i], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const double d = (double)f[e] - mean_d;
+            ss += d * d;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const float mean = (float)mean_d, rstd = (float)(1.0 / sqrt(ss / (double)K + (double)q.eps));
+    auto load_wb = [&](int i, float (&w)[8], float (&b)[8]) {
+        const float4 w0 = *reinterpret_cast<const float4 *>(q.ln_w + 8 * i), w1 = *reinterpret_cast<const float4 *>(q.ln_w + 8 * i + 4);
+        const float4 b0 = *reinterpret_cast<const float4 *>(q.ln_b + 8 * i), b1 = *reinterpret_cast<const float4 *>(q.ln_b + 8 * i + 4);
+        w[0] = w0.x; w[1] = w0.y; w[2] = w0.z; w[3] = w0.w; w[4] = w1.x; w[5] = w1.y; w[6] = w1.z; w[7] = w1.w;
+        b[0] = b0.x; b[1] = b0.y; b[2] = b0.z; b[3] = b0.w; b[4] = b1.x; b[5] = b1.y; b[6] = b1.z; b[7] = b1.w;
+    };
+    float amax = 0.0f, w[8], b[8];
+    for (int i = lane; i < nv; i += 32) {
+        unpack8(xv[i], f);
+        load_wb(i, w, b);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(ln_value(f[e], mean, rstd, w[e], b[e])));
+    }
+    const float g = fmaxf(warp_max(amax), 1e-5f);
+    const float scale = __fdiv_rn(127.0f, g);
+    int sum_q = 0;
+    uint2 *qv = reinterpret_cast<uint2 *>(q.xq);
+    for (int i = lane; i < nv; i += 32) {
+        unpack8(xv[i], f);
+        load_wb(i, w, b);
+        uint32_t c[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            float v = rintf(__fmul_rn(ln_value(f[e], mean, rstd, w[e], b[e]), scale));
+            v = fminf(fmaxf(v, -127.0f), 127.0f);
+            c[e] = (uint32_t)__float2int_rn(v);
+        }
+        uint32_t o[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t p01 = __byte_perm(c[4 * h], c[4 * h + 1], 0x0040), p23 = __byte_perm(c[4 * h + 2], c[4 * h + 3], 0x0040);
+            o[h] = __byte_perm(p01, p23, 0x5410);
+            sum_q = __dp4a((int)o[h], 0x01010101, sum_q);
+        }
+        qv[i] = make_uint2(o[0], o[1]);
+    }
+    sum_q = warp_sum_i(sum_q);
+    if (lane == 0) {
+        *q.row_sum = sum_q;
+        *q.gamma_x = g;
+        if (q.mean_out) *q.mean_out = mean;
+        if (q.rstd_out) *q.rstd_out = rstd;
+    }
+}
+
 template <int NT>
 __global__ void __launch_bounds__(kPgThreads, 1)
 decode_prologue_group_kernel(const QuantItem *quant_items, int n_quant, const LoraItem *lora, int n_lora) {
@@ -532,14 +605,15 @@ decode_prologue_group_kernel(const QuantItem *quant_items, int n_quant, const Lo
     // LoRA items are dealt from the first warp up, quantisation items from the last warp down, so the
     // warps with one LoRA item fewer take the rows
     const int q_first = nw - 1 - gw;
-    QuantItem q = {nullptr, nullptr, nullptr, nullptr, 0, 0};
+    QuantItem q = {};
     if (q_first < n_quant) q = quant_items[q_first];
     pdl_wait();  // x, and the scratch this kernel overwrites, belong to earlier work
 
     for (int i = q_first; i < n_quant; i += nw) {
         QuantItem q_next = q;
         if (i + nw < n_quant) q_next = quant_items[i + nw];  // travels while this row is worked on
-        warp_quant_row(q, buf - 16 * lane, pg_smem + warp * kWarpBytes, kWarpBytes, lane);
+        if (q.ln_w) warp_quant_row_ln(q, lane);
+        else warp_quant_row(q, buf - 16 * lane, pg_smem + warp * kWarpBytes, kWarpBytes, lane);
         q = q_next;
     }
 

@@ -30,7 +30,7 @@ EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_wo
            "hgf_group_destroy", "hgf_group_forward_phases", "hgf_linear_forward_static", "hgf_group_debug",
            "hgf_linear_forward_phases", "hgf_linear_forward_ln",
            "hgf_packed_bytes_b3", "hgf_pack_ternary_b3", "hgf_unpack_ternary_b3",
-           "hgf_selftest_wait_timeout"]
+           "hgf_selftest_wait_timeout", "hgf_group_create_ln"]
 
 
 class HgfError(RuntimeError):
@@ -106,6 +106,8 @@ def lib() -> ctypes.CDLL:
         L.hgf_launch_count.argtypes = []
         L.hgf_group_create.restype = c.c_int
         L.hgf_group_create.argtypes = [c.POINTER(Problem), i32, u32, c.POINTER(vp)]
+        L.hgf_group_create_ln.restype = c.c_int
+        L.hgf_group_create_ln.argtypes = [c.POINTER(Problem), c.POINTER(FrontEnd), i32, u32, c.POINTER(vp)]
         L.hgf_group_forward.restype = c.c_int
         L.hgf_group_forward.argtypes = [vp, vp]
         L.hgf_group_forward_phases.restype = c.c_int
@@ -253,8 +255,9 @@ def linear_forward_static(x, packed, gamma, d_in, d_out, y, At=None, Bt=None, ga
 
 class Group:
     """A group of independent decode-sized problems (hgf_group_*).  `problems` is a list of dicts
-    with keys x, packed, gamma, d_in, d_out, y and optionally At, Bt, gate (device tensors);
-    the tensors are kept alive by this object."""
+    with keys x, packed, gamma, d_in, d_out, y and optionally At, Bt, gate (device tensors), and for
+    the front end of hgf_group_create_ln: ln_weight, ln_bias (fp32 [d_in]), eps, gate_group, mean_out,
+    rstd_out; the tensors are kept alive by this object."""
 
     def __init__(self, problems, flags: int = 0):
         self._keep = problems
@@ -266,6 +269,16 @@ class Group:
                              None if q.get("Bt") is None else q["Bt"].data_ptr(), 0 if At is None else At.shape[0],
                              None if q.get("gate") is None else q["gate"].data_ptr(), q["y"].data_ptr())
         self._handle = ctypes.c_void_p()
+        if any(("ln_weight" in q or "gate_group" in q) for q in problems):
+            fes = (FrontEnd * len(problems))()
+            for i, q in enumerate(problems):
+                fes[i] = FrontEnd(None if q.get("ln_weight") is None else q["ln_weight"].data_ptr(),
+                                  None if q.get("ln_bias") is None else q["ln_bias"].data_ptr(), float(q.get("eps", 1e-5)),
+                                  int(q.get("gate_group", 1)),
+                                  None if q.get("mean_out") is None else q["mean_out"].data_ptr(),
+                                  None if q.get("rstd_out") is None else q["rstd_out"].data_ptr())
+            _check("hgf_group_create_ln", lib().hgf_group_create_ln(arr, fes, len(problems), flags, ctypes.byref(self._handle)))
+            return
         _check("hgf_group_create", lib().hgf_group_create(arr, len(problems), flags, ctypes.byref(self._handle)))
 
     def forward(self, stream=None) -> None:

@@ -124,3 +124,50 @@ def test_front_end_rejects_bad_arguments(hgf):
     with pytest.raises(hgf.HgfError) as e:      # a group that cuts through 16-row tiles
         hgf.linear_forward(x, packed, 1.0, 256, 64, At, Bt, gate, gate_group=24)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("M", [1, 5, 16])
+def test_attention_projections_as_one_group(hgf, M):
+    """The paper's attention block (HeadAdaptiveDiffAttention): Q, K and V are three HGF layers of the same
+    x, each behind a LayerNorm of its own, with one gate per head; plus an output projection without a
+    correction on another input.  One hgf_group_create_ln group; every problem against the oracle, integer
+    results bit for bit under the library's statistics."""
+    d, heads = 1024, 8
+    specs = [("q", d, d, 32, d // heads), ("k", d, d, 32, d // heads), ("v", d, d // 2, 32, d // 2 // heads), ("o", d // 2, d, 0, 1)]
+    x_shared = syn.make_x(M, d, config=23, layer=M)
+    probs, hosts = [], []
+    for i, (name, K, N, r, group) in enumerate(specs):
+        L = syn.make_layer(syn.LayerShape(name, K, N, max(r, 16)), M, config=23, layer=10 * M + i)
+        x = x_shared if K == d else L["x"]
+        packed, gamma = hgf.pack_ternary(dev(L["W"]))
+        T = oracle.ternarise(L["W"], np.float32(gamma))
+        w, b = ln_params(K, 50 + i)
+        gate = np.random.default_rng([33, i]).random((N + group - 1) // group).astype(np.float32)
+        q = {"x": dev(x, torch.bfloat16), "packed": packed, "gamma": gamma, "d_in": K, "d_out": N,
+             "y": torch.zeros((M, N), dtype=torch.float32, device="cuda"), "ln_weight": dev(w), "ln_bias": dev(b), "eps": 1e-5,
+             "gate_group": group, "mean_out": torch.zeros(M, device="cuda"), "rstd_out": torch.zeros(M, device="cuda")}
+        if r:
+            q.update(At=dev(L["At"], torch.float16), Bt=dev(L["Bt"], torch.float16), gate=dev(gate))
+        probs.append(q)
+        hosts.append((x, T, gamma, w, b, L["At"] if r else None, L["Bt"] if r else None, gate if r else None, group))
+    for i in (1, 2):
+        probs[i]["x"] = probs[0]["x"]          # one device buffer for Q, K and V
+    group = hgf.Group(probs)
+    y_ints = [torch.full((M, q["d_out"]), -1, dtype=torch.int32, device="cuda") for q in probs]
+    views = [group.debug(i, yi) for i, yi in enumerate(y_ints)]
+    group.forward()
+    group.forward()
+    hgf.check_status()
+    for i, (q, (x, T, gamma, w, b, At, Bt, gate, grp)) in enumerate(zip(probs, hosts)):
+        mean_g, rstd_g = q["mean_out"].cpu().numpy(), q["rstd_out"].cpu().numpy()
+        mean_o, rstd_o = oracle.ln_stats(x, 1e-5)
+        assert np.all(np.abs(mean_g - mean_o) <= 2e-7 * np.sqrt(1.0 / rstd_o ** 2 + mean_o ** 2)) and np.all(np.abs(rstd_g / rstd_o - 1) <= 3e-7)
+        own = oracle.forward_ln(x, T, gamma, w, b, 1e-5, At, Bt, gate, gate_group=grp, mean=mean_g, rstd=rstd_g)
+        assert np.array_equal(views[i]["xq"].cpu().numpy(), own["xq"]), f"problem {i}: quantised activations differ"
+        assert np.array_equal(views[i]["gamma_x"].cpu().numpy(), own["gamma_x"])
+        assert np.array_equal(y_ints[i].cpu().numpy(), own["y_int"]), f"problem {i}: int32 accumulators differ"
+        err = np.abs(q["y"].cpu().numpy().astype(np.float64) - own["y"]).max() / np.abs(own["y"]).max()
+        assert err <= TOL_DECODE, (i, err)
+    # Q, K and V have LayerNorms of their own: three quantisations of the same x, all different
+    assert not np.array_equal(views[0]["xq"].cpu().numpy(), views[1]["xq"].cpu().numpy())
+    group.close()
