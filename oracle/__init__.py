@@ -5,12 +5,14 @@ Only the tests, the smoke check and the benchmark's cpu-baseline leg import this
 from .hgf_oracle import (  # noqa: F401
     FLAG_NO_SILU,
     act_quant,
+    diff_attention,
     build,
     effective_bits,
     forward,
     forward_ln,
     gamma_w,
     int_gemm,
+    lambda0,
     ln_quant,
     ln_stats,
     pack,

@@ -20,12 +20,15 @@
  * front end: numpy float64 statistics, a constant row, rows that are already normalised (the
  * front end then reduces to the plain quantiser), sign and power-of-two invariances, the listing's
  * rounding of the tie 76/152 (-> 63), the library layer_norm routine, and the equivalence of a
- * grouped gate with its expanded per-channel vector.
+ * grouped gate with its expanded per-channel vector; for the differential attention: the library
+ * scaled_dot_product_attention routine, lambda = 0, identical streams, a single token, constant V,
+ * causality, and the lambda_0 formula's value.
  * No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 #ifdef _OPENMP
@@ -405,6 +408,56 @@ int oracle_forward_ln(const uint16_t *x_bf16, int64_t M, const int8_t *T, float 
         }
     return overflow;
 }
+
+/* ---- Section 2.4, Definition "Differential Attention" ------------------------------------------ */
+/* O = ( Softmax(Q1 K1^T / sqrt(d_h)) - lambda * Softmax(Q2 K2^T / sqrt(d_h)) ) V, per batch element and
+ * head, causal (token i attends to tokens j <= i: the model is a language model; the listing passes
+ * is_causal), times out_scale (1 in the Definition; the listing multiplies by 0.5).
+ * Storage, token-major as the projections write it: q, k [B*L][2*h*d_h] bf16 bits, where the first
+ * h*d_h columns are the h heads of stream 1 and the last h*d_h those of stream 2 (the Definition's
+ * [Q1; Q2], the listing's chunk over 2h heads); v [B*L][h*d_h] bf16 bits; out [B*L][h*d_h] double.
+ * Everything in double from the exact bf16 values; the softmax subtracts the row maximum. */
+void oracle_diff_attention(const uint16_t *q, const uint16_t *k, const uint16_t *v, int64_t B, int64_t L, int64_t h,
+                           int64_t dh, double lambda, double out_scale, double *out) {
+    const int64_t dq = 2 * h * dh, dv = h * dh;
+    const double inv = 1.0 / sqrt((double)dh);
+#pragma omp parallel for schedule(dynamic) collapse(2)
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t hd = 0; hd < h; ++hd) {
+            double *p = (double *)malloc(sizeof(double) * (size_t)L);
+            for (int64_t i = 0; i < L; ++i) {
+                double *o = out + ((b * L + i) * dv + hd * dh);
+                for (int64_t c = 0; c < dh; ++c) o[c] = 0.0;
+                for (int s = 0; s < 2; ++s) {
+                    const uint16_t *qi = q + (b * L + i) * dq + (s * h + hd) * dh;
+                    double mx = -INFINITY;
+                    for (int64_t j = 0; j <= i; ++j) {
+                        const uint16_t *kj = k + (b * L + j) * dq + (s * h + hd) * dh;
+                        double dot = 0.0;
+                        for (int64_t c = 0; c < dh; ++c) dot += bf16_to_double(qi[c]) * bf16_to_double(kj[c]);
+                        p[j] = dot * inv;
+                        if (p[j] > mx) mx = p[j];
+                    }
+                    double sum = 0.0;
+                    for (int64_t j = 0; j <= i; ++j) {
+                        p[j] = exp(p[j] - mx);
+                        sum += p[j];
+                    }
+                    const double w = (s == 0 ? 1.0 : -lambda) / sum;
+                    for (int64_t j = 0; j <= i; ++j) {
+                        const uint16_t *vj = v + (b * L + j) * dv + hd * dh;
+                        const double pj = p[j] * w;
+                        for (int64_t c = 0; c < dh; ++c) o[c] += pj * bf16_to_double(vj[c]);
+                    }
+                }
+                for (int64_t c = 0; c < dh; ++c) o[c] *= out_scale;
+            }
+            free(p);
+        }
+}
+
+/* lambda_0 = 0.8 - 0.6 exp(-0.3 d_h) (same Definition). */
+double oracle_lambda0(double dh) { return 0.8 - 0.6 * exp(-0.3 * dh); }
 
 /* ---- Introduction, memory-wall bound: T_max = B_mem / (P * b / 8) tokens per second ----------- */
 double oracle_tmax(double bmem_bytes_per_s, double params, double bits_per_param) {

@@ -71,6 +71,10 @@ def _load():
         lib.oracle_forward_ln.restype = c.c_int
         lib.oracle_forward_ln.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, c.c_double, vp, vp, vp, vp, i32, vp,
                                           i64, u32, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_diff_attention.restype = None
+        lib.oracle_diff_attention.argtypes = [vp, vp, vp, i64, i64, i64, i64, c.c_double, c.c_double, vp]
+        lib.oracle_lambda0.restype = c.c_double
+        lib.oracle_lambda0.argtypes = [c.c_double]
         lib.oracle_tmax.restype = c.c_double
         lib.oracle_tmax.argtypes = [c.c_double] * 3
         lib.oracle_effective_bits.restype = c.c_double
@@ -254,6 +258,21 @@ def forward_ln(x_bf16_bits, T, gamma, ln_w, ln_b, eps=1e-5, At_fp16_bits=None, B
     if ovf:
         raise OverflowError("integer accumulator left the int32 range")
     return {"y": y, "xq": xq, "gamma_x": gx, "y_int": yi, "h": h[:, :r], "mean": mo, "rstd": ro}
+
+
+def diff_attention(q_bf16_bits, k_bf16_bits, v_bf16_bits, B: int, L: int, h: int, dh: int, lam: float, out_scale: float = 1.0):
+    """Causal differential attention.  q, k: [B*L][2*h*dh] bf16 bits (stream 1's heads, then stream 2's);
+    v: [B*L][h*dh]; returns float64 [B*L][h*dh]."""
+    q = _arr(q_bf16_bits, np.uint16, (B * L, 2 * h * dh))
+    k = _arr(k_bf16_bits, np.uint16, (B * L, 2 * h * dh))
+    v = _arr(v_bf16_bits, np.uint16, (B * L, h * dh))
+    out = np.empty((B * L, h * dh), np.float64)
+    _load().oracle_diff_attention(_p(q), _p(k), _p(v), B, L, h, dh, float(lam), float(out_scale), _p(out))
+    return out
+
+
+def lambda0(dh: float) -> float:
+    return float(_load().oracle_lambda0(float(dh)))
 
 
 def tmax(bmem_bytes_per_s: float, params: float, bits: float) -> float:
