@@ -605,6 +605,33 @@ def run_extra(hgf, torch, syn, stream, args, peaks, int8_peak_measured=None):
                                      "frac_2x_measured_bf16": tops / int8_peak_2x_bf16})
             del w
             torch.cuda.empty_cache()
+    # differential attention forward on projection-shaped inputs (1.2B-class block: 16 heads of 64), causal
+    B_, L_, h_, dh_ = 4, 4096, 16, 64
+    gq = torch.Generator(device="cuda")
+    gq.manual_seed(5)
+    qa = torch.randn((B_ * L_, 2 * h_ * dh_), generator=gq, device="cuda").to(torch.bfloat16)
+    ka = torch.randn((B_ * L_, 2 * h_ * dh_), generator=gq, device="cuda").to(torch.bfloat16)
+    va = torch.randn((B_ * L_, h_ * dh_), generator=gq, device="cuda").to(torch.bfloat16)
+    oa = torch.empty((B_ * L_, h_ * dh_), dtype=torch.bfloat16, device="cuda")
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            hgf.diff_attention_forward(qa, ka, va, B_, L_, h_, dh_, 0.8, out=oa, flags=hgf.FLAG_OUT_BF16, stream=stream)
+        stream.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(10):
+            hgf.diff_attention_forward(qa, ka, va, B_, L_, h_, dh_, 0.8, out=oa, flags=hgf.FLAG_OUT_BF16, stream=stream)
+        t1.record(stream)
+        stream.synchronize()
+    ms = t0.elapsed_time(t1) / 10
+    at_flops = 4.0 * L_ * L_ * dh_ * B_ * h_ * 0.5 * 2   # two streams x (Q K^T and P V) x the causal half
+    extra["diff_attention"] = {"workload": f"causal differential attention forward, B={B_}, L={L_}, {h_} heads of {dh_}, bf16",
+                               "ms": ms, "TFLOP/s": at_flops / (ms * 1e-3) / 1e12,
+                               "frac_measured_bf16": at_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                               "note": "warp-level MMA kernel built for parity (a 'next' row), not tuned"}
+    del qa, ka, va, oa
+    torch.cuda.empty_cache()
+
     # config 4 prefill: the whole 7B-class stack, 32 blocks x 7 projections = 224 layers, each with its own
     # weights (generated and packed layer by layer) and its own seeded x, M = 4096, bf16 y
     stack = Workload(hgf, torch, syn.CONFIGS[4]["layers"], 4096, 32, flags=hgf.FLAG_OUT_BF16)

@@ -321,6 +321,26 @@ hgf_status hgf_act_quant(const void *x, int64_t M, int64_t d_in, int8_t *xq, flo
                          int32_t *row_sum, void *stream);
 
 /*
+ * Causal differential attention forward on the outputs of the HGF attention projections (paper,
+ * Section 2.4, Definitions "HGF Attention Projections" and "Differential Attention"):
+ *     O = ( Softmax(Q1 K1^T / sqrt(d_h)) - lambda * Softmax(Q2 K2^T / sqrt(d_h)) ) V * out_scale
+ * per batch element and head; token i attends to tokens j <= i.
+ *   q, k   [B*L][2 * n_heads * head_dim]  bfloat16, token-major as the Q and K projections write them
+ *          (HGF_FLAG_OUT_BF16): the first n_heads * head_dim columns are the heads of stream 1, the
+ *          rest those of stream 2 ([Q1; Q2] of the Definition)
+ *   v      [B*L][n_heads * head_dim]      bfloat16 (the V projection, width d / 2)
+ *   out    [B*L][n_heads * head_dim]      fp32, or bfloat16 with HGF_FLAG_OUT_BF16 (the input of the
+ *          output projection)
+ *   lambda the learnable scalar (hgf_diff_lambda0(head_dim) is its initial value 0.8 - 0.6 exp(-0.3 d_h));
+ *   out_scale 1 for the Definition; the reference module of Appendix E multiplies by 0.5.
+ * head_dim 64 or 128; 16-byte aligned pointers.  Enqueue only; no workspace.
+ */
+hgf_status hgf_diff_attention_forward(const void *q, const void *k, const void *v, int64_t B, int64_t L,
+                                      int32_t n_heads, int32_t head_dim, float lambda, float out_scale,
+                                      void *out, uint32_t flags, void *stream);
+double hgf_diff_lambda0(double head_dim);
+
+/*
  * Device-side waits in the GEMM path are bounded; when one gives up the kernel records it and
  * returns.  This call synchronises `stream`, reads and clears that record, and returns
  * HGF_ERR_TIMEOUT if a wait gave up since the last check (HGF_OK otherwise).

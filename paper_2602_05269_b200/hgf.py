@@ -30,7 +30,8 @@ EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_wo
            "hgf_group_destroy", "hgf_group_forward_phases", "hgf_linear_forward_static", "hgf_group_debug",
            "hgf_linear_forward_phases", "hgf_linear_forward_ln",
            "hgf_packed_bytes_b3", "hgf_pack_ternary_b3", "hgf_unpack_ternary_b3",
-           "hgf_selftest_wait_timeout", "hgf_group_create_ln"]
+           "hgf_selftest_wait_timeout", "hgf_group_create_ln",
+           "hgf_diff_attention_forward", "hgf_diff_lambda0"]
 
 
 class HgfError(RuntimeError):
@@ -98,6 +99,10 @@ def lib() -> ctypes.CDLL:
         L.hgf_act_quant.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.hgf_selftest_wait_timeout.restype = c.c_int
         L.hgf_selftest_wait_timeout.argtypes = [u32, vp]
+        L.hgf_diff_attention_forward.restype = c.c_int
+        L.hgf_diff_attention_forward.argtypes = [vp, vp, vp, i64, i64, i32, i32, c.c_float, c.c_float, vp, u32, vp]
+        L.hgf_diff_lambda0.restype = c.c_double
+        L.hgf_diff_lambda0.argtypes = [c.c_double]
         L.hgf_check_status.restype = c.c_int
         L.hgf_check_status.argtypes = [vp]
         L.hgf_tmax_tokens_per_s.restype = c.c_double
@@ -319,6 +324,24 @@ class Group:
 def check_status(stream=None) -> None:
     """Synchronise and raise if a bounded device-side wait gave up since the last check."""
     _check("hgf_check_status", lib().hgf_check_status(_stream(stream)))
+
+
+def diff_attention_forward(q, k, v, B: int, L: int, n_heads: int, head_dim: int, lam: float, out_scale: float = 1.0, *,
+                           out=None, flags: int = 0, stream=None):
+    """hgf_diff_attention_forward: q, k bf16 [B*L][2*n_heads*head_dim], v bf16 [B*L][n_heads*head_dim] ->
+    out [B*L][n_heads*head_dim] fp32 (bf16 with FLAG_OUT_BF16)."""
+    assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous() and k.is_contiguous() and v.is_contiguous()
+    if out is None:
+        out = torch.empty((B * L, n_heads * head_dim), dtype=torch.bfloat16 if flags & FLAG_OUT_BF16 else torch.float32,
+                          device=q.device)
+    _check("hgf_diff_attention_forward",
+           lib().hgf_diff_attention_forward(_ptr(q), _ptr(k), _ptr(v), B, L, n_heads, head_dim, ctypes.c_float(lam),
+                                            ctypes.c_float(out_scale), _ptr(out), flags, _stream(stream)))
+    return out
+
+
+def diff_lambda0(head_dim: float) -> float:
+    return float(lib().hgf_diff_lambda0(float(head_dim)))
 
 
 def selftest_wait_timeout(limit_us: int = 200, stream=None) -> None:
