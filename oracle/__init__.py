@@ -5,6 +5,7 @@ Only the tests, the smoke check and the benchmark's cpu-baseline leg import this
 from .hgf_oracle import (  # noqa: F401
     FLAG_NO_SILU,
     act_quant,
+    backward,
     diff_attention,
     build,
     effective_bits,

@@ -22,7 +22,9 @@
  * rounding of the tie 76/152 (-> 63), the library layer_norm routine, and the equivalence of a
  * grouped gate with its expanded per-channel vector; for the differential attention: the library
  * scaled_dot_product_attention routine, lambda = 0, identical streams, a single token, constant V,
- * causality, and the lambda_0 formula's value.
+ * causality, and the lambda_0 formula's value; for the backward pass: automatic differentiation
+ * (a library routine) of a float64 restatement whose quantisers are made straight-through with the
+ * value-plus-detached-difference construction, gate = 0, and linearity in dY.
  * No function here is "parity unpinned".
  */
 #include <math.h>
@@ -407,6 +409,88 @@ int oracle_forward_ln(const uint16_t *x_bf16, int64_t M, const int8_t *T, float 
             y[m * d_out + n] = y_tern + y_corr;
         }
     return overflow;
+}
+
+/* ---- Section 2.2, Definition "Straight-Through Estimator": backward pass of the layer ----------- */
+/* Forward, as differentiated: y = Xd Wd^T + g (.) (SiLU(x A) B), with Xd = x~ gamma_x / 127 the
+ * dequantised activations and Wd = gamma_W t the dequantised weights.  The estimator treats both
+ * quantisers as the identity in the backward pass (every activation lies inside its clipping range,
+ * and the reference module passes the weight gradient unchanged), everything else is differentiated
+ * exactly.  With dY the gradient of the loss with respect to y:
+ *     dW[n][k]   = sum_m dY[m][n] Xd[m][k]                      (gradient for the latent weights)
+ *     dX[m][k]   = sum_n dY[m][n] Wd[n][k]  +  sum_j dZ[m][j] A[k][j]
+ *     Z = x A,  H = SiLU(Z),  dH[m][j] = sum_n dY[m][n] g[n] B[j][n],  dZ = dH (.) SiLU'(Z)
+ *     dA[k][j]   = sum_m x[m][k] dZ[m][j],   dB[j][n] = g[n] sum_m H[m][j] dY[m][n]
+ *     dg[n]      = sum_m dY[m][n] (H B)[m][n]   (with respect to the evaluated gate g = tanh(alpha))
+ * Storage as in the forward pass: At [r][d_in], Bt [d_out][r] fp16 bits; dAt, dBt in the same shapes.
+ * dy [M][d_out] bf16 bits.  All sums in double.  Outputs nullable. */
+void oracle_backward(const uint16_t *x_bf16, int64_t M, const int8_t *T, float gamma_w, int64_t d_in, int64_t d_out,
+                     const uint16_t *At_fp16, const uint16_t *Bt_fp16, int32_t r, const float *gate, const uint16_t *dy_bf16,
+                     uint32_t flags, double *dx, double *dW, double *dAt, double *dBt, double *dgate, int8_t *xq_scratch,
+                     float *gx_scratch, double *zh_scratch /* 3 M r doubles: Z, H, dZ */) {
+    int have_corr = (r > 0 && At_fp16 && Bt_fp16 && gate);
+    oracle_act_quant(x_bf16, M, d_in, xq_scratch, gx_scratch);
+    double *Z = zh_scratch, *H = zh_scratch + M * (have_corr ? r : 0), *dZ = zh_scratch + 2 * M * (have_corr ? r : 0);
+    if (have_corr) {
+#pragma omp parallel for schedule(static)
+        for (int64_t m = 0; m < M; ++m)
+            for (int32_t j = 0; j < r; ++j) {
+                double z = 0.0;
+                for (int64_t k = 0; k < d_in; ++k)
+                    z += bf16_to_double(x_bf16[m * d_in + k]) * fp16_to_double(At_fp16[(int64_t)j * d_in + k]);
+                double dh = 0.0;
+                for (int64_t n = 0; n < d_out; ++n)
+                    dh += bf16_to_double(dy_bf16[m * d_out + n]) * (double)gate[n] * fp16_to_double(Bt_fp16[n * r + j]);
+                double sg = 1.0 / (1.0 + exp(-z));
+                Z[m * r + j] = z;
+                H[m * r + j] = (flags & ORACLE_FLAG_NO_SILU) ? z : z * sg;
+                dZ[m * r + j] = (flags & ORACLE_FLAG_NO_SILU) ? dh : dh * (sg * (1.0 + z * (1.0 - sg)));
+            }
+    }
+    if (dx) {
+#pragma omp parallel for schedule(static)
+        for (int64_t m = 0; m < M; ++m)
+            for (int64_t k = 0; k < d_in; ++k) {
+                double a = 0.0;
+                for (int64_t n = 0; n < d_out; ++n) a += bf16_to_double(dy_bf16[m * d_out + n]) * (double)T[n * d_in + k];
+                a *= (double)gamma_w;
+                if (have_corr)
+                    for (int32_t j = 0; j < r; ++j) a += dZ[m * r + j] * fp16_to_double(At_fp16[(int64_t)j * d_in + k]);
+                dx[m * d_in + k] = a;
+            }
+    }
+    if (dW) {
+#pragma omp parallel for schedule(static)
+        for (int64_t n = 0; n < d_out; ++n)
+            for (int64_t k = 0; k < d_in; ++k) {
+                double a = 0.0;
+                for (int64_t m = 0; m < M; ++m)
+                    a += bf16_to_double(dy_bf16[m * d_out + n]) * ((double)xq_scratch[m * d_in + k] * (double)gx_scratch[m] / 127.0);
+                dW[n * d_in + k] = a;
+            }
+    }
+    if (have_corr && dAt) {
+#pragma omp parallel for schedule(static)
+        for (int64_t k = 0; k < d_in; ++k)
+            for (int32_t j = 0; j < r; ++j) {
+                double a = 0.0;
+                for (int64_t m = 0; m < M; ++m) a += dZ[m * r + j] * bf16_to_double(x_bf16[m * d_in + k]);
+                dAt[(int64_t)j * d_in + k] = a;
+            }
+    }
+    if (have_corr && (dBt || dgate)) {
+#pragma omp parallel for schedule(static)
+        for (int64_t n = 0; n < d_out; ++n) {
+            double dg = 0.0;
+            for (int32_t j = 0; j < r; ++j) {
+                double a = 0.0;
+                for (int64_t m = 0; m < M; ++m) a += bf16_to_double(dy_bf16[m * d_out + n]) * H[m * r + j];
+                if (dBt) dBt[n * r + j] = (double)gate[n] * a;
+                dg += a * fp16_to_double(Bt_fp16[n * r + j]);
+            }
+            if (dgate) dgate[n] = dg;
+        }
+    }
 }
 
 /* ---- Section 2.4, Definition "Differential Attention" ------------------------------------------ */

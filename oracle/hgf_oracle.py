@@ -71,6 +71,8 @@ def _load():
         lib.oracle_forward_ln.restype = c.c_int
         lib.oracle_forward_ln.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, c.c_double, vp, vp, vp, vp, i32, vp,
                                           i64, u32, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_backward.restype = None
+        lib.oracle_backward.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, u32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_diff_attention.restype = None
         lib.oracle_diff_attention.argtypes = [vp, vp, vp, i64, i64, i64, i64, c.c_double, c.c_double, vp]
         lib.oracle_lambda0.restype = c.c_double
@@ -258,6 +260,33 @@ def forward_ln(x_bf16_bits, T, gamma, ln_w, ln_b, eps=1e-5, At_fp16_bits=None, B
     if ovf:
         raise OverflowError("integer accumulator left the int32 range")
     return {"y": y, "xq": xq, "gamma_x": gx, "y_int": yi, "h": h[:, :r], "mean": mo, "rstd": ro}
+
+
+def backward(x_bf16_bits, T, gamma, dy_bf16_bits, At_fp16_bits=None, Bt_fp16_bits=None, gate=None, flags: int = 0):
+    """Straight-through backward pass of the layer.  Returns a dict of float64 arrays: dx [M][K], dW [N][K],
+    and with a correction dAt [r][K], dBt [N][r], dgate [N]."""
+    x = _arr(x_bf16_bits, np.uint16)
+    T = _arr(T, np.int8)
+    M, K = x.shape
+    N = T.shape[0]
+    dy = _arr(dy_bf16_bits, np.uint16, (M, N))
+    r = 0
+    At = Bt = g = None
+    if At_fp16_bits is not None and Bt_fp16_bits is not None and gate is not None:
+        At = _arr(At_fp16_bits, np.uint16)
+        r = At.shape[0]
+        Bt = _arr(Bt_fp16_bits, np.uint16, (N, r))
+        g = _arr(gate, np.float32, (N,))
+    out = {"dx": np.empty((M, K), np.float64), "dW": np.empty((N, K), np.float64)}
+    if r:
+        out.update(dAt=np.empty((r, K), np.float64), dBt=np.empty((N, r), np.float64), dgate=np.empty(N, np.float64))
+    xq = np.empty((M, K), np.int8)
+    gx = np.empty(M, np.float32)
+    scratch = np.empty(3 * M * max(r, 1), np.float64)
+    _load().oracle_backward(_p(x), M, _p(T), float(np.float32(gamma)), K, N, _p(At), _p(Bt), r, _p(g), _p(dy), flags,
+                            _p(out["dx"]), _p(out["dW"]), _p(out.get("dAt")), _p(out.get("dBt")), _p(out.get("dgate")),
+                            _p(xq), _p(gx), _p(scratch))
+    return out
 
 
 def diff_attention(q_bf16_bits, k_bf16_bits, v_bf16_bits, B: int, L: int, h: int, dh: int, lam: float, out_scale: float = 1.0):
