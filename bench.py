@@ -632,6 +632,32 @@ def run_extra(hgf, torch, syn, stream, args, peaks, int8_peak_measured=None):
     del qa, ka, va, oa
     torch.cuda.empty_cache()
 
+    # straight-through backward pass of one layer (2048 -> 5632, r = 32, M = 8192): all five gradients
+    sb = syn.CONFIGS[3]["layers"][4]
+    Mb = 8192
+    wb = Workload(hgf, torch, [sb], Mb, 1)
+    (_s, xb, pb, gb, Ab, Bb, gateb, _y) = wb.layers[0]
+    dyb = torch.randn((Mb, sb.d_out), generator=gq, device="cuda").to(torch.bfloat16)
+    hgf.linear_backward(xb, pb, gb, sb.d_in, sb.d_out, dyb, Ab, Bb, gateb, stream=stream)
+    stream.synchronize()
+    with torch.cuda.stream(stream):
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        keep = hgf.linear_backward(xb, pb, gb, sb.d_in, sb.d_out, dyb, Ab, Bb, gateb, stream=stream)
+        t0.record(stream)
+        for _ in range(5):
+            keep = hgf.linear_backward(xb, pb, gb, sb.d_in, sb.d_out, dyb, Ab, Bb, gateb, stream=stream)
+        t1.record(stream)
+        stream.synchronize()
+    ms = t0.elapsed_time(t1) / 5
+    bw_flops = 2.0 * Mb * sb.d_in * sb.d_out * 2 + 2.0 * Mb * sb.r * (sb.d_in + sb.d_out) * 3
+    extra["ste_backward"] = {"workload": f"straight-through backward of one layer {sb.d_in}->{sb.d_out}, r={sb.r}, M={Mb}: dX, dW, dA, dB, dgate",
+                             "ms": ms, "TFLOP/s": bw_flops / (ms * 1e-3) / 1e12,
+                             "frac_measured_bf16": bw_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                             "note": "warp-level bf16 MMA GEMMs built for parity (a 'next' row), not tuned; includes the "
+                                     "operand preparation and a device allocation of the workspace per call"}
+    del wb, keep, dyb
+    torch.cuda.empty_cache()
+
     # config 4 prefill: the whole 7B-class stack, 32 blocks x 7 projections = 224 layers, each with its own
     # weights (generated and packed layer by layer) and its own seeded x, M = 4096, bf16 y
     stack = Workload(hgf, torch, syn.CONFIGS[4]["layers"], 4096, 32, flags=hgf.FLAG_OUT_BF16)

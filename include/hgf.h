@@ -341,6 +341,36 @@ hgf_status hgf_diff_attention_forward(const void *q, const void *k, const void *
 double hgf_diff_lambda0(double head_dim);
 
 /*
+ * Straight-through backward pass of the layer (paper, Section 2.2, Definition "Straight-Through
+ * Estimator"): the forward pass of hgf_linear_forward is differentiated with both quantisers treated
+ * as the identity (every activation lies inside its clipping range; the weight gradient is passed
+ * unchanged, as in the reference module), everything else exactly.  With Xd = x~ gamma_x / 127,
+ * Wd = gamma_W t, Z = x A, H = SiLU(Z) and dY the gradient with respect to y:
+ *     dW = dY^T Xd                          [d_out][d_in]  (gradient for the latent fp32 weights)
+ *     dX = dY Wd + dZ A^T                   [M][d_in],   dZ = ((dY (.) g) B^T) (.) SiLU'(Z)
+ *     dAt = dZ^T x  [r][d_in],  dBt = g (.) (dY^T H)  [d_out][r],  dgate = sum_m dY (.) (H B)  [d_out]
+ * (dgate is with respect to the evaluated gate g; d alpha = dgate (1 - g^2) is the caller's.)
+ * x, packed, gamma, At, Bt, gate as in the forward call; dy [M][d_out] bfloat16.  Every output is fp32
+ * and nullable (skipped).  The matrix products run on the tensor cores with bf16 operands and fp32
+ * accumulation (the precision the paper trains in): x~ and t enter exactly, dY scaled by gamma_x / 127
+ * or by g, A, B, H and dZ rounded to bf16.  Requirements: d_in % 64 == 0, d_out % 8 == 0, r in
+ * {0,16,32,48,64}; 16-byte aligned pointers; workspace of hgf_backward_workspace_bytes(...) bytes,
+ * 256-byte aligned.  Flags: HGF_FLAG_NO_SILU.  Enqueue only.
+ */
+typedef struct {
+    float *dx;
+    float *dW;
+    float *dAt;
+    float *dBt;
+    float *dgate;
+} hgf_grads;
+size_t hgf_backward_workspace_bytes(int64_t M, int64_t d_in, int64_t d_out, int32_t r);
+hgf_status hgf_linear_backward(const void *x, int64_t M, const void *packed, float gamma, int64_t d_in,
+                               int64_t d_out, const void *At, const void *Bt, int32_t r, const float *gate,
+                               const void *dy, const hgf_grads *grads, void *workspace,
+                               size_t workspace_bytes, uint32_t flags, void *stream);
+
+/*
  * Device-side waits in the GEMM path are bounded; when one gives up the kernel records it and
  * returns.  This call synchronises `stream`, reads and clears that record, and returns
  * HGF_ERR_TIMEOUT if a wait gave up since the last check (HGF_OK otherwise).

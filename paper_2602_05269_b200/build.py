@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhgf_b200.so")
 OBJ_DIR = os.path.join(HERE, "_build")
-SOURCES = ["hgf_api.cu", "hgf_pack.cu", "hgf_prologue.cu", "hgf_decode.cu", "hgf_prefill.cu", "hgf_attention.cu"]
+SOURCES = ["hgf_api.cu", "hgf_pack.cu", "hgf_prologue.cu", "hgf_decode.cu", "hgf_prefill.cu", "hgf_attention.cu", "hgf_backward.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

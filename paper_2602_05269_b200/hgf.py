@@ -31,7 +31,7 @@ EXPORTS = ["hgf_packed_bytes", "hgf_pack_ternary", "hgf_unpack_ternary", "hgf_wo
            "hgf_linear_forward_phases", "hgf_linear_forward_ln",
            "hgf_packed_bytes_b3", "hgf_pack_ternary_b3", "hgf_unpack_ternary_b3",
            "hgf_selftest_wait_timeout", "hgf_group_create_ln",
-           "hgf_diff_attention_forward", "hgf_diff_lambda0"]
+           "hgf_diff_attention_forward", "hgf_diff_lambda0", "hgf_backward_workspace_bytes", "hgf_linear_backward"]
 
 
 class HgfError(RuntimeError):
@@ -50,6 +50,11 @@ class Problem(ctypes.Structure):
 class DebugOut(ctypes.Structure):
     _fields_ = [("xq", ctypes.c_void_p), ("gamma_x", ctypes.c_void_p), ("y_int", ctypes.c_void_p),
                 ("h", ctypes.c_void_p)]
+
+
+class Grads(ctypes.Structure):
+    _fields_ = [("dx", ctypes.c_void_p), ("dW", ctypes.c_void_p), ("dAt", ctypes.c_void_p), ("dBt", ctypes.c_void_p),
+                ("dgate", ctypes.c_void_p)]
 
 
 class FrontEnd(ctypes.Structure):
@@ -103,6 +108,10 @@ def lib() -> ctypes.CDLL:
         L.hgf_diff_attention_forward.argtypes = [vp, vp, vp, i64, i64, i32, i32, c.c_float, c.c_float, vp, u32, vp]
         L.hgf_diff_lambda0.restype = c.c_double
         L.hgf_diff_lambda0.argtypes = [c.c_double]
+        L.hgf_backward_workspace_bytes.restype = sz
+        L.hgf_backward_workspace_bytes.argtypes = [i64, i64, i64, i32]
+        L.hgf_linear_backward.restype = c.c_int
+        L.hgf_linear_backward.argtypes = [vp, i64, vp, c.c_float, i64, i64, vp, vp, i32, vp, vp, c.POINTER(Grads), vp, sz, u32, vp]
         L.hgf_check_status.restype = c.c_int
         L.hgf_check_status.argtypes = [vp]
         L.hgf_tmax_tokens_per_s.restype = c.c_double
@@ -324,6 +333,26 @@ class Group:
 def check_status(stream=None) -> None:
     """Synchronise and raise if a bounded device-side wait gave up since the last check."""
     _check("hgf_check_status", lib().hgf_check_status(_stream(stream)))
+
+
+def linear_backward(x, packed, gamma, d_in, d_out, dy, At=None, Bt=None, gate=None, *, flags=0, stream=None, want=None):
+    """hgf_linear_backward: straight-through backward pass.  dy bf16 [M][d_out].  Returns a dict of fp32 device
+    tensors dx, dW and (with a correction) dAt, dBt, dgate; `want` restricts which are computed."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and dy.dtype == torch.bfloat16 and x.is_contiguous() and dy.is_contiguous()
+    M = x.shape[0]
+    r = 0 if At is None else At.shape[0]
+    names = ["dx", "dW"] + (["dAt", "dBt", "dgate"] if r else [])
+    if want is not None:
+        names = [n for n in names if n in want]
+    shapes = {"dx": (M, d_in), "dW": (d_out, d_in), "dAt": (r, d_in), "dBt": (d_out, r), "dgate": (d_out,)}
+    out = {n: torch.empty(shapes[n], dtype=torch.float32, device=x.device) for n in names}
+    g = Grads(*[out[n].data_ptr() if n in out else None for n in ("dx", "dW", "dAt", "dBt", "dgate")])
+    ws = torch.empty(int(lib().hgf_backward_workspace_bytes(M, d_in, d_out, r)), dtype=torch.uint8, device=x.device)
+    _check("hgf_linear_backward",
+           lib().hgf_linear_backward(_ptr(x), M, _ptr(packed), ctypes.c_float(gamma), d_in, d_out, _ptr(At), _ptr(Bt), r, _ptr(gate),
+                                     _ptr(dy), ctypes.byref(g), _ptr(ws), ws.numel(), flags, _stream(stream)))
+    out["_workspace"] = ws
+    return out
 
 
 def diff_attention_forward(q, k, v, B: int, L: int, n_heads: int, head_dim: int, lam: float, out_scale: float = 1.0, *,
