@@ -461,6 +461,20 @@ DECODE_TRAFFIC = {"source_sha1": "7b2cc479563a0d062a4c3a356e67630e5471a690",
                   "dram_bytes_per_algorithmic_byte": (517.347072e6 + 7.010560e6) / 518805504.0}
 
 
+# DRAM traffic of the prefill GEMM launch from one ncu capture of the very shape the bench times
+# (2048 -> 5632, r = 32, M = 8192, bf16 y): dram__bytes_read.sum + dram__bytes_write.sum of one launch.  Below
+# the launch's algorithmic bytes because most of y is still in L2 when the kernel ends.
+PREFILL_TRAFFIC = {"source_sha1": "c92a00a1521c868c5ff9abd1dae7e14e3ccfed06", "dram_bytes_per_launch": 21.571072e6 + 43.429632e6}
+
+
+def prefill_traffic():
+    import hashlib
+    src = os.path.join(ROOT, "paper_2602_05269_b200", "csrc", "hgf_prefill.cu")
+    if not os.path.exists(src) or hashlib.sha1(open(src, "rb").read()).hexdigest() != PREFILL_TRAFFIC["source_sha1"]:
+        return None
+    return PREFILL_TRAFFIC["dram_bytes_per_launch"]
+
+
 def decode_traffic(gemv_bytes):
     import hashlib
     src = os.path.join(ROOT, "paper_2602_05269_b200", "csrc", "hgf_decode.cu")
@@ -529,7 +543,10 @@ def measure_prefill_headline(hgf, torch, syn, stream, args, peaks):
     prol_bytes = 2 * M * s.d_in + M * s.d_in + 2 * s.r * s.d_in      # x read, x~ written, A read
     return {"bound": "tensor", "kernel": "prefill_gemm_kernel (the contraction launch of hgf_linear_forward, timed alone)",
             "workload": f"config3 {s.d_in}->{s.d_out}, r={s.r}, M={M}, bf16 y, {copies} distinct layers in rotation (inputs larger than L2)",
-            "achieved": tops_gemm, "peak": peak, "unit": "TOPS (int8, 2*M*K*N)", "frac": tops_gemm / peak, "traffic": None,
+            "achieved": tops_gemm, "peak": peak, "unit": "TOPS (int8, 2*M*K*N)", "frac": tops_gemm / peak, "traffic": prefill_traffic(),
+            "traffic_note": "ncu dram bytes of one launch of this shape (x~ 16.8 MB + W 2.9 MB read, y 92 MB written, of which "
+                            "about half is still in L2 at kernel end); null when hgf_prefill.cu differs from the captured source",
+            "algorithmic_bytes_per_launch": M * s.d_in + s.d_in * s.d_out // 4 + 2 * M * s.d_out + 2 * 64 * (M + s.d_out),
             "peak_source": peak_source, "int8_stick": stick,
             "ops_per_launch": ops, "us_per_launch": ms_gemm * 1e3,
             "frac_of_2x_measured_bf16": tops_gemm / (2.0 * peaks["bf16_tflops"]), "frac_of_nominal_4500": tops_gemm / 4500.0,
