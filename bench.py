@@ -464,13 +464,15 @@ DECODE_TRAFFIC = {"source_sha1": "7b2cc479563a0d062a4c3a356e67630e5471a690",
 # DRAM traffic of the prefill GEMM launch from one ncu capture of the very shape the bench times
 # (2048 -> 5632, r = 32, M = 8192, bf16 y): dram__bytes_read.sum + dram__bytes_write.sum of one launch.  Below
 # the launch's algorithmic bytes because most of y is still in L2 when the kernel ends.
-PREFILL_TRAFFIC = {"source_sha1": "c92a00a1521c868c5ff9abd1dae7e14e3ccfed06", "dram_bytes_per_launch": 21.571072e6 + 43.429632e6}
+PREFILL_TRAFFIC = {"source_sha1": "820e55be152b4392c9290353ebaab2bf22b8e090", "dram_bytes_per_launch": 21.571072e6 + 43.429632e6}
 
 
 def prefill_traffic():
     import hashlib
-    src = os.path.join(ROOT, "paper_2602_05269_b200", "csrc", "hgf_prefill.cu")
-    if not os.path.exists(src) or hashlib.sha1(open(src, "rb").read()).hexdigest() != PREFILL_TRAFFIC["source_sha1"]:
+    srcs = [os.path.join(ROOT, "paper_2602_05269_b200", "csrc", f) for f in ("hgf_prefill.cu", "hgf_tc.cuh")]
+    if not all(os.path.exists(f) for f in srcs):
+        return None
+    if hashlib.sha1(b"".join(open(f, "rb").read() for f in srcs)).hexdigest() != PREFILL_TRAFFIC["source_sha1"]:
         return None
     return PREFILL_TRAFFIC["dram_bytes_per_launch"]
 
@@ -545,7 +547,7 @@ def measure_prefill_headline(hgf, torch, syn, stream, args, peaks):
             "workload": f"config3 {s.d_in}->{s.d_out}, r={s.r}, M={M}, bf16 y, {copies} distinct layers in rotation (inputs larger than L2)",
             "achieved": tops_gemm, "peak": peak, "unit": "TOPS (int8, 2*M*K*N)", "frac": tops_gemm / peak, "traffic": prefill_traffic(),
             "traffic_note": "ncu dram bytes of one launch of this shape (x~ 16.8 MB + W 2.9 MB read, y 92 MB written, of which "
-                            "about half is still in L2 at kernel end); null when hgf_prefill.cu differs from the captured source",
+                            "about half is still in L2 at kernel end); null when hgf_prefill.cu or hgf_tc.cuh differs from the captured source",
             "algorithmic_bytes_per_launch": M * s.d_in + s.d_in * s.d_out // 4 + 2 * M * s.d_out + 2 * 64 * (M + s.d_out),
             "peak_source": peak_source, "int8_stick": stick,
             "ops_per_launch": ops, "us_per_launch": ms_gemm * 1e3,
@@ -670,8 +672,8 @@ def run_extra(hgf, torch, syn, stream, args, peaks, int8_peak_measured=None):
     extra["ste_backward"] = {"workload": f"straight-through backward of one layer {sb.d_in}->{sb.d_out}, r={sb.r}, M={Mb}: dX, dW, dA, dB, dgate",
                              "ms": ms, "TFLOP/s": bw_flops / (ms * 1e-3) / 1e12,
                              "frac_measured_bf16": bw_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                             "note": "warp-level bf16 MMA GEMMs built for parity (a 'next' row), not tuned; includes the "
-                                     "operand preparation and a device allocation of the workspace per call"}
+                             "note": "tcgen05 bf16 GEMMs (a 'next' row); includes the operand preparation "
+                                     "kernels and a device allocation of the workspace per call"}
     del wb, keep, dyb
     torch.cuda.empty_cache()
 

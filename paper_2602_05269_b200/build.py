@@ -23,7 +23,7 @@ def _nvcc() -> str:
 
 
 def _deps(src: str):
-    return [src, os.path.join(CSRC, "hgf_common.cuh"), os.path.join(HERE, "..", "include", "hgf.h")]
+    return [src, os.path.join(CSRC, "hgf_common.cuh"), os.path.join(CSRC, "hgf_tc.cuh"), os.path.join(HERE, "..", "include", "hgf.h")]
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
