@@ -664,7 +664,7 @@ def run_extra(hgf, torch, syn, stream, args, peaks, int8_peak_measured=None):
         keep = hgf.linear_backward(xb, pb, gb, sb.d_in, sb.d_out, dyb, Ab, Bb, gateb, stream=stream)
         t0.record(stream)
         for _ in range(5):
-            keep = hgf.linear_backward(xb, pb, gb, sb.d_in, sb.d_out, dyb, Ab, Bb, gateb, stream=stream)
+            keep = hgf.linear_backward(xb, pb, gb, sb.d_in, sb.d_out, dyb, Ab, Bb, gateb, stream=stream, out=keep)
         t1.record(stream)
         stream.synchronize()
     ms = t0.elapsed_time(t1) / 5
@@ -672,8 +672,8 @@ def run_extra(hgf, torch, syn, stream, args, peaks, int8_peak_measured=None):
     extra["ste_backward"] = {"workload": f"straight-through backward of one layer {sb.d_in}->{sb.d_out}, r={sb.r}, M={Mb}: dX, dW, dA, dB, dgate",
                              "ms": ms, "TFLOP/s": bw_flops / (ms * 1e-3) / 1e12,
                              "frac_measured_bf16": bw_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                             "note": "tcgen05 bf16 GEMMs (a 'next' row); includes the operand preparation "
-                                     "kernels and a device allocation of the workspace per call"}
+                             "note": "tcgen05 bf16 GEMMs reading every operand in its stored form (a 'next' row); "
+                                     "includes the operand preparation kernels; gradients and workspace preallocated"}
     del wb, keep, dyb
     torch.cuda.empty_cache()
 

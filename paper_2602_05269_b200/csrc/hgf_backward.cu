@@ -12,21 +12,28 @@
 
 namespace hgf {
 
-// ---- generic GEMM on the 5th-generation tensor cores: C[I][J] (fp32) = alpha * A B^T (+ C) ----------
-// A is stored [I][Cn], B [J][Cn], both bf16 with the contraction index contiguous ("K-major"): the form
-// TMA stages with the 128-byte swizzle and tcgen05.mma reads straight from shared memory.  Operands
-// that the backward pass has the other way round are transposed by the preparation kernels below.
-// Persistent, one CTA per SM, six warps: warp 0 stages operand tiles with TMA (128 rows of A, BN rows
-// of B, 64 contraction elements = 128 bytes per row and stage), one lane of warp 1 issues
+// ---- generic GEMM on the 5th-generation tensor cores: C[I][J] (fp32) = alpha * sum_c A[i][c] B[j][c] (+ C) ----
+// Either operand may be stored with the contraction index contiguous ([rows][Cn], "K-major") or with its
+// row index contiguous ([Cn][rows], "MN-major"): tcgen05.mma reads both forms from shared memory (the
+// instruction descriptor says which), so no operand of the backward pass is ever transposed in memory.
+// A K-major tile of R rows x 64 contraction elements is one TMA box of R rows of 128 bytes; an MN-major
+// tile is R / 64 boxes of 64 contraction rows of 128 bytes (64 operand rows each), 8 KiB apart; both use
+// the 128-byte swizzle.  The contraction may continue over a second pair of operands (A2, B2: the
+// low-rank term of dX), and may be split over several CTAs that write partial sums which a second
+// kernel adds up in a fixed order.
+// Persistent, one CTA per SM, six warps: warp 0 stages operand tiles with TMA, one lane of warp 1 issues
 // tcgen05.mma.kind::f16 (bf16 inputs, 128 x BN x 16 per instruction, fp32 accumulators in tensor memory,
 // two of them so that a tile's epilogue runs under the next tile's main loop), warps 2-5 read the
 // accumulator back (tcgen05.ld) and write C.  Rows and columns past the matrices, and contraction
 // elements past Cn, are zeros from TMA's out-of-bounds fill; stores are guarded.  Every wait is bounded.
-constexpr int kTBM = 128, kTBK = 64, kTThreads = 192;
+constexpr int kTBM = 128, kTBK = 64, kTThreads = 192, kTBox = 64 * 128;
 
 struct TcGemmArgs {
-    float *C;
-    int I, J, Cn, ldc;
+    float *C;          // output, or the partial sums [splits][I][ldc] when splits > 1
+    int I, J, ldc;
+    int kb1, kb2;      // 64-element contraction blocks of the first and of the second operand pair
+    int splits, kb_per_split;
+    int a_mn, b_mn;    // operand forms (both pairs alike)
     float alpha;
     int accumulate;
 };
@@ -43,9 +50,18 @@ struct TcCfg {
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
 };
 
+// Shared-memory descriptor of an MN-major tile with the 128-byte swizzle: 64 operand rows x 8 contraction
+// rows per 1 KiB swizzle atom; leading byte offset (bits 16-29) = distance between 64-row blocks (one TMA
+// box), stride byte offset (32-45) = distance between groups of 8 contraction rows.
+__device__ __forceinline__ uint64_t make_sw128_mn_desc(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(kTBox >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+
 template <int BN>
 __global__ void __launch_bounds__(kTThreads, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const TcGemmArgs g,
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+               const __grid_constant__ CUtensorMap tmap_a2, const __grid_constant__ CUtensorMap tmap_b2, const TcGemmArgs g,
                unsigned int *status) {
     using C = TcCfg<BN>;
     extern __shared__ uint8_t tc_smem_raw[];
@@ -55,8 +71,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::OFF_BAR + C::BAR_COUNT * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_BAR + C::BAR_COUNT * 8 + 4);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int tiles_i = (g.I + kTBM - 1) / kTBM, tiles_j = (g.J + BN - 1) / BN, num_tiles = tiles_i * tiles_j;
-    const int kblocks = (g.Cn + kTBK - 1) / kTBK;
+    const int tiles_i = (g.I + kTBM - 1) / kTBM, tiles_j = (g.J + BN - 1) / BN, tiles_ij = tiles_i * tiles_j;
+    const int num_work = tiles_ij * g.splits, kb_all = g.kb1 + g.kb2;
+    // work item w: output tile w % tiles_ij, contraction blocks [kb_lo, kb_hi) of split w / tiles_ij
+    auto kb_lo = [&](int w) { return (w / tiles_ij) * g.kb_per_split; };
+    auto kb_hi = [&](int w) { const int e = (w / tiles_ij + 1) * g.kb_per_split; return e < kb_all ? e : kb_all; };
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
@@ -87,15 +106,27 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         uint32_t ph = 0;
         uint32_t issued[C::STAGES] = {};
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-            const int i0 = (tile / tiles_j) * kTBM, j0 = (tile % tiles_j) * BN;
-            for (int kb = 0; kb < kblocks; ++kb) {
+        for (int w = blockIdx.x; ok && w < num_work; w += gridDim.x) {
+            const int tile = w % tiles_ij, i0 = (tile / tiles_j) * kTBM, j0 = (tile % tiles_j) * BN;
+            for (int kb = kb_lo(w); kb < kb_hi(w); ++kb) {
                 ok = mbar_wait(bar(C::BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x800u + s);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(bar(C::BAR_FULL + s), C::STAGE_BYTES);
-                    tma_load_2d(sbase + s * C::STAGE_BYTES, &tmap_a, kb * kTBK, i0, bar(C::BAR_FULL + s));
-                    tma_load_2d(sbase + s * C::STAGE_BYTES + C::A_BYTES, &tmap_b, kb * kTBK, j0, bar(C::BAR_FULL + s));
+                    const bool second = kb >= g.kb1;
+                    const CUtensorMap *ma = second ? &tmap_a2 : &tmap_a, *mb = second ? &tmap_b2 : &tmap_b;
+                    const int c0 = (second ? kb - g.kb1 : kb) * kTBK;
+                    const uint32_t dst_a = sbase + s * C::STAGE_BYTES, dst_b = dst_a + C::A_BYTES, full = bar(C::BAR_FULL + s);
+                    mbar_arrive_expect_tx(full, C::STAGE_BYTES);
+                    if (g.a_mn) {
+                        for (int h = 0; h < kTBM / 64; ++h) tma_load_2d(dst_a + h * kTBox, ma, i0 + 64 * h, c0, full);
+                    } else {
+                        tma_load_2d(dst_a, ma, c0, i0, full);
+                    }
+                    if (g.b_mn) {
+                        for (int h = 0; h < BN / 64; ++h) tma_load_2d(dst_b + h * kTBox, mb, j0 + 64 * h, c0, full);
+                    } else {
+                        tma_load_2d(dst_b, mb, c0, j0, full);
+                    }
                 }
                 ++issued[s];
                 if (++s == C::STAGES) { s = 0; ph ^= 1u; }
@@ -112,20 +143,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int s = 0, it = 0;
             uint32_t ph = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+            const uint32_t idesc = C::IDESC | (g.a_mn ? 1u << 15 : 0u) | (g.b_mn ? 1u << 16 : 0u);
+            const uint32_t a_step = g.a_mn ? (16 * 128) >> 4 : 32 >> 4, b_step = g.b_mn ? (16 * 128) >> 4 : 32 >> 4;  // 16 contraction elements
+            for (int w = blockIdx.x; ok && w < num_work; w += gridDim.x, ++it) {
                 const int b = it & 1;
                 const uint32_t acc = tmem_base + b * BN;
                 if (it >= 2 && !(ok = mbar_wait(bar(C::BAR_ACCEMPTY + b), (uint32_t)((it >> 1) - 1) & 1u, abort_flag, status, 0x810u)))
                     break;
                 tc_fence_after();
-                for (int kb = 0; kb < kblocks; ++kb) {
+                const int lo = kb_lo(w), hi = kb_hi(w);
+                for (int kb = lo; kb < hi; ++kb) {
                     if (!(ok = mbar_wait(bar(C::BAR_FULL + s), ph, abort_flag, status, 0x820u + s))) break;
                     tc_fence_after();
-                    const uint64_t adesc = make_sw128_desc(sbase + s * C::STAGE_BYTES);
-                    const uint64_t bdesc = make_sw128_desc(sbase + s * C::STAGE_BYTES + C::A_BYTES);
+                    const uint32_t sa = sbase + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+                    const uint64_t adesc = g.a_mn ? make_sw128_mn_desc(sa) : make_sw128_desc(sa);
+                    const uint64_t bdesc = g.b_mn ? make_sw128_mn_desc(sb) : make_sw128_desc(sb);
 #pragma unroll
-                    for (int kk = 0; kk < kTBK / 16; ++kk)  // 16 bf16 = 32 bytes of a row per MMA
-                        mma_f16(acc, adesc + 2u * kk, bdesc + 2u * kk, C::IDESC, (kb | kk) ? 1u : 0u);
+                    for (int kk = 0; kk < kTBK / 16; ++kk)
+                        mma_f16(acc, adesc + (uint64_t)(a_step * kk), bdesc + (uint64_t)(b_step * kk), idesc, (kb > lo || kk) ? 1u : 0u);
                     tc_commit(bar(C::BAR_EMPTY + s));
                     if (++s == C::STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -138,26 +173,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int q = warp & 3;  // tensor-memory lane quarter this warp may access
         bool ok = true;
         int it = 0;
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-            const int i0 = (tile / tiles_j) * kTBM, j0 = (tile % tiles_j) * BN;
+        for (int w = blockIdx.x; ok && w < num_work; w += gridDim.x, ++it) {
+            const int tile = w % tiles_ij, i0 = (tile / tiles_j) * kTBM, j0 = (tile % tiles_j) * BN;
+            float *Cw = g.C + (size_t)(w / tiles_ij) * g.I * g.ldc;
             const int b = it & 1;
             ok = mbar_wait(bar(C::BAR_ACCFULL + b), (uint32_t)(it >> 1) & 1u, abort_flag, status, 0x830u);
             if (!(ok = __all_sync(0xffffffffu, ok))) break;
             tc_fence_after();
             const int i = i0 + 32 * q + lane;  // this thread's row of C = its tensor-memory lane
             const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16) + b * BN;
+            const bool empty = kb_lo(w) >= kb_hi(w);  // a split past the end of the contraction: zeros
             for (int cc = 0; cc < BN; cc += 32) {
                 if (j0 + cc >= g.J) break;  // (warp-uniform)
                 uint32_t v[32];
                 tmem_ld32(lane_base + cc, v);
                 tmem_ld_wait();
                 if (i < g.I) {
-                    float *row = g.C + (size_t)i * g.ldc + j0 + cc;
+                    float *row = Cw + (size_t)i * g.ldc + j0 + cc;
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
                         if (j0 + cc + 4 * u < g.J) {  // J is a multiple of 4
                             float4 o = make_float4(g.alpha * __uint_as_float(v[4 * u]), g.alpha * __uint_as_float(v[4 * u + 1]),
                                                    g.alpha * __uint_as_float(v[4 * u + 2]), g.alpha * __uint_as_float(v[4 * u + 3]));
+                            if (empty) o = make_float4(0.f, 0.f, 0.f, 0.f);
                             float4 *dst = reinterpret_cast<float4 *>(row + 4 * u);
                             if (g.accumulate) { const float4 c = *dst; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
                             *dst = o;
@@ -178,118 +216,135 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(C::TMEM_COLS) : "memory");
     }
 }
+// Sum of the partial results of a split contraction, in split order: C = alpha * sum_s P[s] (+ C).
+__global__ void __launch_bounds__(256) tc_reduce_kernel(const float4 *P, int splits, size_t n4, float alpha, int accumulate, float4 *C) {
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= n4) return;
+    float4 a = P[i];
+    for (int s = 1; s < splits; ++s) {
+        const float4 b = P[(size_t)s * n4 + i];
+        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+    }
+    a.x *= alpha; a.y *= alpha; a.z *= alpha; a.w *= alpha;
+    if (accumulate) { const float4 c = C[i]; a.x += c.x; a.y += c.y; a.z += c.z; a.w += c.w; }
+    C[i] = a;
+}
+
+// One operand: `rows` x `cn` values; mn = stored [cn][rows] (row index contiguous), else [rows][cn]; ld in elements.
+struct TcOperand {
+    const __nv_bfloat16 *p;
+    int ld;
+    bool mn;
+};
+
+static bool tc_map(CUtensorMap *m, const TcOperand &o, int rows, int cn, int tile_rows) {
+    if (o.mn) return make_map_2d(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, o.p, (uint64_t)rows, (uint64_t)cn, (uint64_t)o.ld * 2, 64, kTBK, CU_TENSOR_MAP_SWIZZLE_128B);
+    return make_map_2d(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, o.p, (uint64_t)cn, (uint64_t)rows, (uint64_t)o.ld * 2, kTBK, (uint32_t)tile_rows, CU_TENSOR_MAP_SWIZZLE_128B);
+}
 
 template <int BN>
-static cudaError_t tc_gemm_bn(const CUtensorMap &ma, const CUtensorMap &mb, const TcGemmArgs &g, cudaStream_t stream) {
+static cudaError_t tc_gemm_bn(const CUtensorMap *maps, const TcGemmArgs &g, cudaStream_t stream) {
     static std::atomic<unsigned long long> attr_done{0};
     cudaError_t e = ensure_dynamic_smem(tc_gemm_kernel<BN>, TcCfg<BN>::SMEM_BYTES, attr_done);
     if (e != cudaSuccess) return e;
     const int sms = device_sm_count();
     if (!sms) return cudaErrorInvalidDevice;
-    const int tiles = ((g.I + kTBM - 1) / kTBM) * ((g.J + BN - 1) / BN);
+    const int work = ((g.I + kTBM - 1) / kTBM) * ((g.J + BN - 1) / BN) * g.splits;
     unsigned int *status = device_status_word();
     if (!status) return cudaErrorMemoryAllocation;
-    tc_gemm_kernel<BN><<<tiles < sms ? tiles : sms, kTThreads, TcCfg<BN>::SMEM_BYTES, stream>>>(ma, mb, g, status);
+    tc_gemm_kernel<BN><<<work < sms ? work : sms, kTThreads, TcCfg<BN>::SMEM_BYTES, stream>>>(maps[0], maps[1], maps[2], maps[3], g, status);
     count_launch();
     return cudaGetLastError();
 }
 
-// C[I][J] = alpha * A[I][Cn] B[J][Cn]^T (+ C); lda, ldb in elements (multiples of 8), bases 16-byte aligned.
-static cudaError_t tc_gemm(const __nv_bfloat16 *A, int lda, const __nv_bfloat16 *B, int ldb, float *C, int ldc, int I, int J, int Cn,
-                           float alpha, bool accumulate, cudaStream_t stream) {
+// C[I][J] = alpha * (A B^T + A2 B2^T) (+ C).  A2.p == nullptr: one pair only.  Both pairs have the same
+// operand forms.  `partials` (splits_max * I * ldc floats) enables splitting the contraction when the
+// output has fewer tiles than the device has SMs; ldc must then be J.  Bases 16-byte aligned, ld % 8 == 0.
+static cudaError_t tc_gemm(TcOperand A, TcOperand B, int Cn, TcOperand A2, TcOperand B2, int Cn2, float *C, int ldc, int I, int J,
+                           float alpha, bool accumulate, float *partials, int splits_max, cudaStream_t stream) {
     const int BN = J > 128 ? 256 : (J > 64 ? 128 : 64);
-    CUtensorMap ma, mb;
-    if (!make_map_2d(&ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, A, (uint64_t)Cn, (uint64_t)I, (uint64_t)lda * 2, kTBK, kTBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_2d(&mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, B, (uint64_t)Cn, (uint64_t)J, (uint64_t)ldb * 2, kTBK, (uint32_t)BN, CU_TENSOR_MAP_SWIZZLE_128B))
-        return cudaErrorInvalidValue;
-    TcGemmArgs g = {C, I, J, Cn, ldc, alpha, accumulate ? 1 : 0};
-    return BN == 256 ? tc_gemm_bn<256>(ma, mb, g, stream) : (BN == 128 ? tc_gemm_bn<128>(ma, mb, g, stream) : tc_gemm_bn<64>(ma, mb, g, stream));
+    CUtensorMap maps[4];
+    if (!tc_map(&maps[0], A, I, Cn, kTBM) || !tc_map(&maps[1], B, J, Cn, BN)) return cudaErrorInvalidValue;
+    maps[2] = maps[0];
+    maps[3] = maps[1];
+    if (A2.p && (!tc_map(&maps[2], A2, I, Cn2, kTBM) || !tc_map(&maps[3], B2, J, Cn2, BN))) return cudaErrorInvalidValue;
+    TcGemmArgs g = {};
+    g.I = I; g.J = J; g.ldc = ldc;
+    g.kb1 = (Cn + kTBK - 1) / kTBK;
+    g.kb2 = A2.p ? (Cn2 + kTBK - 1) / kTBK : 0;
+    g.a_mn = A.mn; g.b_mn = B.mn;
+    const int kb_all = g.kb1 + g.kb2, tiles = ((I + kTBM - 1) / kTBM) * ((J + BN - 1) / BN), sms = device_sm_count();
+    int splits = 1;
+    if (partials && ldc == J && sms > 0 && tiles * 2 <= sms) {
+        splits = sms / tiles;
+        if (splits > splits_max) splits = splits_max;
+        if (splits > kb_all / 4) splits = kb_all / 4 > 0 ? kb_all / 4 : 1;   // at least four blocks per split
+    }
+    g.kb_per_split = (kb_all + splits - 1) / splits;
+    g.splits = (kb_all + g.kb_per_split - 1) / g.kb_per_split;  // no empty split
+    if (g.splits == 1) {
+        g.C = C; g.alpha = alpha; g.accumulate = accumulate ? 1 : 0;
+    } else {
+        g.C = partials; g.alpha = 1.0f; g.accumulate = 0;
+    }
+    cudaError_t e = BN == 256 ? tc_gemm_bn<256>(maps, g, stream) : (BN == 128 ? tc_gemm_bn<128>(maps, g, stream) : tc_gemm_bn<64>(maps, g, stream));
+    if (e != cudaSuccess || g.splits == 1) return e;
+    const size_t n4 = (size_t)I * J / 4;
+    tc_reduce_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, stream>>>((const float4 *)partials, g.splits, n4, alpha, accumulate ? 1 : 0, (float4 *)C);
+    count_launch();
+    return cudaGetLastError();
 }
 
 // ---- operand preparation ---------------------------------------------------------------------------
-// Transposes go through a 32 x 33 shared-memory tile; a block of 32 x 8 threads handles 32 x 32 elements.
-// ldt = row pitch of the transposed outputs (the row count rounded up to 8: 16-byte rows for TMA).
-
-// dY [M][N] bf16 -> dY^T [N][ldt], (dY * gamma_x[m] / 127)^T [N][ldt], and dY * gate[n] [M][N] (each nullable).
-__global__ void __launch_bounds__(256) bw_prepare_dy_kernel(const __nv_bfloat16 *dy, const float *gamma_x, const float *gate, int M, int N,
-                                                            int ldt, __nv_bfloat16 *dy_t, __nv_bfloat16 *dys_t, __nv_bfloat16 *dyg) {
-    __shared__ float tile[32][33];
-    __shared__ float tile_s[32][33];
-    const int n0 = blockIdx.x * 32, m0 = blockIdx.y * 32, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    for (int r = ty; r < 32; r += 8) {
-        const int m = m0 + r, n = n0 + tx;
-        float v = 0.0f;
-        if (m < M && n < N) v = __bfloat162float(dy[(size_t)m * N + n]);
-        tile[r][tx] = v;
-        tile_s[r][tx] = m < M ? v * (gamma_x[m] * (1.0f / 127.0f)) : 0.0f;
-        if (dyg && m < M && n < N) dyg[(size_t)m * N + n] = __float2bfloat16_rn(v * gate[n]);
+// Xd = x~ gamma_x / 127 as bf16 [M][K] (eight values per thread).
+__global__ void __launch_bounds__(256) bw_dequant_kernel(const int8_t *xq, const float *gamma_x, int K, size_t n8, __nv_bfloat16 *xd) {
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= n8) return;
+    const float s = gamma_x[(i * 8) / (size_t)K] * (1.0f / 127.0f);
+    const uint2 w = reinterpret_cast<const uint2 *>(xq)[i];
+    const uint32_t ww[2] = {w.x, w.y};
+    uint32_t o[4];
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+        const int c0 = (int)(int8_t)(ww[h >> 1] >> (16 * (h & 1))), c1 = (int)(int8_t)(ww[h >> 1] >> (16 * (h & 1) + 8));
+        const __nv_bfloat162 v = __floats2bfloat162_rn((float)c0 * s, (float)c1 * s);
+        o[h] = *reinterpret_cast<const uint32_t *>(&v);
     }
-    __syncthreads();
-    for (int r = ty; r < 32; r += 8) {
-        const int n = n0 + r, m = m0 + tx;
-        if (n < N && m < M) {
-            if (dy_t) dy_t[(size_t)n * ldt + m] = __float2bfloat16_rn(tile[tx][r]);
-            if (dys_t) dys_t[(size_t)n * ldt + m] = __float2bfloat16_rn(tile_s[tx][r]);
-        }
-    }
+    reinterpret_cast<uint4 *>(xd)[i] = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-// src [R][Cc] (bf16, fp16, int8 or fp32, by `kind` 0..3) -> dst [Cc][ldt] bf16, optionally also a plain bf16 copy [R][Cc].
-__global__ void __launch_bounds__(256) bw_transpose_kernel(const void *src, int kind, int R, int Cc, int ldt, __nv_bfloat16 *dst_t,
-                                                           __nv_bfloat16 *dst_plain) {
-    __shared__ float tile[32][33];
-    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    for (int rr = ty; rr < 32; rr += 8) {
-        const int r = r0 + rr, c = c0 + tx;
-        float v = 0.0f;
-        if (r < R && c < Cc) {
-            const size_t o = (size_t)r * Cc + c;
-            v = kind == 0 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(src)[o])
-              : kind == 1 ? __half2float(reinterpret_cast<const __half *>(src)[o])
-              : kind == 2 ? (float)reinterpret_cast<const int8_t *>(src)[o]
-                          : reinterpret_cast<const float *>(src)[o];
-            if (dst_plain) dst_plain[o] = __float2bfloat16_rn(v);
+// Ternary codes of the packed matrix as a bf16 matrix T [N][K] of -1 / 0 / +1 (one packed word = 16 columns per thread).
+__global__ void __launch_bounds__(256) bw_expand_ternary_kernel(const uint32_t *packed, int N, int K, int steps, size_t n_words,
+                                                                __nv_bfloat16 *T) {
+    const size_t w = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (w >= n_words) return;
+    const int kw = (int)(w & 15), r = (int)((w >> 4) & 15);
+    const size_t tile = w >> 8;
+    const int n = (int)(tile / steps) * 16 + r, k0 = (int)(tile % steps) * 256 + kw * 16;
+    if (n >= N || k0 >= K) return;
+    const uint32_t word = packed[w];
+    uint32_t o[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t e = (word >> (2 * j)) & 0x03030303u;
+#pragma unroll
+        for (int b = 0; b < 4; b += 2) {
+            const int c0 = (e >> (8 * b)) & 0xff, c1 = (e >> (8 * b + 8)) & 0xff;
+            const __nv_bfloat162 v = __floats2bfloat162_rn((float)(c0 == 3 ? 0 : c0 - 1), (float)(c1 == 3 ? 0 : c1 - 1));
+            o[2 * j + (b >> 1)] = *reinterpret_cast<const uint32_t *>(&v);
         }
-        tile[rr][tx] = v;
     }
-    __syncthreads();
-    for (int rr = ty; rr < 32; rr += 8) {
-        const int c = c0 + rr, r = r0 + tx;
-        if (c < Cc && r < R) dst_t[(size_t)c * ldt + r] = __float2bfloat16_rn(tile[tx][rr]);
-    }
+    uint4 *dst = reinterpret_cast<uint4 *>(T + (size_t)n * K + k0);
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
-// Ternary codes of the packed matrix as a transposed bf16 matrix T^T [K][N] of -1 / 0 / +1.  One block per
-// packed 1 KiB tile (16 rows x 256 columns): expanded into shared memory, written as 256 rows of 16 values.
-__global__ void __launch_bounds__(256) bw_expand_ternary_t_kernel(const uint32_t *packed, int N, int K, int steps, __nv_bfloat16 *Tt) {
-    __shared__ __nv_bfloat16 tile[256][16];
-    const size_t t = blockIdx.x;
-    const int n0 = (int)(t / steps) * 16, k0 = (int)(t % steps) * 256;
-    {
-        const int w = threadIdx.x, r = w >> 4, kw = w & 15;  // word w of the tile: row r, columns 16 kw ..
-        const uint32_t word = packed[t * 256 + w];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint32_t e = (word >> (2 * j)) & 0x03030303u;
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const int c = (e >> (8 * b)) & 0xff;
-                tile[16 * kw + 4 * j + b][r] = __float2bfloat16_rn((float)(c == 3 ? 0 : c - 1));
-            }
-        }
-    }
-    __syncthreads();
-    const int k = k0 + (int)threadIdx.x;
-    if (k < K) {
-        if (n0 + 16 <= N) {
-            uint4 *dst = reinterpret_cast<uint4 *>(Tt + (size_t)k * N + n0);  // N is a multiple of 8: 16-byte aligned
-            const uint4 *srcv = reinterpret_cast<const uint4 *>(&tile[threadIdx.x][0]);
-            dst[0] = srcv[0];
-            dst[1] = srcv[1];
-        } else {
-            for (int r = 0; n0 + r < N; ++r) Tt[(size_t)k * N + n0 + r] = tile[threadIdx.x][r];
-        }
-    }
+// fp16 -> bf16, optionally times a per-row factor (the gate folded into B^T).
+__global__ void __launch_bounds__(256) bw_half_to_bf16_kernel(const __half *src, const float *row_scale, int cols, size_t n, __nv_bfloat16 *dst) {
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= n) return;
+    const float s = row_scale ? row_scale[i / (size_t)cols] : 1.0f;
+    dst[i] = __float2bfloat16_rn(__half2float(src[i]) * s);
 }
 
 // Z (fp32 [M][r]) -> H = act(Z) as bf16 [M][r] and SiLU'(Z) as fp32 (in place of Z).
@@ -302,10 +357,14 @@ __global__ void __launch_bounds__(256) bw_act_kernel(float *z, size_t n, int no_
     z[i] = no_silu ? 1.0f : sg * (1.0f + v * (1.0f - sg));
 }
 
-// dZ = dH * SiLU'(Z), rounded to bf16.
-__global__ void __launch_bounds__(256) bw_dz_kernel(const float *dh, const float *dact, size_t n, __nv_bfloat16 *dz) {
+// dZ = dH * SiLU'(Z), rounded to bf16, and dZ * scale (the copy that enters dX next to gamma_W dY T).
+__global__ void __launch_bounds__(256) bw_dz_kernel(const float *dh, const float *dact, size_t n, float scale, __nv_bfloat16 *dz,
+                                                    __nv_bfloat16 *dz_scaled) {
     const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
-    if (i < n) dz[i] = __float2bfloat16_rn(dh[i] * dact[i]);
+    if (i >= n) return;
+    const float v = dh[i] * dact[i];
+    dz[i] = __float2bfloat16_rn(v);
+    dz_scaled[i] = __float2bfloat16_rn(v * scale);
 }
 
 // From G[n][j] = sum_m dY[m][n] H[m][j]: dBt[n][j] = gate[n] G[n][j] (in place), dgate[n] = sum_j G[n][j] Bt[n][j].
@@ -322,32 +381,30 @@ __global__ void __launch_bounds__(256) bw_gate_kernel(float *G, const __half *Bt
     if (dgate) dgate[n] = dg;
 }
 
+constexpr int kBwSplitsMax = 16;
+
 struct BwLayout {
-    size_t xq, gamma_x, x_t, xq_t, T_t, dy_t, dys_t, dyg, At_b, At_t, Bt_t, z, h_b, h_t, dh, dz_b, dz_t, G, total;
+    size_t xq, gamma_x, xd, T, At_b, gBt, z, h_b, dh, dz_b, dzs_b, G, partials, total;
 };
 static BwLayout bw_layout(int64_t M, int64_t K, int64_t N, int32_t r) {
     BwLayout L;
     size_t off = 0;
     auto take = [&](size_t bytes) { const size_t o = off; off += align_up(bytes, 256); return o; };
-    const size_t rr = (size_t)(r > 0 ? r : 16), Mp = (size_t)(M + 7) / 8 * 8;
+    const size_t rr = (size_t)(r > 0 ? r : 16);
     L.xq = take((size_t)M * K);
     L.gamma_x = take((size_t)M * 4);
-    L.x_t = take((size_t)K * Mp * 2);
-    L.xq_t = take((size_t)K * Mp * 2);
-    L.T_t = take((size_t)K * N * 2);
-    L.dy_t = take((size_t)N * Mp * 2);
-    L.dys_t = take((size_t)N * Mp * 2);
-    L.dyg = take((size_t)M * N * 2);
+    L.xd = take((size_t)M * K * 2);
+    L.T = take((size_t)N * K * 2);
     L.At_b = take(rr * K * 2);
-    L.At_t = take((size_t)K * rr * 2);
-    L.Bt_t = take(rr * N * 2);
+    L.gBt = take((size_t)N * rr * 2);
     L.z = take((size_t)M * rr * 4);
     L.h_b = take((size_t)M * rr * 2);
-    L.h_t = take(rr * Mp * 2);
     L.dh = take((size_t)M * rr * 4);
     L.dz_b = take((size_t)M * rr * 2);
-    L.dz_t = take(rr * Mp * 2);
+    L.dzs_b = take((size_t)M * rr * 2);
     L.G = take((size_t)N * rr * 4);
+    const size_t big = (size_t)(M > N ? (M > K ? M : K) : (N > K ? N : K));
+    L.partials = take((size_t)kBwSplitsMax * big * rr * 4);  // split contractions all have r as one output extent
     L.total = off;
     return L;
 }
@@ -379,64 +436,73 @@ extern "C" hgf_status hgf_linear_backward(const void *x, int64_t M, const void *
     if (((uintptr_t)workspace) & 255u) return HGF_ERR_MISALIGNED;
     cudaStream_t stream = (cudaStream_t)stream_;
     char *ws = (char *)workspace;
-    const int Mi = (int)M, K = (int)d_in, N = (int)d_out, Mp = (Mi + 7) / 8 * 8;
+    const int Mi = (int)M, K = (int)d_in, N = (int)d_out;
     auto bf = [&](size_t off) { return (__nv_bfloat16 *)(ws + off); };
     auto blocks1 = [](size_t n) { return (unsigned)((n + 255) / 256); };
-    auto tgrid = [](int R, int Cc) { return dim3((unsigned)((Cc + 31) / 32), (unsigned)((R + 31) / 32)); };
+    const TcOperand none = {nullptr, 0, false};
+    float *partials = (float *)(ws + L.partials);
     bool ok = true;
-    auto gemm = [&](const __nv_bfloat16 *A, int lda, const __nv_bfloat16 *B, int ldb, float *C, int ldc, int I, int J, int Cn, float alpha,
-                    bool acc) { ok = ok && tc_gemm(A, lda, B, ldb, C, ldc, I, J, Cn, alpha, acc, stream) == cudaSuccess; };
-    const bool need_t = grads->dW || (r && (grads->dAt || grads->dBt || grads->dgate));  // products that contract over the tokens
+    auto gemm = [&](TcOperand A, TcOperand B, int Cn, TcOperand A2, TcOperand B2, int Cn2, float *C, int ldc, int I, int J, float alpha,
+                    bool acc, bool may_split) {
+        ok = ok && tc_gemm(A, B, Cn, A2, B2, Cn2, C, ldc, I, J, alpha, acc, may_split ? partials : nullptr, kBwSplitsMax, stream) == cudaSuccess;
+    };
+    const TcOperand dy_k = {(const __nv_bfloat16 *)dy, N, false};  // dY as [M rows][N contraction]
+    const TcOperand dy_mn = {(const __nv_bfloat16 *)dy, N, true};  // dY as [N rows] contracted over its M stored rows
+    const TcOperand x_k = {(const __nv_bfloat16 *)x, K, false}, x_mn = {(const __nv_bfloat16 *)x, K, true};
 
-    // Algorithm 1, steps 1-2 again: the quantised activations and their scales
-    PrologueParams pp = {};
-    pp.x = (const __nv_bfloat16 *)x;
-    pp.xq = (int8_t *)(ws + L.xq);
-    pp.gamma_x = (float *)(ws + L.gamma_x);
-    pp.M = Mi;
-    pp.K = K;
-    pp.flags = HGF_FLAG_NO_PDL;
-    if (launch_quant(pp, GemmPrologueExtra{}, stream) != cudaSuccess) return HGF_ERR_CUDA;
-
-    bw_prepare_dy_kernel<<<tgrid(Mi, N), 256, 0, stream>>>((const __nv_bfloat16 *)dy, pp.gamma_x, gate, Mi, N, Mp,
-                                                           need_t ? bf(L.dy_t) : nullptr, grads->dW ? bf(L.dys_t) : nullptr,
-                                                           r ? bf(L.dyg) : nullptr);
-    count_launch();
-    if (grads->dW) {  // dW[n][k] = sum_m dYs[m][n] x~[m][k]
-        bw_transpose_kernel<<<tgrid(Mi, K), 256, 0, stream>>>(pp.xq, 2, Mi, K, Mp, bf(L.xq_t), nullptr);
+    if (grads->dW) {  // Algorithm 1, steps 1-2 again, then dW[n][k] = sum_m dY[m][n] Xd[m][k]
+        PrologueParams pp = {};
+        pp.x = (const __nv_bfloat16 *)x;
+        pp.xq = (int8_t *)(ws + L.xq);
+        pp.gamma_x = (float *)(ws + L.gamma_x);
+        pp.M = Mi;
+        pp.K = K;
+        pp.flags = HGF_FLAG_NO_PDL;
+        if (launch_quant(pp, GemmPrologueExtra{}, stream) != cudaSuccess) return HGF_ERR_CUDA;
+        const size_t n8 = (size_t)M * K / 8;
+        bw_dequant_kernel<<<blocks1(n8), 256, 0, stream>>>(pp.xq, pp.gamma_x, K, n8, bf(L.xd));
         count_launch();
-        gemm(bf(L.dys_t), Mp, bf(L.xq_t), Mp, grads->dW, K, N, K, Mi, 1.0f, false);
+        gemm(dy_mn, TcOperand{bf(L.xd), K, true}, Mi, none, none, 0, grads->dW, K, N, K, 1.0f, false, false);
     }
-    if (grads->dx) {  // dX = gamma_W (dY T)
-        const int steps = (int)(padded_k(d_in) / 256);
-        bw_expand_ternary_t_kernel<<<(unsigned)(row_tiles(d_out) * steps), 256, 0, stream>>>((const uint32_t *)packed, N, K, steps, bf(L.T_t));
-        count_launch();
-        gemm((const __nv_bfloat16 *)dy, N, bf(L.T_t), N, grads->dx, K, Mi, K, N, gamma, false);
-    }
-    if (r) {
-        float *z = (float *)(ws + L.z), *dh = (float *)(ws + L.dh), *G = grads->dBt ? grads->dBt : (float *)(ws + L.G);
-        bw_transpose_kernel<<<tgrid(r, K), 256, 0, stream>>>(At, 1, r, K, r, bf(L.At_t), bf(L.At_b));       // A^T [r][K] -> [K][r]
-        bw_transpose_kernel<<<tgrid(N, r), 256, 0, stream>>>(Bt, 1, N, r, N, bf(L.Bt_t), nullptr);          // B^T [N][r] -> [r][N]
-        count_launch(2);
-        gemm((const __nv_bfloat16 *)x, K, bf(L.At_b), K, z, r, Mi, r, K, 1.0f, false);                      // Z = x A
-        bw_act_kernel<<<blocks1((size_t)M * r), 256, 0, stream>>>(z, (size_t)M * r, (flags & HGF_FLAG_NO_SILU) ? 1 : 0, bf(L.h_b));
-        gemm(bf(L.dyg), N, bf(L.Bt_t), N, dh, r, Mi, r, N, 1.0f, false);                                    // dH = (dY g) B^T
-        bw_dz_kernel<<<blocks1((size_t)M * r), 256, 0, stream>>>(dh, z, (size_t)M * r, bf(L.dz_b));
-        count_launch(2);
-        if (grads->dx) gemm(bf(L.dz_b), r, bf(L.At_t), r, grads->dx, K, Mi, K, r, 1.0f, true);             // dX += dZ A^T
-        if (grads->dAt) {                                                                                   // dA^T = dZ^T x
-            bw_transpose_kernel<<<tgrid(Mi, r), 256, 0, stream>>>(bf(L.dz_b), 0, Mi, r, Mp, bf(L.dz_t), nullptr);
-            bw_transpose_kernel<<<tgrid(Mi, K), 256, 0, stream>>>(x, 0, Mi, K, Mp, bf(L.x_t), nullptr);
-            count_launch(2);
-            gemm(bf(L.dz_t), Mp, bf(L.x_t), Mp, grads->dAt, K, r, K, Mi, 1.0f, false);
-        }
-        if (grads->dBt || grads->dgate) {                                                                   // G = dY^T H
-            bw_transpose_kernel<<<tgrid(Mi, r), 256, 0, stream>>>(bf(L.h_b), 0, Mi, r, Mp, bf(L.h_t), nullptr);
-            count_launch();
-            gemm(bf(L.dy_t), Mp, bf(L.h_t), Mp, G, r, N, r, Mi, 1.0f, false);
-            bw_gate_kernel<<<blocks1((size_t)N), 256, 0, stream>>>(G, (const __half *)Bt, gate, N, r, grads->dgate);
+    const bool fold = gamma > 1e-20f;  // the low-rank term of dX rides in the same contraction, pre-divided by gamma_W
+    if (grads->dx || r) {
+        if (grads->dx) {
+            const int steps = (int)(padded_k(d_in) / 256);
+            const size_t n_words = (size_t)row_tiles(d_out) * steps * 256;
+            bw_expand_ternary_kernel<<<blocks1(n_words), 256, 0, stream>>>((const uint32_t *)packed, N, K, steps, n_words, bf(L.T));
             count_launch();
         }
+    }
+    const TcOperand T_mn = {bf(L.T), K, true};  // T [N][K]: rows k of the product, contracted over n
+    if (!r) {
+        if (grads->dx) gemm(dy_k, T_mn, N, none, none, 0, grads->dx, K, Mi, K, gamma, false, false);
+        return (ok && cudaGetLastError() == cudaSuccess) ? HGF_OK : HGF_ERR_CUDA;
+    }
+    float *z = (float *)(ws + L.z), *dh = (float *)(ws + L.dh), *G = grads->dBt ? grads->dBt : (float *)(ws + L.G);
+    bw_half_to_bf16_kernel<<<blocks1((size_t)r * K), 256, 0, stream>>>((const __half *)At, nullptr, K, (size_t)r * K, bf(L.At_b));
+    bw_half_to_bf16_kernel<<<blocks1((size_t)N * r), 256, 0, stream>>>((const __half *)Bt, gate, r, (size_t)N * r, bf(L.gBt));
+    count_launch(2);
+    const TcOperand At_k = {bf(L.At_b), K, false}, At_mn = {bf(L.At_b), K, true};
+    gemm(x_k, At_k, K, none, none, 0, z, r, Mi, r, 1.0f, false, true);                                       // Z = x A
+    bw_act_kernel<<<blocks1((size_t)M * r), 256, 0, stream>>>(z, (size_t)M * r, (flags & HGF_FLAG_NO_SILU) ? 1 : 0, bf(L.h_b));
+    gemm(dy_k, TcOperand{bf(L.gBt), r, true}, N, none, none, 0, dh, r, Mi, r, 1.0f, false, true);            // dH = dY (g (.) B^T)
+    bw_dz_kernel<<<blocks1((size_t)M * r), 256, 0, stream>>>(dh, z, (size_t)M * r, fold ? 1.0f / gamma : 1.0f, bf(L.dz_b), bf(L.dzs_b));
+    count_launch(2);
+    if (grads->dx) {                                                                                         // dX = gamma_W dY T + dZ A^T
+        const TcOperand dzs_k = {bf(L.dzs_b), r, false};
+        if (fold) {
+            gemm(dy_k, T_mn, N, dzs_k, At_mn, r, grads->dx, K, Mi, K, gamma, false, false);
+        } else {
+            gemm(dy_k, T_mn, N, none, none, 0, grads->dx, K, Mi, K, gamma, false, false);
+            gemm(dzs_k, At_mn, r, none, none, 0, grads->dx, K, Mi, K, 1.0f, true, false);
+        }
+    }
+    if (grads->dAt)                                                                                          // dA^T[j][k] = sum_m dZ[m][j] x[m][k]
+        gemm(TcOperand{bf(L.dz_b), r, true}, x_mn, Mi, none, none, 0, grads->dAt, K, r, K, 1.0f, false, true);
+    if (grads->dBt || grads->dgate) {                                                                        // G[n][j] = sum_m dY[m][n] H[m][j]
+        gemm(dy_mn, TcOperand{bf(L.h_b), r, true}, Mi, none, none, 0, G, r, N, r, 1.0f, false, true);
+        bw_gate_kernel<<<blocks1((size_t)N), 256, 0, stream>>>(G, (const __half *)Bt, gate, N, r, grads->dgate);
+        count_launch();
     }
     return (ok && cudaGetLastError() == cudaSuccess) ? HGF_OK : HGF_ERR_CUDA;
 }

@@ -335,9 +335,15 @@ def check_status(stream=None) -> None:
     _check("hgf_check_status", lib().hgf_check_status(_stream(stream)))
 
 
-def linear_backward(x, packed, gamma, d_in, d_out, dy, At=None, Bt=None, gate=None, *, flags=0, stream=None, want=None):
+def backward_workspace_bytes(M, d_in, d_out, r) -> int:
+    return int(lib().hgf_backward_workspace_bytes(M, d_in, d_out, r))
+
+
+def linear_backward(x, packed, gamma, d_in, d_out, dy, At=None, Bt=None, gate=None, *, flags=0, stream=None, want=None,
+                    out=None, workspace=None):
     """hgf_linear_backward: straight-through backward pass.  dy bf16 [M][d_out].  Returns a dict of fp32 device
-    tensors dx, dW and (with a correction) dAt, dBt, dgate; `want` restricts which are computed."""
+    tensors dx, dW and (with a correction) dAt, dBt, dgate; `want` restricts which are computed.  `out` (a dict
+    returned by an earlier call of the same shape) and `workspace` are reused when given."""
     assert x.is_cuda and x.dtype == torch.bfloat16 and dy.dtype == torch.bfloat16 and x.is_contiguous() and dy.is_contiguous()
     M = x.shape[0]
     r = 0 if At is None else At.shape[0]
@@ -345,12 +351,18 @@ def linear_backward(x, packed, gamma, d_in, d_out, dy, At=None, Bt=None, gate=No
     if want is not None:
         names = [n for n in names if n in want]
     shapes = {"dx": (M, d_in), "dW": (d_out, d_in), "dAt": (r, d_in), "dBt": (d_out, r), "dgate": (d_out,)}
-    out = {n: torch.empty(shapes[n], dtype=torch.float32, device=x.device) for n in names}
+    if out is None:
+        out = {n: torch.empty(shapes[n], dtype=torch.float32, device=x.device) for n in names}
+    else:
+        assert all(n in out and tuple(out[n].shape) == shapes[n] and out[n].dtype == torch.float32 for n in names)
+        workspace = workspace if workspace is not None else out.get("_workspace")
     g = Grads(*[out[n].data_ptr() if n in out else None for n in ("dx", "dW", "dAt", "dBt", "dgate")])
-    ws = torch.empty(int(lib().hgf_backward_workspace_bytes(M, d_in, d_out, r)), dtype=torch.uint8, device=x.device)
+    need = backward_workspace_bytes(M, d_in, d_out, r)
+    ws = workspace if workspace is not None and workspace.numel() >= need else torch.empty(need, dtype=torch.uint8, device=x.device)
     _check("hgf_linear_backward",
            lib().hgf_linear_backward(_ptr(x), M, _ptr(packed), ctypes.c_float(gamma), d_in, d_out, _ptr(At), _ptr(Bt), r, _ptr(gate),
                                      _ptr(dy), ctypes.byref(g), _ptr(ws), ws.numel(), flags, _stream(stream)))
+    out = dict(out)
     out["_workspace"] = ws
     return out
 
