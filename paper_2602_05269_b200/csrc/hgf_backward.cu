@@ -50,14 +50,6 @@ struct TcCfg {
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
 };
 
-// Shared-memory descriptor of an MN-major tile with the 128-byte swizzle: 64 operand rows x 8 contraction
-// rows per 1 KiB swizzle atom; leading byte offset (bits 16-29) = distance between 64-row blocks (one TMA
-// box), stride byte offset (32-45) = distance between groups of 8 contraction rows.
-__device__ __forceinline__ uint64_t make_sw128_mn_desc(uint32_t saddr) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(kTBox >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
-           (2ull << 61);
-}
-
 template <int BN>
 __global__ void __launch_bounds__(kTThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -156,8 +148,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     if (!(ok = mbar_wait(bar(C::BAR_FULL + s), ph, abort_flag, status, 0x820u + s))) break;
                     tc_fence_after();
                     const uint32_t sa = sbase + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
-                    const uint64_t adesc = g.a_mn ? make_sw128_mn_desc(sa) : make_sw128_desc(sa);
-                    const uint64_t bdesc = g.b_mn ? make_sw128_mn_desc(sb) : make_sw128_desc(sb);
+                    const uint64_t adesc = g.a_mn ? make_sw128_mn_desc(sa, kTBox) : make_sw128_desc(sa);
+                    const uint64_t bdesc = g.b_mn ? make_sw128_mn_desc(sb, kTBox) : make_sw128_desc(sb);
 #pragma unroll
                     for (int kk = 0; kk < kTBK / 16; ++kk)
                         mma_f16(acc, adesc + (uint64_t)(a_step * kk), bdesc + (uint64_t)(b_step * kk), idesc, (kb > lo || kk) ? 1u : 0u);
