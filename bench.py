@@ -647,7 +647,7 @@ def run_extra(hgf, torch, syn, stream, args, peaks, int8_peak_measured=None):
     extra["diff_attention"] = {"workload": f"causal differential attention forward, B={B_}, L={L_}, {h_} heads of {dh_}, bf16",
                                "ms": ms, "TFLOP/s": at_flops / (ms * 1e-3) / 1e12,
                                "frac_measured_bf16": at_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                               "note": "warp-level MMA kernel built for parity (a 'next' row), not tuned"}
+                               "note": "tcgen05 kernel (a 'next' row): scores and outputs in tensor memory, one softmax thread per row and stream"}
     del qa, ka, va, oa
     torch.cuda.empty_cache()
 
