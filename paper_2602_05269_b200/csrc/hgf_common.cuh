@@ -120,6 +120,7 @@ struct GemmPrologueExtra {
     int N;
     int tokens_per_block;    // set by the launcher of the GEMM path's prologue kernel
     int gate_group;          // channels per gate value (1 = one per channel)
+    int split_round;         // set by the launcher: the rounding pass runs as a launch of its own (round_rows_kernel)
 };
 
 // LayerNorm front end (Appendix E of the paper): parameters and where the statistics go.
