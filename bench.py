@@ -464,7 +464,7 @@ DECODE_TRAFFIC = {"source_sha1": "7b2cc479563a0d062a4c3a356e67630e5471a690",
 # DRAM traffic of the prefill GEMM launch from one ncu capture of the very shape the bench times
 # (2048 -> 5632, r = 32, M = 8192, bf16 y): dram__bytes_read.sum + dram__bytes_write.sum of one launch.  Below
 # the launch's algorithmic bytes because most of y is still in L2 when the kernel ends.
-PREFILL_TRAFFIC = {"source_sha1": "820e55be152b4392c9290353ebaab2bf22b8e090", "dram_bytes_per_launch": 21.571072e6 + 43.429632e6}
+PREFILL_TRAFFIC = {"source_sha1": "1aa0a24ce7a1e6dbd36de8d29d9bd7518719bb4f", "dram_bytes_per_launch": 21.568768e6 + 43.333632e6}
 
 
 def prefill_traffic():
@@ -761,6 +761,8 @@ def run_profile_case(spec: str, reps: int):
 
     parts = spec.split(":")
     dims = [int(v) for v in parts[1].split("x")]
+    if parts[0] in ("attention", "backward"):
+        return run_profile_next_rows(parts[0], dims, reps)
     K, N, M = dims[:3]
     r = dims[3] if len(dims) > 3 else 32
     flags = hgf.FLAG_OUT_BF16 if (len(parts) > 2 and parts[2] == "bf16") else 0
@@ -774,6 +776,41 @@ def run_profile_case(spec: str, reps: int):
         stream.synchronize()
     hgf.check_status(stream)
     print(json.dumps({"profile_case": spec, "reps": reps, "launches": hgf.launch_count()}))
+
+
+def run_profile_next_rows(kind, dims, reps):
+    """`attention:BxLxhxdh` (differential attention forward, bf16 output) or `backward:KxNxMxr` (straight-through
+    backward of one layer, all five gradients): plain launches for use under a profiler."""
+    import torch
+
+    from paper_2602_05269_b200 import hgf, inputs as syn
+
+    torch.cuda.set_device(0)
+    stream = torch.cuda.Stream()
+    g = torch.Generator(device="cuda")
+    g.manual_seed(7)
+    if kind == "attention":
+        B, L, h, dh = dims
+        q = torch.randn((B * L, 2 * h * dh), generator=g, device="cuda").to(torch.bfloat16)
+        k = torch.randn((B * L, 2 * h * dh), generator=g, device="cuda").to(torch.bfloat16)
+        v = torch.randn((B * L, h * dh), generator=g, device="cuda").to(torch.bfloat16)
+        o = torch.empty((B * L, h * dh), dtype=torch.bfloat16, device="cuda")
+        with torch.cuda.stream(stream):
+            for _ in range(reps):
+                hgf.diff_attention_forward(q, k, v, B, L, h, dh, 0.8, out=o, flags=hgf.FLAG_OUT_BF16, stream=stream)
+            stream.synchronize()
+    else:
+        K, N, M, r = dims
+        w = Workload(hgf, torch, [syn.LayerShape("p", K, N, r)], M, 1)
+        (_s, x, packed, gamma, At, Bt, gate, _y) = w.layers[0]
+        dy = torch.randn((M, N), generator=g, device="cuda").to(torch.bfloat16)
+        keep = None
+        with torch.cuda.stream(stream):
+            for _ in range(reps):
+                keep = hgf.linear_backward(x, packed, gamma, K, N, dy, At, Bt, gate, stream=stream, out=keep)
+            stream.synchronize()
+    hgf.check_status(stream)
+    print(json.dumps({"profile_case": kind, "dims": dims, "reps": reps, "launches": hgf.launch_count()}))
 
 
 def run_profile_group(spec: str, reps: int):

@@ -62,6 +62,23 @@ def test_listing_scale_bf16_output_and_peaked_scores(hgf):
     assert abs(hgf.diff_lambda0(64) - oracle.lambda0(64)) < 1e-15
 
 
+@pytest.mark.parametrize("dh", [64, 128])
+def test_scores_that_grow_along_the_sequence(hgf, dh):
+    """Keys whose magnitude grows with their position: the row maxima keep moving, by far more than the slack
+    within which the kernel keeps an old reference point, so the accumulated outputs and sums are rescaled in
+    tensor memory at many key tiles (and not at others)."""
+    B, L, h, lam = 1, 700, 2, 0.8
+    rng = np.random.default_rng([67, dh])
+    grow = np.linspace(0.3, 7.0, L, dtype=np.float32)[:, None]
+    q = syn.f32_to_bf16_bits(rng.standard_normal((L, 2 * h * dh)).astype(np.float32))
+    k = syn.f32_to_bf16_bits((rng.standard_normal((L, 2 * h * dh)) * grow).astype(np.float32))
+    v = syn.f32_to_bf16_bits(rng.standard_normal((L, h * dh)).astype(np.float32))
+    out = hgf.diff_attention_forward(_dev(q), _dev(k), _dev(v), B, L, h, dh, lam).float().cpu().numpy()
+    ref = oracle.diff_attention(q, k, v, B, L, h, dh, lam)
+    assert np.isfinite(out).all()
+    assert np.abs(out - ref).max() <= 4e-3 * (1 + lam) * np.abs(syn.bf16_bits_to_f32(v)).max()
+
+
 def test_properties_at_model_size(hgf):
     """d = 2048, 16 heads of 64 (the 1.2B-class block), L = 2048: too long for the oracle in full, so
     the first 256 tokens are compared with it (causality makes them independent of the rest) and the
