@@ -360,17 +360,20 @@ __global__ void __launch_bounds__(256) bw_dz_kernel(const float *dh, const float
 }
 
 // From G[n][j] = sum_m dY[m][n] H[m][j]: dBt[n][j] = gate[n] G[n][j] (in place), dgate[n] = sum_j G[n][j] Bt[n][j].
+// One warp per output channel n (its r values are contiguous).
 __global__ void __launch_bounds__(256) bw_gate_kernel(float *G, const __half *Bt, const float *gate, int N, int r, float *dgate) {
-    const int n = blockIdx.x * 256 + threadIdx.x;
+    const int n = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (n >= N) return;
     float dg = 0.0f;
     const float gn = gate[n];
-    for (int j = 0; j < r; ++j) {
+    for (int j = lane; j < r; j += 32) {
         const float v = G[(size_t)n * r + j];
         dg = fmaf(v, __half2float(Bt[(size_t)n * r + j]), dg);
         G[(size_t)n * r + j] = gn * v;
     }
-    if (dgate) dgate[n] = dg;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dg += __shfl_xor_sync(0xffffffffu, dg, o);
+    if (dgate && lane == 0) dgate[n] = dg;
 }
 
 constexpr int kBwSplitsMax = 16;
@@ -493,7 +496,7 @@ extern "C" hgf_status hgf_linear_backward(const void *x, int64_t M, const void *
         gemm(TcOperand{bf(L.dz_b), r, true}, x_mn, Mi, none, none, 0, grads->dAt, K, r, K, 1.0f, false, true);
     if (grads->dBt || grads->dgate) {                                                                        // G[n][j] = sum_m dY[m][n] H[m][j]
         gemm(dy_mn, TcOperand{bf(L.h_b), r, true}, Mi, none, none, 0, G, r, N, r, 1.0f, false, true);
-        bw_gate_kernel<<<blocks1((size_t)N), 256, 0, stream>>>(G, (const __half *)Bt, gate, N, r, grads->dgate);
+        bw_gate_kernel<<<(unsigned)((N + 7) / 8), 256, 0, stream>>>(G, (const __half *)Bt, gate, N, r, grads->dgate);
         count_launch();
     }
     return (ok && cudaGetLastError() == cudaSuccess) ? HGF_OK : HGF_ERR_CUDA;
