@@ -273,6 +273,25 @@ def test_gemm_long_rows_without_correction_and_without_dependent_launch(hgf):
     assert torch.equal(y1, y2)
 
 
+@pytest.mark.parametrize("M,K", [(1536, 2048), (2304, 2048), (600, 5632), (800, 5632)])
+def test_gemm_path_quantises_every_row_like_the_oracle(hgf, M, K):
+    """Every row's codes and scale on the GEMM path against the oracle's quantiser (Algorithm 1, steps 1-2): the
+    prefill tests above look at sampled rows only.  6 MB of x keeps the rounding pass inside the prologue
+    kernel, 9 MB makes it the launch of its own (one warp per row), K = 5632 has rows longer than one pass
+    of a warp's unrolled loop."""
+    shape = syn.LayerShape("p", K, 256, 32)
+    packed, gamma, T = packed_layer(hgf, shape, 3, 11)
+    x = syn.make_x(M, K, config=3, layer=11)
+    x[5] = 0
+    At, Bt, gate = syn.make_lora(K, 256, 32, config=3, layer=11)
+    y, dbg = hgf.linear_forward(dev(x, torch.bfloat16), packed, float(gamma), K, 256, dev(At, torch.float16),
+                                dev(Bt, torch.float16), dev(gate), debug=True)
+    hgf.check_status()
+    ref = oracle.act_quant(x)
+    assert np.array_equal(dbg["xq"].cpu().numpy(), ref[0]), "quantised activations differ"
+    assert np.array_equal(dbg["gamma_x"].cpu().numpy(), ref[1]), "per-token scales differ"
+
+
 def test_config3_prefill_m512_full(hgf):
     for i, shape in enumerate(syn.distinct_shapes(3)):
         check_layer(hgf, shape, 512, config=3, layer=i, tol2=TOL_GEMM)
