@@ -352,10 +352,13 @@ double hgf_diff_lambda0(double head_dim);
  * (dgate is with respect to the evaluated gate g; d alpha = dgate (1 - g^2) is the caller's.)
  * x, packed, gamma, At, Bt, gate as in the forward call; dy [M][d_out] bfloat16.  Every output is fp32
  * and nullable (skipped).  The matrix products run on the tensor cores with bf16 operands and fp32
- * accumulation (the precision the paper trains in): x~ and t enter exactly, dY scaled by gamma_x / 127
- * or by g, A, B, H and dZ rounded to bf16.  Requirements: d_in % 64 == 0, d_out % 8 == 0, r in
- * {0,16,32,48,64}; 16-byte aligned pointers; workspace of hgf_backward_workspace_bytes(...) bytes,
- * 256-byte aligned.  Flags: HGF_FLAG_NO_SILU.  Enqueue only.
+ * accumulation (the precision the paper trains in): dY, x and t enter exactly; Xd, A, g (.) B, H, dZ and
+ * dZ / gamma_W (the low-rank term of dX is accumulated together with dY t and the sum scaled by gamma_W)
+ * are rounded to bf16.  Requirements: d_in % 64 == 0, d_out % 8 == 0, M <= 2^22, r in {0,16,32,48,64};
+ * 16-byte aligned pointers; workspace of hgf_backward_workspace_bytes(...) bytes, 256-byte aligned (it
+ * holds the operands above and the partial sums of the thin products; its contents are scratch).
+ * Flags: HGF_FLAG_NO_SILU.  Enqueue only; errors of the launches come back as HGF_ERR_CUDA, a bounded
+ * wait that ran out through hgf_check_status.
  */
 typedef struct {
     float *dx;

@@ -460,13 +460,11 @@ extern "C" hgf_status hgf_linear_backward(const void *x, int64_t M, const void *
         gemm(dy_mn, TcOperand{bf(L.xd), K, true}, Mi, none, none, 0, grads->dW, K, N, K, 1.0f, false, false);
     }
     const bool fold = gamma > 1e-20f;  // the low-rank term of dX rides in the same contraction, pre-divided by gamma_W
-    if (grads->dx || r) {
-        if (grads->dx) {
-            const int steps = (int)(padded_k(d_in) / 256);
-            const size_t n_words = (size_t)row_tiles(d_out) * steps * 256;
-            bw_expand_ternary_kernel<<<blocks1(n_words), 256, 0, stream>>>((const uint32_t *)packed, N, K, steps, n_words, bf(L.T));
-            count_launch();
-        }
+    if (grads->dx) {
+        const int steps = (int)(padded_k(d_in) / 256);
+        const size_t n_words = (size_t)row_tiles(d_out) * steps * 256;
+        bw_expand_ternary_kernel<<<blocks1(n_words), 256, 0, stream>>>((const uint32_t *)packed, N, K, steps, n_words, bf(L.T));
+        count_launch();
     }
     const TcOperand T_mn = {bf(L.T), K, true};  // T [N][K]: rows k of the product, contracted over n
     if (!r) {
