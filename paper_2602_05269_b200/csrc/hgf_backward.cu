@@ -33,6 +33,7 @@ struct TcGemmArgs {
     int I, J, ldc;
     int kb1, kb2;      // 64-element contraction blocks of the first and of the second operand pair
     int splits, kb_per_split;
+    int n_half;        // splits == 1 only: the last n_half / 2 tiles are worked as halves of BN / 2 columns (see tc_gemm)
     int a_mn, b_mn;    // operand forms (both pairs alike)
     float alpha;
     int accumulate;
@@ -64,10 +65,27 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_BAR + C::BAR_COUNT * 8 + 4);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int tiles_i = (g.I + kTBM - 1) / kTBM, tiles_j = (g.J + BN - 1) / BN, tiles_ij = tiles_i * tiles_j;
-    const int num_work = tiles_ij * g.splits, kb_all = g.kb1 + g.kb2;
-    // work item w: output tile w % tiles_ij, contraction blocks [kb_lo, kb_hi) of split w / tiles_ij
-    auto kb_lo = [&](int w) { return (w / tiles_ij) * g.kb_per_split; };
-    auto kb_hi = [&](int w) { const int e = (w / tiles_ij + 1) * g.kb_per_split; return e < kb_all ? e : kb_all; };
+    const int n_full = tiles_ij - g.n_half / 2;  // tiles worked whole (all of them unless n_half > 0)
+    const int num_work = g.n_half ? n_full + g.n_half : tiles_ij * g.splits, kb_all = g.kb1 + g.kb2;
+    // work item w: output tile w % tiles_ij, contraction blocks [kb_lo, kb_hi) of split w / tiles_ij; with
+    // half tiles (one split): items past n_full are the two halves of the remaining tiles, in turn
+    auto kb_lo = [&](int w) { return g.n_half ? 0 : (w / tiles_ij) * g.kb_per_split; };
+    auto kb_hi = [&](int w) {
+        if (g.n_half) return kb_all;
+        const int e = (w / tiles_ij + 1) * g.kb_per_split;
+        return e < kb_all ? e : kb_all;
+    };
+    auto tile_of = [&](int w, int &i0, int &j0, int &bn) {
+        int tile = w % tiles_ij, half = 0;
+        bn = BN;
+        if (g.n_half && w >= n_full) {
+            tile = n_full + (w - n_full) / 2;
+            half = (w - n_full) & 1;
+            bn = BN / 2;
+        }
+        i0 = (tile / tiles_j) * kTBM;
+        j0 = (tile % tiles_j) * BN + half * (BN / 2);
+    };
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
@@ -99,7 +117,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         uint32_t issued[C::STAGES] = {};
         bool ok = true;
         for (int w = blockIdx.x; ok && w < num_work; w += gridDim.x) {
-            const int tile = w % tiles_ij, i0 = (tile / tiles_j) * kTBM, j0 = (tile % tiles_j) * BN;
+            int i0, j0, bn;
+            tile_of(w, i0, j0, bn);
             for (int kb = kb_lo(w); kb < kb_hi(w); ++kb) {
                 ok = mbar_wait(bar(C::BAR_EMPTY + s), ph ^ 1u, abort_flag, status, 0x800u + s);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;
@@ -108,14 +127,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     const CUtensorMap *ma = second ? &tmap_a2 : &tmap_a, *mb = second ? &tmap_b2 : &tmap_b;
                     const int c0 = (second ? kb - g.kb1 : kb) * kTBK;
                     const uint32_t dst_a = sbase + s * C::STAGE_BYTES, dst_b = dst_a + C::A_BYTES, full = bar(C::BAR_FULL + s);
-                    mbar_arrive_expect_tx(full, C::STAGE_BYTES);
+                    mbar_arrive_expect_tx(full, C::A_BYTES + (g.b_mn ? bn * 128 : C::B_BYTES));  // (a K-major box always has BN rows)
                     if (g.a_mn) {
                         for (int h = 0; h < kTBM / 64; ++h) tma_load_2d(dst_a + h * kTBox, ma, i0 + 64 * h, c0, full);
                     } else {
                         tma_load_2d(dst_a, ma, c0, i0, full);
                     }
                     if (g.b_mn) {
-                        for (int h = 0; h < BN / 64; ++h) tma_load_2d(dst_b + h * kTBox, mb, j0 + 64 * h, c0, full);
+                        for (int h = 0; h < bn / 64; ++h) tma_load_2d(dst_b + h * kTBox, mb, j0 + 64 * h, c0, full);
                     } else {
                         tma_load_2d(dst_b, mb, c0, j0, full);
                     }
@@ -144,6 +163,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     break;
                 tc_fence_after();
                 const int lo = kb_lo(w), hi = kb_hi(w);
+                int ti0, tj0, bn;
+                tile_of(w, ti0, tj0, bn);
+                const uint32_t idesc_w = (idesc & ~(0x3fu << 17)) | ((uint32_t)(bn >> 3) << 17);
                 for (int kb = lo; kb < hi; ++kb) {
                     if (!(ok = mbar_wait(bar(C::BAR_FULL + s), ph, abort_flag, status, 0x820u + s))) break;
                     tc_fence_after();
@@ -152,7 +174,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     const uint64_t bdesc = g.b_mn ? make_sw128_mn_desc(sb, kTBox) : make_sw128_desc(sb);
 #pragma unroll
                     for (int kk = 0; kk < kTBK / 16; ++kk)
-                        mma_f16(acc, adesc + (uint64_t)(a_step * kk), bdesc + (uint64_t)(b_step * kk), idesc, (kb > lo || kk) ? 1u : 0u);
+                        mma_f16(acc, adesc + (uint64_t)(a_step * kk), bdesc + (uint64_t)(b_step * kk), idesc_w, (kb > lo || kk) ? 1u : 0u);
                     tc_commit(bar(C::BAR_EMPTY + s));
                     if (++s == C::STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -166,8 +188,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         bool ok = true;
         int it = 0;
         for (int w = blockIdx.x; ok && w < num_work; w += gridDim.x, ++it) {
-            const int tile = w % tiles_ij, i0 = (tile / tiles_j) * kTBM, j0 = (tile % tiles_j) * BN;
-            float *Cw = g.C + (size_t)(w / tiles_ij) * g.I * g.ldc;
+            int i0, j0, bn;
+            tile_of(w, i0, j0, bn);
+            float *Cw = g.C + (g.n_half ? (size_t)0 : (size_t)(w / tiles_ij) * g.I * g.ldc);
             const int b = it & 1;
             ok = mbar_wait(bar(C::BAR_ACCFULL + b), (uint32_t)(it >> 1) & 1u, abort_flag, status, 0x830u);
             if (!(ok = __all_sync(0xffffffffu, ok))) break;
@@ -175,7 +198,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int i = i0 + 32 * q + lane;  // this thread's row of C = its tensor-memory lane
             const uint32_t lane_base = tmem_base + ((uint32_t)(32 * q) << 16) + b * BN;
             const bool empty = kb_lo(w) >= kb_hi(w);  // a split past the end of the contraction: zeros
-            for (int cc = 0; cc < BN; cc += 32) {
+            for (int cc = 0; cc < bn; cc += 32) {
                 if (j0 + cc >= g.J) break;  // (warp-uniform)
                 uint32_t v[32];
                 tmem_ld32(lane_base + cc, v);
@@ -241,7 +264,8 @@ static cudaError_t tc_gemm_bn(const CUtensorMap *maps, const TcGemmArgs &g, cuda
     if (e != cudaSuccess) return e;
     const int sms = device_sm_count();
     if (!sms) return cudaErrorInvalidDevice;
-    const int work = ((g.I + kTBM - 1) / kTBM) * ((g.J + BN - 1) / BN) * g.splits;
+    const int tiles = ((g.I + kTBM - 1) / kTBM) * ((g.J + BN - 1) / BN);
+    const int work = g.n_half ? tiles + g.n_half / 2 : tiles * g.splits;
     unsigned int *status = device_status_word();
     if (!status) return cudaErrorMemoryAllocation;
     tc_gemm_kernel<BN><<<work < sms ? work : sms, kTThreads, TcCfg<BN>::SMEM_BYTES, stream>>>(maps[0], maps[1], maps[2], maps[3], g, status);
@@ -272,6 +296,11 @@ static cudaError_t tc_gemm(TcOperand A, TcOperand B, int Cn, TcOperand A2, TcOpe
         if (splits > splits_max) splits = splits_max;
         if (splits > kb_all / 4) splits = kb_all / 4 > 0 ? kb_all / 4 : 1;   // at least four blocks per split
     }
+    // Tail of the tile schedule: when the tiles left for the last round of the persistent CTAs would keep at most
+    // half of the SMs busy, they are worked as twice as many tiles of half the width, which fills the round.
+    if (splits == 1 && BN == 256 && B.mn && sms > 0 && tiles > sms && tiles % sms != 0 && 2 * (tiles % sms) <= sms &&
+        J % 256 == 0)
+        g.n_half = 2 * (tiles % sms);
     g.kb_per_split = (kb_all + splits - 1) / splits;
     g.splits = (kb_all + g.kb_per_split - 1) / g.kb_per_split;  // no empty split
     if (g.splits == 1) {

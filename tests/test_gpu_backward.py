@@ -65,6 +65,15 @@ def test_pure_ternary_layer_no_silu_and_selected_outputs(hgf):
     check(hgf, 150, 512, 256, 32, layer=4, want=("dx", "dgate"))
 
 
+def test_more_tiles_than_sms_with_a_ragged_last_round(hgf):
+    """dW of 2560 x 2048 and dX of 2560 x 2048 are 160 output tiles of 128 x 256 each: more than the SMs of the
+    part, with a last round of the persistent schedule that the kernel works as twice as many half-width tiles.
+    The small other extent keeps the oracle affordable."""
+    check(hgf, 64, 2048, 2560, 32, layer=6)    # dW [2560][2048]
+    check(hgf, 2560, 2048, 64, 32, layer=7)    # dX [2560][2048], with the low-rank term in the same contraction
+    check(hgf, 2560, 2048, 64, 0, layer=8, lora=False)
+
+
 def test_decode_sized_batch(hgf):
     check(hgf, 4, 2048, 512, 32, layer=5)
 
