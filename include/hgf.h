@@ -50,7 +50,7 @@ typedef enum {
                                     path on decode-sized inputs) */
 
 #define HGF_FLAG_NO_PDL 0x8u     /* do not use programmatic dependent launch (see hgf_linear_forward) */
-#define HGF_FLAG_BASE3 0x10u     /* `packed` is in the base-3 layout of hgf_pack_ternary_b3 (decode path only) */
+#define HGF_FLAG_BASE3 0x10u     /* `packed` is in the base-3 layout of hgf_pack_ternary_b3 */
 
 /* Largest token count the register-resident decode path handles; above it the GEMM path runs. */
 #define HGF_DECODE_MAX_M 16
@@ -101,9 +101,12 @@ hgf_status hgf_unpack_ternary(const void *packed, int64_t d_out, int64_t d_in, i
  * c0 + 3 c1 + 9 c2 + 27 c3 + 81 c4 (0..242), the nearest byte-aligned packing to the log2(3) = 1.58
  * bits the paper counts per ternary weight (Introduction, the T_max bound; Section 4.2, the
  * effective bit-width).  It takes a fifth off the weight stream of the memory-bound decode path at
- * the price of a table look-up per byte; forward calls take it with HGF_FLAG_BASE3, on the decode
- * path only (M <= HGF_DECODE_MAX_M; the compute-bound GEMM path wants the two-bit layout and returns
- * HGF_ERR_UNSUPPORTED_SHAPE).
+ * the price of a table look-up per byte; forward calls take it with HGF_FLAG_BASE3.  The decode
+ * path (M <= HGF_DECODE_MAX_M) computes straight from the base-3 bytes.  The compute-bound GEMM path
+ * reads two-bit tiles: given base-3 weights, hgf_linear_forward first rewrites the layer's tiles into
+ * its workspace (one small launch; hgf_workspace_bytes with the flag includes the room), so a model
+ * stored at 1.6 bits needs no second copy of its weights for prefill.  Groups and the allocation-free
+ * entry point take base-3 weights on the decode path only.
  * Layout: tiles of 16 output rows by 320 input columns (d_out padded to 16, d_in to 320, with zero
  * weights); a tile is 1024 bytes, its 16 rows one after the other, 64 bytes per row; tile (R, C)
  * starts at byte (R * (d_in_padded / 320) + C) * 1024.  Byte q = 16 t + j (t in 0..3, j in 0..15) of a

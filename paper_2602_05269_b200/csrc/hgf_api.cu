@@ -63,7 +63,7 @@ using namespace hgf;
 
 extern "C" size_t hgf_workspace_bytes(int64_t M, int64_t d_in, int64_t d_out, int32_t r, uint32_t flags) {
     if (M <= 0 || d_in <= 0 || d_in > 65536 || r < 0) return 256;
-    return ws_layout(M, d_in, d_out, r, takes_gemm_path(M, d_in, flags)).total;
+    return ws_layout(M, d_in, d_out, r, takes_gemm_path(M, d_in, flags), (flags & HGF_FLAG_BASE3) != 0).total;
 }
 
 extern "C" hgf_status hgf_act_quant(const void *x, int64_t M, int64_t d_in, int8_t *xq, float *gamma_x,
@@ -95,7 +95,6 @@ static hgf_status validate_problem(const void *x, int64_t M, const void *packed,
     if (r != 0 && r != 16 && r != 32 && r != 48 && r != 64) return HGF_ERR_UNSUPPORTED_SHAPE;
     *gemm = takes_gemm_path(M, d_in, flags);
     if (*gemm && (d_out % 8 != 0)) return HGF_ERR_UNSUPPORTED_SHAPE;
-    if (*gemm && (flags & HGF_FLAG_BASE3)) return HGF_ERR_UNSUPPORTED_SHAPE;  // base-3 weights serve the byte-bound decode path
     if (misaligned(x) || misaligned(packed) || misaligned(y) || misaligned(At) || misaligned(Bt) || misaligned(gate))
         return HGF_ERR_MISALIGNED;
     *r_eff = r;
@@ -221,7 +220,7 @@ hgf_status hgf::forward_impl(const void *x, int64_t M, const void *packed, float
     if (st != HGF_OK) return st;
     if (dbg && (misaligned(dbg->xq) || misaligned(dbg->gamma_x) || misaligned(dbg->y_int) || misaligned(dbg->h)))
         return HGF_ERR_MISALIGNED;
-    const WsLayout L = ws_layout(M, d_in, d_out, r, gemm);
+    const WsLayout L = ws_layout(M, d_in, d_out, r, gemm, (flags & HGF_FLAG_BASE3) != 0);
     if (!workspace || workspace_bytes < L.total) return HGF_ERR_WORKSPACE;
     if (((uintptr_t)workspace) & 255u) return HGF_ERR_MISALIGNED;
     cudaStream_t stream = (cudaStream_t)stream_;
@@ -255,6 +254,14 @@ hgf_status hgf::forward_impl(const void *x, int64_t M, const void *packed, float
         return launch_decode_gemv(dl, &dp, pdl, stream) == cudaSuccess ? HGF_OK : HGF_ERR_CUDA;
     }
 
+    // Base-3 weights on the GEMM path: the tensor-core kernel reads two-bit tiles, so the layer's tiles are
+    // rewritten from the base-3 bytes into the workspace first (a few microseconds; the prefill is bound by
+    // arithmetic, not by the weight bytes the base-3 layout saves).
+    const void *packed2 = packed;
+    if (do_main && (flags & HGF_FLAG_BASE3)) {
+        if (launch_repack_b3(packed, d_out, d_in, (char *)workspace + L.w2, stream) != cudaSuccess) return HGF_ERR_CUDA;
+        packed2 = (char *)workspace + L.w2;
+    }
     GemmPrologueExtra gx = {};
     gx.tok_sc = (float *)((char *)workspace + L.tok_sc);
     gx.gb16 = r ? (__half *)((char *)workspace + L.gb16) : nullptr;
@@ -278,7 +285,7 @@ hgf_status hgf::forward_impl(const void *x, int64_t M, const void *packed, float
     if (!do_main) return HGF_OK;
     GemmParams gp = {};
     gp.xq = pp.xq;
-    gp.packed = (const uint8_t *)packed;
+    gp.packed = (const uint8_t *)packed2;
     gp.gamma_x = pp.gamma_x;
     gp.row_sum = pp.row_sum;
     gp.h16 = pp.h16;

@@ -65,12 +65,12 @@ static inline int64_t padded_k_b3(int64_t d_in) { return (d_in + 319) / 320 * 32
 // On the GEMM path the per-token arrays have room for M rounded up to 128: the kernel fetches them
 // 128 tokens at a time (what lies past M is never used).
 struct WsLayout {
-    size_t xq, gamma_x, row_sum, h, h_hi, h_lo, hpart, h16, tok_sc, gb16, total;
+    size_t xq, gamma_x, row_sum, h, h_hi, h_lo, hpart, h16, tok_sc, gb16, w2, total;
 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-static inline WsLayout ws_layout(int64_t M, int64_t d_in, int64_t d_out, int32_t r, bool gemm_path) {
+static inline WsLayout ws_layout(int64_t M, int64_t d_in, int64_t d_out, int32_t r, bool gemm_path, bool base3 = false) {
     WsLayout L;
     size_t off = 0;
     const size_t rr = (size_t)(r > 0 ? r : 1);
@@ -85,6 +85,8 @@ static inline WsLayout ws_layout(int64_t M, int64_t d_in, int64_t d_out, int32_t
     L.h16 = off;     off += gemm_path ? align_up((size_t)M * 64 * 2, 256) : 0;
     L.tok_sc = off;  off += gemm_path ? align_up(Mp * 4, 256) : 0;
     L.gb16 = off;    off += (gemm_path && r > 0) ? align_up((size_t)d_out * 64 * 2, 256) : 0;
+    // GEMM path on base-3 weights: the layer's two-bit tiles, rewritten from the base-3 bytes before the GEMM
+    L.w2 = off;      off += (gemm_path && base3) ? align_up((size_t)((d_out + 15) / 16) * (size_t)((d_in + 255) / 256) * 1024, 256) : 0;
     L.total = off ? off : 256;
     return L;
 }
@@ -210,6 +212,8 @@ cudaError_t launch_decode_prologue_group(const QuantItem *d_quant_items, int n_q
                                          const LoraItem *d_lora_items, int n_lora, int max_M, bool pdl,
                                          cudaStream_t stream);
 cudaError_t launch_gemm_prologue(const PrologueParams &p, const GemmPrologueExtra &x, cudaStream_t stream);
+// base-3 bytes of a layer -> its two-bit tiles (the GEMM path's weight format)
+cudaError_t launch_repack_b3(const void *packed_b3, int64_t d_out, int64_t d_in, void *packed2, cudaStream_t stream);
 cudaError_t launch_decode_gemv(const DecodeLaunch &L, const DecodeProblem *single, bool pdl, cudaStream_t stream);
 // Shared memory the decode kernel needs for one problem's activations, and the largest it accepts.
 int decode_xq_smem_bytes(int M, int K, uint32_t flags);

@@ -153,6 +153,43 @@ __global__ void __launch_bounds__(256) unpack_b3_kernel(const uint8_t *packed, i
     T[idx] = (int8_t)(c - 1);
 }
 
+// Base-3 bytes -> two-bit tiles (the GEMM path reads only those).  One thread per two-bit word: its sixteen
+// codes are digits of up to sixteen bytes of the row's 64 in the base-3 tile that holds those columns.
+__global__ void __launch_bounds__(256) repack_b3_kernel(const uint8_t *packed_b3, int64_t N, int64_t K, int64_t steps2, int64_t steps3,
+                                                        size_t n_words, uint32_t *packed2) {
+    const size_t w = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (w >= n_words) return;
+    const WordPos p = word_pos(w, steps2);
+    uint32_t word = 0x55555555u;
+    if (p.n < N && p.k0 < K) {
+        word = 0;
+        const uint8_t *row_base = packed_b3 + (size_t)(p.n / 16) * steps3 * 1024 + (size_t)(p.n % 16) * 64;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int64_t k = p.k0 + i;  // K is a multiple of 64: the word's sixteen columns are all inside the matrix
+            const int col = (int)(k % 320), q = 2 * (col / 32) + (col % 32) / 16, t = (col % 16) / 4, e = col % 4;
+            const int j = q < 16 ? q : 4 * (q - 16) + e, digit = q < 16 ? e : 4;
+            int v = row_base[(size_t)(k / 320) * 1024 + 16 * t + j];
+            int c = 1;
+            if (v <= 242) {
+                for (int d = 0; d < digit; ++d) v /= 3;
+                c = v % 3;
+            }
+            word |= (uint32_t)c << (8 * (i & 3) + 2 * (i >> 2));
+        }
+    }
+    packed2[w] = word;
+}
+
+cudaError_t launch_repack_b3(const void *packed_b3, int64_t d_out, int64_t d_in, void *packed2, cudaStream_t stream) {
+    const int64_t steps2 = padded_k(d_in) / 256, steps3 = padded_k_b3(d_in) / 320;
+    const size_t n_words = (size_t)row_tiles(d_out) * steps2 * 256;
+    repack_b3_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, stream>>>((const uint8_t *)packed_b3, d_out, d_in, steps2, steps3, n_words,
+                                                                            (uint32_t *)packed2);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // gamma_W = mean |W| into *gamma_dev (two launches; partials: kAbsBlocks doubles)
 static void enqueue_gamma(const float *W, size_t n, double *partials, float *gamma_dev, cudaStream_t stream) {
     abs_sum_partial_kernel<<<kAbsBlocks, kAbsThreads, 0, stream>>>((const float4 *)W, n / 4, partials);

@@ -82,14 +82,32 @@ def test_model_shapes(hgf, config, M):
         check(hgf, shape, M, config=config, layer=i)
 
 
-def test_bf16_output_and_gemm_path_is_refused(hgf):
-    shape = syn.LayerShape("b", 1024, 512, 32)
-    check(hgf, shape, 4, config=21, layer=200, flags=hgf.FLAG_OUT_BF16)
-    packed, gamma, _ = packed_b3(hgf, shape, 21, 200)
-    x = torch.zeros((64, 1024), dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(hgf.HgfError) as e:
-        hgf.linear_forward(x, packed, float(gamma), 1024, 512, flags=hgf.FLAG_BASE3)
-    assert e.value.status == 2
+def test_bf16_output(hgf):
+    check(hgf, syn.LayerShape("b", 1024, 512, 32), 4, config=21, layer=200, flags=hgf.FLAG_OUT_BF16)
+
+
+@pytest.mark.parametrize("M,K,N,r", [(64, 1024, 512, 32), (300, 2048, 2048, 32), (130, 5632, 264, 16), (257, 704, 1000, 64)])
+def test_gemm_path_on_base3_weights(hgf, M, K, N, r):
+    """More tokens than the decode path takes: the layer's two-bit tiles are rewritten from the base-3 bytes into
+    the workspace and the tensor-core kernel runs on those.  Integer accumulators bit for bit, y within the GEMM
+    path's tolerance; K = 704 and 5632 are not multiples of either tile width (256, 320), d_out = 264 and 1000
+    leave ragged row tiles."""
+    shape = syn.LayerShape("b", K, N, r)
+    packed, gamma, T = packed_b3(hgf, shape, 22, M)
+    x = syn.make_x(M, K, config=22, layer=M)
+    At, Bt, gate = syn.make_lora(K, N, r, config=22, layer=M)
+    y, dbg = hgf.linear_forward(dev(x, torch.bfloat16), packed, float(gamma), K, N, dev(At, torch.float16), dev(Bt, torch.float16),
+                                dev(gate), debug=True, flags=hgf.FLAG_BASE3)
+    hgf.check_status()
+    ref = oracle.forward(x, T, gamma, At, Bt, gate)
+    assert np.array_equal(dbg["xq"].cpu().numpy(), ref["xq"])
+    assert np.array_equal(dbg["y_int"].cpu().numpy(), ref["y_int"]), "int32 accumulators differ"
+    err = np.abs(y.float().cpu().numpy().astype(np.float64) - ref["y"]).max() / np.abs(ref["y"]).max()
+    assert err <= 6e-4, err
+    # and the same call on the two-bit weights gives the same bits
+    packed2, gamma2 = hgf.pack_ternary(dev(syn.make_weights(N, K, config=22, layer=M)))
+    y2 = hgf.linear_forward(dev(x, torch.bfloat16), packed2, float(gamma2), K, N, dev(At, torch.float16), dev(Bt, torch.float16), dev(gate))
+    assert torch.equal(y, y2)
 
 
 def test_group_on_base3_weights(hgf):
