@@ -939,11 +939,11 @@ __global__ void __launch_bounds__(kThreads, 4) round_rows_kernel(const PrologueP
     uint2 *dq = p.dbg_xq ? reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * K) : nullptr;
     int sum = 0;
     int i = lane;
-    for (; i + 32 < nv; i += 64) {  // two units in flight per lane
-        const uint4 v0 = xv[i], v1 = xv[i + 32];
-        const uint2 o0 = quant8(v0, qs, sum), o1 = quant8(v1, qs, sum);
-        qv[i] = o0; qv[i + 32] = o1;
-        if (dq) { dq[i] = o0; dq[i + 32] = o1; }
+    for (; i + 96 < nv; i += 128) {  // four units in flight per lane
+        const uint4 v0 = xv[i], v1 = xv[i + 32], v2 = xv[i + 64], v3 = xv[i + 96];
+        const uint2 o0 = quant8(v0, qs, sum), o1 = quant8(v1, qs, sum), o2 = quant8(v2, qs, sum), o3 = quant8(v3, qs, sum);
+        qv[i] = o0; qv[i + 32] = o1; qv[i + 64] = o2; qv[i + 96] = o3;
+        if (dq) { dq[i] = o0; dq[i + 32] = o1; dq[i + 64] = o2; dq[i + 96] = o3; }
     }
     for (; i < nv; i += 32) {
         const uint2 o = quant8(xv[i], qs, sum);
