@@ -464,7 +464,7 @@ DECODE_TRAFFIC = {"source_sha1": "7b2cc479563a0d062a4c3a356e67630e5471a690",
 # DRAM traffic of the prefill GEMM launch from one ncu capture of the very shape the bench times
 # (2048 -> 5632, r = 32, M = 8192, bf16 y): dram__bytes_read.sum + dram__bytes_write.sum of one launch.  Below
 # the launch's algorithmic bytes because most of y is still in L2 when the kernel ends.
-PREFILL_TRAFFIC = {"source_sha1": "1aa0a24ce7a1e6dbd36de8d29d9bd7518719bb4f", "dram_bytes_per_launch": 21.568768e6 + 43.333632e6}
+PREFILL_TRAFFIC = {"source_sha1": "8ff95e068f9752902d0b321377a47b0986601768", "dram_bytes_per_launch": 21.581312e6 + 43.126016e6}
 
 
 def prefill_traffic():
