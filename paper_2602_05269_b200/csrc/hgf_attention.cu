@@ -356,6 +356,8 @@ extern "C" hgf_status hgf_diff_attention_forward(const void *q, const void *k, c
     if (!q || !k || !v || !out || B <= 0 || L <= 0 || n_heads <= 0) return HGF_ERR_INVALID_ARG;
     if (flags & ~HGF_FLAG_OUT_BF16) return HGF_ERR_INVALID_ARG;
     if ((head_dim != 64 && head_dim != 128) || B > 65535 || n_heads > 65535 || L > (1 << 24)) return HGF_ERR_UNSUPPORTED_SHAPE;
+    // token rows and CTAs are counted in 32 bits
+    if (B * L > 0x7fffffffll || (uint64_t)B * (uint64_t)n_heads * (uint64_t)((L + kTaBM - 1) / kTaBM) > 0x7fffffffull) return HGF_ERR_UNSUPPORTED_SHAPE;
     if ((((uintptr_t)q) | ((uintptr_t)k) | ((uintptr_t)v) | ((uintptr_t)out)) & 15u) return HGF_ERR_MISALIGNED;
     AttnParams p = {};
     p.q = (const __nv_bfloat16 *)q;

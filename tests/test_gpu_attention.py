@@ -98,3 +98,6 @@ def test_rejects_bad_arguments(hgf):
     with pytest.raises(hgf.HgfError) as e:
         hgf.diff_attention_forward(q, q, q, 1, 64, 1, 96, 0.5)
     assert e.value.status == 2
+    # more token rows than the kernel's 32-bit row index covers: refused before anything is touched
+    ptr = q.data_ptr()
+    assert hgf.lib().hgf_diff_attention_forward(ptr, ptr, ptr, 40000, 1 << 20, 1, 64, 0.5, 1.0, ptr, 0, None) == 2
