@@ -336,7 +336,9 @@ hgf_status hgf_act_quant(const void *x, int64_t M, int64_t d_in, int8_t *xq, flo
  *          output projection)
  *   lambda the learnable scalar (hgf_diff_lambda0(head_dim) is its initial value 0.8 - 0.6 exp(-0.3 d_h));
  *   out_scale 1 for the Definition; the reference module of Appendix E multiplies by 0.5.
- * head_dim 64 or 128; 16-byte aligned pointers.  Enqueue only; no workspace.
+ * head_dim 64 or 128; B, n_heads <= 65535, L <= 2^24, B * L < 2^31 (else HGF_ERR_UNSUPPORTED_SHAPE); 16-byte
+ * aligned pointers.  Enqueue only; no workspace.  The probabilities enter the second product rounded to
+ * bfloat16 (fp32 accumulation); a bounded wait that ran out is reported by hgf_check_status.
  */
 hgf_status hgf_diff_attention_forward(const void *q, const void *k, const void *v, int64_t B, int64_t L,
                                       int32_t n_heads, int32_t head_dim, float lambda, float out_scale,
