@@ -444,7 +444,7 @@ def run_ours(args):
             "gpu_launches": main_summary["launches_per_step"] * args.steps,
             "clocks": clocks, "roofline": roofline, "roofline_prefill": roofline_prefill,
             "value_prefill": None if roofline_prefill is None else
-            {"value": roofline_prefill["layer"]["TOPS"], "unit": "int8 TOPS (2*M*K*N per layer call, prologue + GEMM)",
+            {"value": roofline_prefill["layer"]["TOPS"], "unit": "int8 TOPS (2*M*K*N per layer call: prologue, rounding and GEMM launches)",
              "frac_of_measured_int8_peak": roofline_prefill["layer"]["frac"], "clocks": prefill_clocks},
             "cpu_baseline": cpu, "extra": extra,
         }
