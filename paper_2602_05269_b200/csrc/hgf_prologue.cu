@@ -585,6 +585,38 @@ __device__ void warp_quant_row_ln(const QuantItem &q, int lane) {
     }
 }
 
+// The LayerNorm front end for many rows (the GEMM path): one warp per token row, eight rows per block, the
+// row's passes (mean, variance, largest |xn|, codes) all from L1 with warp shuffles between them - one block
+// per row spent its time in block-wide barriers between the passes.
+__global__ void __launch_bounds__(kThreads) ln_quant_rows_kernel(const PrologueParams p, const GemmPrologueExtra x, const FrontEnd fe) {
+    pdl_wait();
+    const int lane = threadIdx.x & 31, m = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (m >= p.M) return;
+    QuantItem q;
+    q.x = p.x + (size_t)m * p.K;
+    q.xq = p.xq + (size_t)m * p.K;
+    q.gamma_x = p.gamma_x + m;
+    q.row_sum = p.row_sum + m;
+    q.K = p.K;
+    q.eps = fe.eps;
+    q.ln_w = fe.ln_w;
+    q.ln_b = fe.ln_b;
+    q.mean_out = fe.dbg_mean ? fe.dbg_mean + m : nullptr;
+    q.rstd_out = fe.dbg_rstd ? fe.dbg_rstd + m : nullptr;
+    warp_quant_row_ln(q, lane);
+    __syncwarp();
+    if (lane == 0) {  // (reads back what this lane wrote)
+        const float g = p.gamma_x[m];
+        if (x.tok_sc) x.tok_sc[m] = g * x.gw_over_127;
+        if (p.dbg_gamma_x) p.dbg_gamma_x[m] = g;
+    }
+    if (p.dbg_xq) {  // each lane copies the units it wrote itself
+        const uint2 *qv = reinterpret_cast<const uint2 *>(q.xq);
+        uint2 *dq = reinterpret_cast<uint2 *>(p.dbg_xq + (size_t)m * p.K);
+        for (int i = lane; i < p.K / 8; i += 32) dq[i] = qv[i];
+    }
+}
+
 template <int NT>
 __global__ void __launch_bounds__(kPgThreads, 1)
 decode_prologue_group_kernel(const QuantItem *quant_items, int n_quant, const LoraItem *lora, int n_lora) {
@@ -1066,8 +1098,9 @@ cudaError_t launch_decode_prologue_ln(const PrologueParams &p, const FrontEnd &f
 
 cudaError_t launch_ln_quant(const PrologueParams &p, const GemmPrologueExtra &x, const FrontEnd &fe, cudaStream_t stream) {
     cudaLaunchAttribute attr[1];
-    cudaLaunchConfig_t cfg = prologue_cfg(p.M, !(p.flags & HGF_FLAG_NO_PDL), stream, attr);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, ln_quant_kernel, p, x, fe);
+    const bool by_warp = p.row_sum != nullptr && p.M >= 64;  // many rows: one warp each; few: one block each
+    cudaLaunchConfig_t cfg = prologue_cfg(by_warp ? (p.M + kWarps - 1) / kWarps : p.M, !(p.flags & HGF_FLAG_NO_PDL), stream, attr);
+    cudaError_t e = by_warp ? cudaLaunchKernelEx(&cfg, ln_quant_rows_kernel, p, x, fe) : cudaLaunchKernelEx(&cfg, ln_quant_kernel, p, x, fe);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }
